@@ -1,0 +1,132 @@
+/*
+ * loract.h -- C ABI of the LoRAct online activation-compression hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library compresses a saved activation matrix X (n_tokens x d, row-major, bf16 or fp32) to a
+ * rank-r factor pair (U, V) with the paper's sampling-based orthogonal decomposition (Algorithm 1),
+ * and serves the backward-pass consumers from the factors.  Notation: the paper's A (m x n), k and t
+ * are X (n_tokens x d), rank and power_iters here.
+ *
+ * Conventions common to every call
+ *   - Every pointer named X, U, V, G, dW, gamma, beta, A_out, rstd, mean, idx_*, ws is a DEVICE pointer
+ *     to memory the caller owns (allocate it with any CUDA allocator); the descriptor and the out_host
+ *     arguments are HOST pointers.  The library allocates no device memory and frees none.
+ *   - Matrices are row-major.  X has row stride ldx elements; U is n_tokens x rank (stride rank),
+ *     V is rank x d (stride d).  U, V, X_out, A_out have X's dtype.  dW is always fp32.
+ *   - Alignment: every matrix base pointer 16-byte aligned; d, ldx, ldg multiples of 8 (bf16) or
+ *     4 (fp32) elements, so that every row starts on a 16-byte boundary.
+ *   - rank: a multiple of 16, 16 <= rank <= 512, rank <= n_tokens and rank <= d.
+ *   - Calls are asynchronous on the CUDA stream passed as `stream` (a cudaStream_t cast to void*;
+ *     NULL is the default stream) and never synchronise, except loract_read_device_status.
+ *   - Host-detectable errors return a status and launch nothing.  Conditions found on the device (a
+ *     Cholesky pivot that had to be clamped, a bounded wait that expired) are recorded in a 32-bit word
+ *     at the start of `ws`; outputs are still fully written.  Read it with loract_read_device_status.
+ *   - `ws` is scratch of at least loract_workspace_bytes(desc) bytes, 256-byte aligned, private to one
+ *     in-flight call.  The same (seed, call_id, n_tokens, rank) always selects the same rows.
+ */
+#ifndef LORACT_H_
+#define LORACT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LORACT_OK = 0,
+  LORACT_ERR_INVALID_ARG = 1,
+  LORACT_ERR_UNSUPPORTED = 2,
+  LORACT_ERR_ALIGNMENT = 3,
+  LORACT_ERR_WORKSPACE_TOO_SMALL = 4,
+  LORACT_ERR_CUDA = 5,
+  LORACT_ERR_NUMERIC = 6,
+  LORACT_ERR_TIMEOUT = 7
+} loract_status_t;
+
+typedef enum { LORACT_F32 = 0, LORACT_BF16 = 1 } loract_dtype_t;
+typedef enum { LORACT_NORM_RMS = 0, LORACT_NORM_LAYER = 1 } loract_norm_t;
+
+/* Bits of the device status word (see loract_read_device_status). */
+#define LORACT_DEV_PIVOT_CLAMPED 0x1u  /* a Cholesky pivot was not positive and was clamped       */
+#define LORACT_DEV_WAIT_EXPIRED  0x2u  /* a bounded device-side wait gave up; results are invalid */
+#define LORACT_DEV_SAMPLER_SHORT 0x4u  /* the sampler could not find `rank` distinct rows          */
+#define LORACT_DEV_NONFINITE     0x8u  /* a non-finite value reached the small-block factorisation */
+
+typedef struct {
+  int64_t n_tokens;      /* rows of X (the paper's m)                                        */
+  int64_t d;             /* columns of X (the paper's n)                                     */
+  int64_t ldx;           /* row stride of X in elements, >= d                                */
+  int32_t rank;          /* r (the paper's k)                                                */
+  int32_t power_iters;   /* t of Algorithm 1; only 0 is implemented on the device            */
+  int32_t dtype;         /* loract_dtype_t of X, U, V, X_out, A_out, G, gamma, beta          */
+  int32_t reserved;      /* must be 0                                                        */
+  uint64_t seed;         /* Philox key                                                       */
+  uint64_t call_id;      /* Philox counter high words: distinguishes layer / step / rank     */
+} loract_desc_t;
+
+/* Bytes of scratch that loract_compress / loract_compress_prenorm / loract_weight_grad need for this
+ * descriptor (the maximum over the three).  Returns 0 if the descriptor is invalid. */
+size_t loract_workspace_bytes(const loract_desc_t* desc);
+
+/* Algorithm 1, line 1: the `rank` distinct row indices, uniform without replacement.  The sample is the
+ * first `rank` distinct values of the stream c_i = (w_i * n_tokens) >> 32, w_i = word (i mod 4) of the
+ * Philox4x32-10 block with key (seed lo, seed hi) and counter (i div 4, 0, call_id lo, call_id hi),
+ * in stream order.  idx_dev: device, `rank` int32, written.  ws: device scratch, >= 256 bytes. */
+loract_status_t loract_sample_indices(const loract_desc_t* desc, int32_t* idx_dev, void* ws,
+                                      size_t ws_bytes, void* stream);
+
+/* Algorithm 1 with t = 0: sample rows, Y = X A_k^T, orthonormalise Y to Q, U = Q, V = Q^T X.
+ * X: device, read only.  U (n_tokens x rank), V (rank x d): device, written.  idx_out: device, `rank`
+ * int32, written if not NULL.  U has orthonormal columns; U V is the orthogonal projection of X onto
+ * range(Y).  The entries of U are not unique (any orthonormal basis of range(Y) is a valid result). */
+loract_status_t loract_compress(const loract_desc_t* desc, const void* X, void* U, void* V,
+                                int32_t* idx_out, void* ws, size_t ws_bytes, void* stream);
+
+/* Section 3.1, Reconstruct: X_out = U V (n_tokens x d, row stride ldx, dtype of the descriptor). */
+loract_status_t loract_reconstruct(const loract_desc_t* desc, const void* U, const void* V,
+                                   void* X_out, void* stream);
+
+/* Section 3.1, the gradient taken at the reconstructed activation, for a linear consumer Z = X W:
+ * dW = (U V)^T G, evaluated as V^T (U^T G) so that U V is never formed.  G: device, n_tokens x g, row
+ * stride ldg, dtype of the descriptor; several consumers can be served by one call with their
+ * gradients concatenated along columns.  1 <= g <= 256.  dW: device, d x g fp32, row stride g; if
+ * `accumulate` is non-zero the result is added to dW, otherwise dW is overwritten. */
+loract_status_t loract_weight_grad(const loract_desc_t* desc, const void* U, const void* V,
+                                   const void* G, int32_t g, int64_t ldg, float* dW, int accumulate,
+                                   void* ws, size_t ws_bytes, void* stream);
+
+/* Section 3.3, the pre-norm unit: A = Norm(X) is computed once, compressed once, and that one factor
+ * pair serves the Norm backward and every projection inside the sub-layer.
+ *   RMS   : A = X * rstd * gamma,           rstd_i = 1 / sqrt(mean_j X_ij^2 + eps)
+ *   LAYER : A = (X - mean_i) * rstd_i * gamma + beta   (textbook LayerNorm; beta may be NULL)
+ * gamma, beta: device, d elements, dtype of the descriptor.  rstd: device, n_tokens fp32, written.
+ * mean: device, n_tokens fp32, written for LAYER (may be NULL for RMS).  A_out: device, n_tokens x d with
+ * row stride d, written if not NULL (the forward pass needs it as the sub-layer input); if NULL the
+ * normalised matrix lives only in `ws`.  U, V, ws, stream as for loract_compress; (U, V) factor A. */
+loract_status_t loract_compress_prenorm(const loract_desc_t* desc, const void* X, const void* gamma,
+                                        const void* beta, float eps, int32_t kind, void* A_out,
+                                        float* rstd, float* mean, void* U, void* V, int32_t* idx_out,
+                                        void* ws, size_t ws_bytes, void* stream);
+
+/* Comparator of Section 3.2: randomized SVD at the same rank -- Algorithm 1 with a Gaussian test matrix
+ * of rank + oversample columns (Philox + Box-Muller, counter word 1 set to 1) and `power_iters`
+ * iterations of Y = X (X^T Q).  Writes the un-truncated pair: Uq (n_tokens x l), B (l x d), l = rank +
+ * oversample (a multiple of 16, <= 512).  bf16 only.  ws must hold loract_rsvd_workspace_bytes. */
+size_t loract_rsvd_workspace_bytes(const loract_desc_t* desc, int32_t oversample);
+loract_status_t loract_rsvd(const loract_desc_t* desc, int32_t oversample, const void* X, void* Uq,
+                            void* B, void* ws, size_t ws_bytes, void* stream);
+
+/* Copies the device status word at the start of `ws` to *out_host.  Synchronises `stream`. */
+loract_status_t loract_read_device_status(const void* ws, uint32_t* out_host, void* stream);
+
+const char* loract_status_string(loract_status_t s);
+
+/* Number of kernels the library has launched in this process (all entry points); the benchmark
+ * reports the difference across its timed region. */
+uint64_t loract_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LORACT_H_ */

@@ -1,0 +1,43 @@
+/*
+ * loract_debug.h -- test hooks of libloract: the two building blocks every entry point of loract.h is
+ * composed of, exported so that the GPU tests can check them in isolation.  Not part of the stable ABI.
+ * All pointers are DEVICE pointers owned by the caller unless stated; calls are asynchronous on `stream`.
+ */
+#ifndef LORACT_DEBUG_H_
+#define LORACT_DEBUG_H_
+
+#include "loract.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* The contraction behind Algorithm 1 lines 2 and 8 and behind Reconstruct:
+ * C (M x N) = sum_{t < n_terms} A_t B_t, contraction length K, fp32 accumulation.
+ * a_mn = 0: A_t stored [M][K] (row stride lda); a_mn = 1: stored [K][M].  b_mn = 0: B_t stored [N][K]
+ * (row stride ldb); b_mn = 1: stored [K][N].  a_type / b_type: 0 fp32, 1 bf16.  A and B point to
+ * n_terms operand pointers each (HOST arrays of device pointers).  out_mode: 0 fp32 into C0, 1 bf16 into
+ * C0, 2 bf16 hi/lo pair into C0/C1, 3 fp64 into C0 (CUDA-core kernel only).  splits > 1 writes `splits`
+ * partial results `split_stride` elements apart (fp32/fp64 only).  engine: 0 CUDA-core kernel, 1 tensor-core
+ * (tcgen05) kernel -- returns LORACT_ERR_UNSUPPORTED if that kernel does not take the shape or types.
+ * status_word: device uint32 that receives LORACT_DEV_* bits, may be NULL. */
+loract_status_t loract_debug_gemm(int32_t M, int32_t N, int32_t K, int32_t a_mn, int32_t b_mn,
+                                  const void* const* A, int64_t lda, const void* const* B, int64_t ldb,
+                                  int32_t a_type, int32_t b_type, int32_t n_terms, int32_t out_mode,
+                                  void* C0, void* C1, int64_t ldc, int32_t splits, int64_t split_stride,
+                                  int32_t acc64, int32_t engine, uint32_t* status_word, void* stream);
+
+/* The small-block step of the orthonormalisation (Algorithm 1 line 7 done through Gram matrices):
+ * W = sum of n_partials r x r matrices (fp32 if partial_f64 == 0, else fp64; `partial_stride` elements
+ * apart); L L^T = W + shift_rel * mean(diag W) * I; writes L^{-1} (lower triangular, row-major) as fp32
+ * (linv_f32), as a bf16 hi/lo pair (linv_hi, linv_lo), any of which may be NULL.  use_f64 selects the
+ * arithmetic.  scratch: 2 * (r*r + 32*r) elements of the compute type.  r a multiple of 16, <= 512. */
+loract_status_t loract_debug_small_block(int32_t r, const void* partials, int32_t partial_f64,
+                                         int32_t n_partials, int64_t partial_stride, int32_t use_f64,
+                                         float shift_rel, void* scratch, float* linv_f32, void* linv_hi,
+                                         void* linv_lo, uint32_t* status_word, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LORACT_DEBUG_H_ */

@@ -1,0 +1,298 @@
+"""Thin ctypes binding of libloract.so.
+
+Argument marshalling only: every step of the path runs in the CUDA kernels of the library.
+PyTorch is used for device memory and streams.  There is no CPU fallback: if the library cannot be
+loaded, or a tensor is not on a CUDA device, the call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libloract.so")
+
+F32, BF16 = 0, 1
+NORM_RMS, NORM_LAYER = 0, 1
+DEV_PIVOT_CLAMPED, DEV_WAIT_EXPIRED, DEV_SAMPLER_SHORT, DEV_NONFINITE = 1, 2, 4, 8
+
+EXPORTS = (
+    "loract_workspace_bytes", "loract_sample_indices", "loract_compress", "loract_reconstruct",
+    "loract_weight_grad", "loract_compress_prenorm", "loract_rsvd_workspace_bytes", "loract_rsvd",
+    "loract_read_device_status", "loract_status_string", "loract_kernel_launch_count",
+)
+
+
+class Desc(ctypes.Structure):
+    _fields_ = [("n_tokens", ctypes.c_int64), ("d", ctypes.c_int64), ("ldx", ctypes.c_int64),
+                ("rank", ctypes.c_int32), ("power_iters", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("seed", ctypes.c_uint64), ("call_id", ctypes.c_uint64)]
+
+
+class LoractError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: status {code} ({status_string(code)})")
+        self.code = code
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the library (building nothing: run ``__graft_entry__.build()`` or ``build.py`` first)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2509_23472_b200.build`")
+        l = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+        dp = ctypes.POINTER(Desc)
+        l.loract_workspace_bytes.restype = sz
+        l.loract_workspace_bytes.argtypes = [dp]
+        l.loract_sample_indices.restype = ctypes.c_int
+        l.loract_sample_indices.argtypes = [dp, vp, vp, sz, vp]
+        l.loract_compress.restype = ctypes.c_int
+        l.loract_compress.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp]
+        l.loract_reconstruct.restype = ctypes.c_int
+        l.loract_reconstruct.argtypes = [dp, vp, vp, vp, vp]
+        l.loract_weight_grad.restype = ctypes.c_int
+        l.loract_weight_grad.argtypes = [dp, vp, vp, vp, i32, i64, vp, ctypes.c_int, vp, sz, vp]
+        l.loract_compress_prenorm.restype = ctypes.c_int
+        l.loract_compress_prenorm.argtypes = [dp, vp, vp, vp, ctypes.c_float, i32, vp, vp, vp, vp, vp, vp,
+                                              vp, sz, vp]
+        l.loract_rsvd_workspace_bytes.restype = sz
+        l.loract_rsvd_workspace_bytes.argtypes = [dp, i32]
+        l.loract_rsvd.restype = ctypes.c_int
+        l.loract_rsvd.argtypes = [dp, i32, vp, vp, vp, vp, sz, vp]
+        l.loract_read_device_status.restype = ctypes.c_int
+        l.loract_read_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
+        l.loract_status_string.restype = ctypes.c_char_p
+        l.loract_status_string.argtypes = [ctypes.c_int]
+        l.loract_kernel_launch_count.restype = ctypes.c_uint64
+        l.loract_kernel_launch_count.argtypes = []
+        _lib = l
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().loract_status_string(code).decode()
+
+
+def kernel_launch_count() -> int:
+    return int(lib().loract_kernel_launch_count())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _cuda(t: torch.Tensor, what: str) -> torch.Tensor:
+    if not t.is_cuda:
+        raise RuntimeError(f"{what} must live on a CUDA device (there is no CPU path)")
+    return t
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(dev) -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream(dev).cuda_stream)
+
+
+def make_desc(X: torch.Tensor, rank: int, seed: int = 0, call_id: int = 0, power_iters: int = 0) -> Desc:
+    if X.dim() != 2 or X.stride(1) != 1:
+        raise ValueError("X must be a 2-D row-major tensor")
+    return Desc(X.shape[0], X.shape[1], X.stride(0), rank, power_iters, _dtype_code(X), 0,
+                seed & 0xFFFFFFFFFFFFFFFF, call_id & 0xFFFFFFFFFFFFFFFF)
+
+
+def desc_for(n_tokens: int, d: int, rank: int, dtype: torch.dtype, seed: int = 0, call_id: int = 0) -> Desc:
+    return Desc(n_tokens, d, d, rank, 0, BF16 if dtype == torch.bfloat16 else F32, 0, seed, call_id)
+
+
+def workspace_bytes(desc: Desc) -> int:
+    return int(lib().loract_workspace_bytes(ctypes.byref(desc)))
+
+
+def alloc_workspace(desc: Desc, device) -> torch.Tensor:
+    n = workspace_bytes(desc)
+    if n == 0:
+        raise LoractError(1, "loract_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def _check(code: int, what: str):
+    if code != 0:
+        raise LoractError(code, what)
+
+
+def sample_indices(desc: Desc, device, ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+    idx = torch.empty(desc.rank, dtype=torch.int32, device=device)
+    ws = ws if ws is not None else torch.empty(256, dtype=torch.uint8, device=device)
+    _check(lib().loract_sample_indices(ctypes.byref(desc), _ptr(idx), _ptr(ws), ws.numel(), _stream(device)),
+           "loract_sample_indices")
+    return idx
+
+
+def compress(X: torch.Tensor, rank: int, seed: int = 0, call_id: int = 0, ws: Optional[torch.Tensor] = None,
+             out: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None, desc: Optional[Desc] = None):
+    """Algorithm 1 (t = 0).  Returns (U, V, idx)."""
+    _cuda(X, "X")
+    desc = desc or make_desc(X, rank, seed, call_id)
+    ws = ws if ws is not None else alloc_workspace(desc, X.device)
+    if out is None:
+        U = torch.empty(X.shape[0], rank, dtype=X.dtype, device=X.device)
+        V = torch.empty(rank, X.shape[1], dtype=X.dtype, device=X.device)
+        idx = torch.empty(rank, dtype=torch.int32, device=X.device)
+    else:
+        U, V, idx = out
+    _check(lib().loract_compress(ctypes.byref(desc), _ptr(X), _ptr(U), _ptr(V), _ptr(idx), _ptr(ws), ws.numel(),
+                                 _stream(X.device)), "loract_compress")
+    return U, V, idx
+
+
+def reconstruct(U: torch.Tensor, V: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """X~ = U V."""
+    _cuda(U, "U"); _cuda(V, "V")
+    n, r = U.shape
+    d = V.shape[1]
+    out = out if out is not None else torch.empty(n, d, dtype=U.dtype, device=U.device)
+    desc = Desc(n, d, out.stride(0), r, 0, _dtype_code(U), 0, 0, 0)
+    _check(lib().loract_reconstruct(ctypes.byref(desc), _ptr(U), _ptr(V), _ptr(out), _stream(U.device)),
+           "loract_reconstruct")
+    return out
+
+
+def weight_grad(U: torch.Tensor, V: torch.Tensor, G: torch.Tensor, dW: Optional[torch.Tensor] = None,
+                accumulate: bool = False, ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dW = (U V)^T G from the factors, fp32 (d x g)."""
+    _cuda(U, "U"); _cuda(V, "V"); _cuda(G, "G")
+    n, r = U.shape
+    d = V.shape[1]
+    g = G.shape[1]
+    if G.stride(1) != 1:
+        raise ValueError("G must be row-major")
+    desc = Desc(n, d, d, r, 0, _dtype_code(U), 0, 0, 0)
+    ws = ws if ws is not None else alloc_workspace(desc, U.device)
+    if dW is None:
+        dW = torch.zeros(d, g, dtype=torch.float32, device=U.device) if accumulate else \
+            torch.empty(d, g, dtype=torch.float32, device=U.device)
+    _check(lib().loract_weight_grad(ctypes.byref(desc), _ptr(U), _ptr(V), _ptr(G), g, G.stride(0), _ptr(dW),
+                                    1 if accumulate else 0, _ptr(ws), ws.numel(), _stream(U.device)),
+           "loract_weight_grad")
+    return dW
+
+
+def compress_prenorm(X: torch.Tensor, gamma: torch.Tensor, beta: Optional[torch.Tensor], eps: float, kind: int,
+                     rank: int, seed: int = 0, call_id: int = 0, want_A: bool = True,
+                     ws: Optional[torch.Tensor] = None):
+    """Pre-norm unit: A = Norm(X), compressed once.  Returns (A or None, rstd, mean or None, U, V, idx)."""
+    _cuda(X, "X"); _cuda(gamma, "gamma")
+    desc = make_desc(X, rank, seed, call_id)
+    ws = ws if ws is not None else alloc_workspace(desc, X.device)
+    n, d = X.shape
+    A = torch.empty(n, d, dtype=X.dtype, device=X.device) if want_A else None
+    rstd = torch.empty(n, dtype=torch.float32, device=X.device)
+    mean = torch.empty(n, dtype=torch.float32, device=X.device) if kind == NORM_LAYER else None
+    U = torch.empty(n, rank, dtype=X.dtype, device=X.device)
+    V = torch.empty(rank, d, dtype=X.dtype, device=X.device)
+    idx = torch.empty(rank, dtype=torch.int32, device=X.device)
+    _check(lib().loract_compress_prenorm(ctypes.byref(desc), _ptr(X), _ptr(gamma), _ptr(beta), eps, kind, _ptr(A),
+                                         _ptr(rstd), _ptr(mean), _ptr(U), _ptr(V), _ptr(idx), _ptr(ws),
+                                         ws.numel(), _stream(X.device)), "loract_compress_prenorm")
+    return A, rstd, mean, U, V, idx
+
+
+def rsvd(X: torch.Tensor, rank: int, oversample: int = 8, power_iters: int = 1, seed: int = 0, call_id: int = 0,
+         ws: Optional[torch.Tensor] = None):
+    """Randomized SVD comparator: returns the un-truncated pair (Q (n x l), B (l x d)), l = rank + oversample."""
+    _cuda(X, "X")
+    desc = make_desc(X, rank, seed, call_id, power_iters)
+    d0 = make_desc(X, rank, seed, call_id, 0)
+    need = int(lib().loract_rsvd_workspace_bytes(ctypes.byref(d0), oversample))
+    if need == 0:
+        raise LoractError(1, "loract_rsvd_workspace_bytes")
+    ws = ws if ws is not None else torch.empty(need, dtype=torch.uint8, device=X.device)
+    l = rank + oversample
+    Q = torch.empty(X.shape[0], l, dtype=X.dtype, device=X.device)
+    B = torch.empty(l, X.shape[1], dtype=X.dtype, device=X.device)
+    _check(lib().loract_rsvd(ctypes.byref(desc), oversample, _ptr(X), _ptr(Q), _ptr(B), _ptr(ws), ws.numel(),
+                             _stream(X.device)), "loract_rsvd")
+    return Q, B
+
+
+def read_device_status(ws: torch.Tensor) -> int:
+    out = ctypes.c_uint32(0)
+    _check(lib().loract_read_device_status(_ptr(ws), ctypes.byref(out), _stream(ws.device)),
+           "loract_read_device_status")
+    return int(out.value)
+
+
+# ---------------------------------------------------------------------------------------------
+# Test hooks (include/loract_debug.h)
+# ---------------------------------------------------------------------------------------------
+OUT_F32, OUT_BF16, OUT_SPLIT, OUT_F64 = 0, 1, 2, 3
+DEBUG_EXPORTS = ("loract_debug_gemm", "loract_debug_small_block")
+
+
+def _debug_lib():
+    l = lib()
+    if not getattr(l, "_debug_ready", False):
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+        l.loract_debug_gemm.restype = ctypes.c_int
+        l.loract_debug_gemm.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(vp), i64, ctypes.POINTER(vp), i64,
+                                        i32, i32, i32, i32, vp, vp, i64, i32, i64, i32, i32, vp, vp]
+        l.loract_debug_small_block.restype = ctypes.c_int
+        l.loract_debug_small_block.argtypes = [i32, vp, i32, i32, i64, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp]
+        l._debug_ready = True
+    return l
+
+
+def debug_gemm(A_terms, B_terms, M: int, N: int, K: int, a_mn: bool, b_mn: bool, out_mode: int = OUT_F32,
+               engine: int = 1, splits: int = 1, acc64: bool = False, status: Optional[torch.Tensor] = None):
+    """C = sum_t A_t B_t through one of the two contraction kernels.  Operands are 2-D row-major tensors
+    stored [M][K] / [K][M] (a_mn) and [N][K] / [K][N] (b_mn).  Returns C (or (hi, lo), or the partials)."""
+    l = _debug_lib()
+    dev = A_terms[0].device
+    nt = len(A_terms)
+    PA = (ctypes.c_void_p * nt)(*[a.data_ptr() for a in A_terms])
+    PB = (ctypes.c_void_p * nt)(*[b.data_ptr() for b in B_terms])
+    tcode = lambda t: {torch.float32: 0, torch.bfloat16: 1}[t.dtype]
+    if out_mode == OUT_F32:
+        C0 = torch.zeros(splits, M, N, dtype=torch.float32, device=dev); C1 = None
+    elif out_mode == OUT_F64:
+        C0 = torch.zeros(splits, M, N, dtype=torch.float64, device=dev); C1 = None
+    elif out_mode == OUT_BF16:
+        C0 = torch.zeros(M, N, dtype=torch.bfloat16, device=dev); C1 = None
+    else:
+        C0 = torch.zeros(M, N, dtype=torch.bfloat16, device=dev); C1 = torch.zeros_like(C0)
+    _check(l.loract_debug_gemm(M, N, K, int(a_mn), int(b_mn), PA, A_terms[0].stride(0), PB, B_terms[0].stride(0),
+                               tcode(A_terms[0]), tcode(B_terms[0]), nt, out_mode, _ptr(C0), _ptr(C1), N, splits,
+                               M * N, int(acc64), engine, _ptr(status), _stream(dev)), "loract_debug_gemm")
+    if out_mode in (OUT_F32, OUT_F64):
+        return C0 if splits > 1 else C0[0]
+    return C0 if C1 is None else (C0, C1)
+
+
+def debug_small_block(partials: torch.Tensor, use_f64: bool, shift_rel: float,
+                      status: Optional[torch.Tensor] = None):
+    """partials: (n_partials, r, r) fp32 or fp64.  Returns (Linv fp32, hi bf16, lo bf16)."""
+    l = _debug_lib()
+    dev = partials.device
+    n_p, r, _ = partials.shape
+    scratch = torch.empty(2 * (r * r + 32 * r), dtype=torch.float64 if use_f64 else torch.float32, device=dev)
+    L32 = torch.zeros(r, r, dtype=torch.float32, device=dev)
+    Lh = torch.zeros(r, r, dtype=torch.bfloat16, device=dev)
+    Ll = torch.zeros(r, r, dtype=torch.bfloat16, device=dev)
+    _check(l.loract_debug_small_block(r, _ptr(partials), int(partials.dtype == torch.float64), n_p, r * r,
+                                      int(use_f64), shift_rel, _ptr(scratch), _ptr(L32), _ptr(Lh), _ptr(Ll),
+                                      _ptr(status), _stream(dev)), "loract_debug_small_block")
+    return L32, Lh, Ll

@@ -1,0 +1,519 @@
+// The C ABI (include/loract.h): argument checks, workspace carving and the sequence of kernel launches
+// of each entry point.  All arithmetic happens in the kernels of the other translation units.
+#include <atomic>
+#include <cstring>
+
+#include "common.cuh"
+#include "../../include/loract_debug.h"
+
+namespace loract {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// relative diagonal shifts of the three Cholesky factorisations (fp32 small blocks)
+constexpr float kShiftSample = 1e-6f;  // Gram of the sampled rows
+constexpr float kShiftFirst = 3e-6f;   // first Gram of the sketch
+constexpr float kShiftSecond = 1e-7f;  // second Gram (already close to the identity)
+
+struct Carver {
+  unsigned char* base;
+  size_t off = 0;
+  explicit Carver(void* p) : base((unsigned char*)p) {}
+  void* take(size_t bytes) {
+    void* r = base ? base + off : nullptr;
+    off += align_up(bytes);
+    return r;
+  }
+};
+
+loract_status_t check_desc(const loract_desc_t* d) {
+  if (!d) return LORACT_ERR_INVALID_ARG;
+  if (d->dtype != LORACT_F32 && d->dtype != LORACT_BF16) return LORACT_ERR_INVALID_ARG;
+  if (d->reserved != 0) return LORACT_ERR_INVALID_ARG;
+  if (d->n_tokens < 1 || d->d < 1 || d->ldx < d->d) return LORACT_ERR_INVALID_ARG;
+  if (d->n_tokens > 0x7fffffffLL || d->d > 0x7fffffffLL) return LORACT_ERR_INVALID_ARG;
+  if (d->rank < 16 || d->rank > 512 || d->rank % 16) return LORACT_ERR_INVALID_ARG;
+  if (d->rank > d->n_tokens || d->rank > d->d) return LORACT_ERR_INVALID_ARG;
+  if (d->power_iters < 0) return LORACT_ERR_INVALID_ARG;
+  if (d->power_iters != 0) return LORACT_ERR_UNSUPPORTED;
+  const int64_t mult = d->dtype == LORACT_BF16 ? 8 : 4;
+  if (d->d % mult || d->ldx % mult) return LORACT_ERR_ALIGNMENT;
+  return LORACT_OK;
+}
+inline bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
+inline int elem_bytes(const loract_desc_t* d) { return d->dtype == LORACT_BF16 ? 2 : 4; }
+
+// Workspace of the orthonormalisation + projection of an (n x d) matrix against an l-row test matrix.
+struct BasisWs {
+  // bf16 path
+  __nv_bfloat16 *Lh, *Ll, *Yh, *Yl, *Qh, *Ql;
+  float* gram_partials;
+  float* v_partials;
+  void* sb_scratch;
+  // fp32 path
+  float *Linv32, *Y32, *Q32;
+  double* gram64;
+  int splits_gram_sample, splits_gram, splits_v;
+};
+
+struct Plan {
+  int64_t n, d;
+  int l;
+  bool bf16;
+  int splits_gs, splits_w, splits_v;
+};
+
+Plan make_plan(int64_t n, int64_t d, int l, bool bf16) {
+  Plan p;
+  p.n = n; p.d = d; p.l = l; p.bf16 = bf16;
+  if (bf16) {
+    p.splits_gs = gemm_tc_pick_splits(l, l, (int)d, false, false);
+    p.splits_w = gemm_tc_pick_splits(l, l, (int)n, true, true);
+    p.splits_v = gemm_tc_pick_splits(l, (int)d, (int)n, true, true);
+  } else {
+    p.splits_gs = p.splits_w = p.splits_v = 1;
+  }
+  return p;
+}
+
+void carve_basis(Carver& c, const Plan& p, BasisWs* w) {
+  std::memset(w, 0, sizeof(*w));
+  const size_t l = (size_t)p.l, n = (size_t)p.n, d = (size_t)p.d;
+  w->splits_gram_sample = p.splits_gs; w->splits_gram = p.splits_w; w->splits_v = p.splits_v;
+  if (p.bf16) {
+    w->Lh = (__nv_bfloat16*)c.take(l * l * 2);
+    w->Ll = (__nv_bfloat16*)c.take(l * l * 2);
+    w->sb_scratch = c.take((l * l + l * 32) * sizeof(float));
+    const size_t gs = (size_t)(p.splits_gs > p.splits_w ? p.splits_gs : p.splits_w);
+    w->gram_partials = (float*)c.take(gs * l * l * 4);
+    w->Yh = (__nv_bfloat16*)c.take(n * l * 2);
+    w->Yl = (__nv_bfloat16*)c.take(n * l * 2);
+    w->Qh = (__nv_bfloat16*)c.take(n * l * 2);
+    w->Ql = (__nv_bfloat16*)c.take(n * l * 2);
+    w->v_partials = (float*)c.take((p.splits_v > 1 ? (size_t)p.splits_v : 0) * l * d * 4);
+  } else {
+    w->Linv32 = (float*)c.take(l * l * 4);
+    w->sb_scratch = c.take((l * l + l * 32) * sizeof(double));
+    w->gram64 = (double*)c.take(l * l * 8);
+    w->Y32 = (float*)c.take(n * l * 4);
+    w->Q32 = (float*)c.take(n * l * 4);
+  }
+}
+
+cudaError_t run_gemm(const GemmDesc& g, uint32_t* status, cudaStream_t stream) {
+  if (gemm_tc_supported(g)) return gemm_tc_launch(g, status, stream);
+  return gemm_simt_launch(g, stream);
+}
+
+// r x r Gram partials of a K-major matrix S (l x d): S S^T.
+cudaError_t gram_rows(const void* S, int l, int64_t d, bool bf16, const BasisWs& w, uint32_t* status,
+                      cudaStream_t stream) {
+  GemmDesc g;
+  g.M = l; g.N = l; g.K = (int)d; g.lda = d; g.ldb = d;
+  g.a_type = g.b_type = bf16 ? ELEM_BF16 : ELEM_F32;
+  g.terms[0] = {S, S};
+  g.ldc = l;
+  if (bf16) {
+    g.out = OUT_F32; g.C0 = w.gram_partials; g.splits = w.splits_gram_sample;
+    g.split_stride = (int64_t)l * l;
+  } else {
+    g.out = OUT_F64; g.C0 = w.gram64; g.acc64 = true;
+  }
+  return run_gemm(g, status, stream);
+}
+
+cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs& w, uint32_t* status,
+                   cudaStream_t stream) {
+  SmallBlockArgs a;
+  a.r = l;
+  a.scratch = w.sb_scratch;
+  a.dev_status = status;
+  if (bf16) {
+    a.partials = w.gram_partials; a.partial_type = ELEM_F32; a.n_partials = n_partials;
+    a.partial_stride = (int64_t)l * l;
+    a.use_f64 = false; a.shift_rel = shift;
+    a.linv_hi = w.Lh; a.linv_lo = w.Ll;
+  } else {
+    a.partials = w.gram64; a.partial_type = ELEM_F64; a.n_partials = 1; a.partial_stride = 0;
+    a.use_f64 = true; a.shift_rel = shift * 1e-8f;
+    a.linv_f32 = w.Linv32;
+  }
+  return small_block_launch(a, stream);
+}
+
+// Lines 2 and 7 of Algorithm 1 for a test matrix Omega (l x d, rows are the test vectors):
+// Y = X Omega^T, then two rounds of { W = Y^T Y = L L^T ; Y <- Y L^{-T} }.  U (n x l) receives Q.
+cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* Omega, void* U,
+                        const BasisWs& w, uint32_t* status, cudaStream_t stream) {
+  const int l = p.l;
+  const int n = (int)p.n;
+  const int el = p.bf16 ? ELEM_BF16 : ELEM_F32;
+  {  // Y = X Omega^T
+    GemmDesc g;
+    g.M = n; g.N = l; g.K = (int)p.d; g.lda = ldx; g.ldb = p.d; g.a_type = g.b_type = el;
+    g.terms[0] = {X, Omega};
+    g.ldc = l;
+    if (p.bf16) { g.out = OUT_SPLIT; g.C0 = w.Yh; g.C1 = w.Yl; } else { g.out = OUT_F32; g.C0 = w.Y32; }
+    LORACT_CUDA_TRY(run_gemm(g, status, stream));
+  }
+  for (int round = 0; round < 2; ++round) {
+    const void* Yh = p.bf16 ? (const void*)(round ? w.Qh : w.Yh) : (const void*)(round ? w.Q32 : w.Y32);
+    const void* Yl = round ? w.Ql : w.Yl;
+    {  // W = Y^T Y
+      GemmDesc g;
+      g.M = l; g.N = l; g.K = n; g.a_mn = true; g.b_mn = true; g.lda = l; g.ldb = l;
+      g.a_type = g.b_type = el;
+      g.ldc = l;
+      if (p.bf16) {
+        g.n_terms = 3;
+        g.terms[0] = {Yh, Yh}; g.terms[1] = {Yh, Yl}; g.terms[2] = {Yl, Yh};
+        g.out = OUT_F32; g.C0 = w.gram_partials; g.splits = w.splits_gram; g.split_stride = (int64_t)l * l;
+      } else {
+        g.terms[0] = {Yh, Yh};
+        g.out = OUT_F64; g.C0 = w.gram64; g.acc64 = true;
+      }
+      LORACT_CUDA_TRY(run_gemm(g, status, stream));
+    }
+    LORACT_CUDA_TRY(factor(l, p.bf16, w.splits_gram, round ? kShiftSecond : kShiftFirst, w, status, stream));
+    {  // Y <- Y L^{-T}:  C[m][j] = sum_k Y[m][k] Linv[j][k]
+      GemmDesc g;
+      g.M = n; g.N = l; g.K = l; g.lda = l; g.ldb = l; g.a_type = g.b_type = el;
+      g.ldc = l;
+      if (p.bf16) {
+        g.n_terms = 3;
+        g.terms[0] = {Yh, w.Lh}; g.terms[1] = {Yh, w.Ll}; g.terms[2] = {Yl, w.Lh};
+        if (round == 0) { g.out = OUT_SPLIT; g.C0 = w.Qh; g.C1 = w.Ql; } else { g.out = OUT_BF16; g.C0 = U; }
+      } else {
+        g.terms[0] = {Yh, w.Linv32};
+        g.out = OUT_F32; g.C0 = round == 0 ? (void*)w.Q32 : U;
+      }
+      LORACT_CUDA_TRY(run_gemm(g, status, stream));
+    }
+  }
+  return cudaSuccess;
+}
+
+// Line 8 of Algorithm 1: V = U^T X  (l x d), from the stored U.
+cudaError_t project(const void* U, const void* X, int64_t ldx, const Plan& p, void* V, const BasisWs& w,
+                    uint32_t* status, cudaStream_t stream) {
+  GemmDesc g;
+  g.M = p.l; g.N = (int)p.d; g.K = (int)p.n; g.a_mn = true; g.b_mn = true; g.lda = p.l; g.ldb = ldx;
+  g.a_type = g.b_type = p.bf16 ? ELEM_BF16 : ELEM_F32;
+  g.terms[0] = {U, X};
+  g.ldc = p.d;
+  if (!p.bf16) { g.out = OUT_F32; g.C0 = V; return run_gemm(g, status, stream); }
+  if (w.splits_v <= 1) { g.out = OUT_BF16; g.C0 = V; return run_gemm(g, status, stream); }
+  g.out = OUT_F32; g.C0 = w.v_partials; g.splits = w.splits_v; g.split_stride = (int64_t)p.l * p.d;
+  LORACT_CUDA_TRY(run_gemm(g, status, stream));
+  return reduce_partials_launch(w.v_partials, w.splits_v, g.split_stride, g.split_stride, nullptr,
+                                (__nv_bfloat16*)V, stream);
+}
+
+// ------------------------------------------------------------------ compress
+struct CompressWs {
+  uint32_t* status;
+  int32_t* idx;
+  void* S;      // sampled rows, l x d
+  void* Omega;  // preconditioned test matrix, l x d
+  void* A;      // normalised input of the pre-norm entry (only when it is not returned)
+  BasisWs b;
+};
+
+size_t carve_compress(void* ws, const loract_desc_t* desc, bool with_A, CompressWs* out, Plan* plan) {
+  const bool bf16 = desc->dtype == LORACT_BF16;
+  *plan = make_plan(desc->n_tokens, desc->d, desc->rank, bf16);
+  Carver c(ws);
+  CompressWs w;
+  w.status = (uint32_t*)c.take(256);
+  w.idx = (int32_t*)c.take((size_t)desc->rank * 4);
+  const size_t es = (size_t)elem_bytes(desc);
+  w.S = c.take((size_t)desc->rank * desc->d * es);
+  w.Omega = c.take((size_t)desc->rank * desc->d * es);
+  carve_basis(c, *plan, &w.b);
+  w.A = with_A ? c.take((size_t)desc->n_tokens * desc->d * es) : nullptr;
+  if (out) *out = w;
+  return c.off;
+}
+
+// Algorithm 1, t = 0, on a matrix X that is already in place.
+cudaError_t compress_core(const loract_desc_t* desc, const void* X, int64_t ldx, void* U, void* V,
+                          int32_t* idx_out, const CompressWs& w, const Plan& plan, cudaStream_t stream) {
+  const bool bf16 = plan.bf16;
+  const int r = desc->rank;
+  LORACT_CUDA_TRY(cudaMemsetAsync(w.status, 0, 4, stream));
+  // line 1: sample rows, gather them
+  LORACT_CUDA_TRY(sample_indices_launch(desc->seed, desc->call_id, (uint32_t)desc->n_tokens, r, w.idx,
+                                        w.status, stream));
+  if (idx_out) LORACT_CUDA_TRY(cudaMemcpyAsync(idx_out, w.idx, (size_t)r * 4, cudaMemcpyDeviceToDevice, stream));
+  LORACT_CUDA_TRY(gather_rows_launch(X, ldx, w.idx, r, desc->d, elem_bytes(desc), w.S, stream));
+  // small-block preconditioning: Omega = L_s^{-1} A_k with A_k A_k^T = L_s L_s^T.  Omega has the row
+  // space of A_k, so range(X Omega^T) = range(X A_k^T) (line 2), but its rows are close to orthonormal,
+  // which keeps the spectrum of the sketch from being squared.
+  LORACT_CUDA_TRY(gram_rows(w.S, r, desc->d, bf16, w.b, w.status, stream));
+  LORACT_CUDA_TRY(factor(r, bf16, w.b.splits_gram_sample, kShiftSample, w.b, w.status, stream));
+  {
+    GemmDesc g;
+    g.M = r; g.N = (int)desc->d; g.K = r; g.b_mn = true; g.lda = r; g.ldb = desc->d;
+    g.a_type = g.b_type = bf16 ? ELEM_BF16 : ELEM_F32;
+    g.ldc = desc->d; g.C0 = w.Omega;
+    if (bf16) {
+      g.n_terms = 2; g.terms[0] = {w.b.Lh, w.S}; g.terms[1] = {w.b.Ll, w.S}; g.out = OUT_BF16;
+    } else {
+      g.terms[0] = {w.b.Linv32, w.S}; g.out = OUT_F32;
+    }
+    LORACT_CUDA_TRY(run_gemm(g, w.status, stream));
+  }
+  // lines 2 and 7: Q, written to U;  line 8: V = U^T X
+  LORACT_CUDA_TRY(range_basis(X, ldx, plan, w.Omega, U, w.b, w.status, stream));
+  return project(U, X, ldx, plan, V, w.b, w.status, stream);
+}
+
+struct WgradWs {
+  float* partials;
+  float* T;
+  int splits;
+};
+size_t carve_wgrad(void* ws, const loract_desc_t* desc, int g, WgradWs* out) {
+  Carver c(ws);
+  c.take(256);
+  WgradWs w;
+  w.splits = desc->dtype == LORACT_BF16 ? gemm_tc_pick_splits(desc->rank, g, (int)desc->n_tokens, true, true)
+                                        : (desc->n_tokens >= 4096 ? 16 : 1);
+  w.partials = (float*)c.take((size_t)w.splits * desc->rank * g * 4);
+  w.T = (float*)c.take((size_t)desc->rank * g * 4);
+  if (out) *out = w;
+  return c.off;
+}
+
+loract_status_t from_cuda(cudaError_t e) { return e == cudaSuccess ? LORACT_OK : LORACT_ERR_CUDA; }
+
+}  // namespace
+}  // namespace loract
+
+using namespace loract;
+
+extern "C" {
+
+size_t loract_workspace_bytes(const loract_desc_t* desc) {
+  if (check_desc(desc) != LORACT_OK) return 0;
+  Plan plan;
+  size_t a = carve_compress(nullptr, desc, /*with_A=*/true, nullptr, &plan);
+  size_t b = carve_wgrad(nullptr, desc, 256, nullptr);
+  return a > b ? a : b;
+}
+
+loract_status_t loract_sample_indices(const loract_desc_t* desc, int32_t* idx_dev, void* ws, size_t ws_bytes,
+                                      void* stream) {
+  loract_status_t s = check_desc(desc);
+  if (s != LORACT_OK) return s;
+  if (!idx_dev || !ws) return LORACT_ERR_INVALID_ARG;
+  if (ws_bytes < 256) return LORACT_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMemsetAsync(ws, 0, 4, st);
+  if (e == cudaSuccess)
+    e = sample_indices_launch(desc->seed, desc->call_id, (uint32_t)desc->n_tokens, desc->rank, idx_dev,
+                              (uint32_t*)ws, st);
+  return from_cuda(e);
+}
+
+loract_status_t loract_compress(const loract_desc_t* desc, const void* X, void* U, void* V, int32_t* idx_out,
+                                void* ws, size_t ws_bytes, void* stream) {
+  loract_status_t s = check_desc(desc);
+  if (s != LORACT_OK) return s;
+  if (!X || !U || !V || !ws) return LORACT_ERR_INVALID_ARG;
+  if (misaligned(X) || misaligned(U) || misaligned(V) || ((uintptr_t)ws & 255)) return LORACT_ERR_ALIGNMENT;
+  CompressWs w;
+  Plan plan;
+  const size_t need = carve_compress(ws, desc, /*with_A=*/false, &w, &plan);
+  if (ws_bytes < need) return LORACT_ERR_WORKSPACE_TOO_SMALL;
+  return from_cuda(compress_core(desc, X, desc->ldx, U, V, idx_out, w, plan, (cudaStream_t)stream));
+}
+
+loract_status_t loract_compress_prenorm(const loract_desc_t* desc, const void* X, const void* gamma,
+                                        const void* beta, float eps, int32_t kind, void* A_out, float* rstd,
+                                        float* mean, void* U, void* V, int32_t* idx_out, void* ws,
+                                        size_t ws_bytes, void* stream) {
+  loract_status_t s = check_desc(desc);
+  if (s != LORACT_OK) return s;
+  if (!X || !gamma || !rstd || !U || !V || !ws) return LORACT_ERR_INVALID_ARG;
+  if (kind != LORACT_NORM_RMS && kind != LORACT_NORM_LAYER) return LORACT_ERR_INVALID_ARG;
+  if (kind == LORACT_NORM_LAYER && !mean) return LORACT_ERR_INVALID_ARG;
+  if (!(eps >= 0.f)) return LORACT_ERR_INVALID_ARG;
+  if (misaligned(X) || misaligned(U) || misaligned(V) || (A_out && misaligned(A_out)) || ((uintptr_t)ws & 255))
+    return LORACT_ERR_ALIGNMENT;
+  CompressWs w;
+  Plan plan;
+  const size_t need = carve_compress(ws, desc, /*with_A=*/A_out == nullptr, &w, &plan);
+  if (ws_bytes < need) return LORACT_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  void* A = A_out ? A_out : w.A;
+  cudaError_t e = norm_forward_launch(X, desc->n_tokens, desc->d, desc->ldx,
+                                      desc->dtype == LORACT_BF16 ? ELEM_BF16 : ELEM_F32, gamma, beta, eps, kind,
+                                      A, desc->d, rstd, kind == LORACT_NORM_LAYER ? mean : nullptr, st);
+  if (e != cudaSuccess) return LORACT_ERR_CUDA;
+  return from_cuda(compress_core(desc, A, desc->d, U, V, idx_out, w, plan, st));
+}
+
+loract_status_t loract_reconstruct(const loract_desc_t* desc, const void* U, const void* V, void* X_out,
+                                   void* stream) {
+  loract_status_t s = check_desc(desc);
+  if (s != LORACT_OK) return s;
+  if (!U || !V || !X_out) return LORACT_ERR_INVALID_ARG;
+  if (misaligned(U) || misaligned(V) || misaligned(X_out)) return LORACT_ERR_ALIGNMENT;
+  const bool bf16 = desc->dtype == LORACT_BF16;
+  GemmDesc g;
+  g.M = (int)desc->n_tokens; g.N = (int)desc->d; g.K = desc->rank; g.b_mn = true;
+  g.lda = desc->rank; g.ldb = desc->d;
+  g.a_type = g.b_type = bf16 ? ELEM_BF16 : ELEM_F32;
+  g.terms[0] = {U, V};
+  g.out = bf16 ? OUT_BF16 : OUT_F32; g.C0 = X_out; g.ldc = desc->ldx;
+  return from_cuda(run_gemm(g, nullptr, (cudaStream_t)stream));
+}
+
+loract_status_t loract_weight_grad(const loract_desc_t* desc, const void* U, const void* V, const void* G,
+                                   int32_t g, int64_t ldg, float* dW, int accumulate, void* ws, size_t ws_bytes,
+                                   void* stream) {
+  loract_status_t s = check_desc(desc);
+  if (s != LORACT_OK) return s;
+  if (!U || !V || !G || !dW || !ws) return LORACT_ERR_INVALID_ARG;
+  if (g < 1 || g > 256 || ldg < g) return LORACT_ERR_INVALID_ARG;
+  if (misaligned(U) || misaligned(V) || misaligned(G) || ((uintptr_t)ws & 255)) return LORACT_ERR_ALIGNMENT;
+  if (ldg % (desc->dtype == LORACT_BF16 ? 8 : 4)) return LORACT_ERR_ALIGNMENT;
+  WgradWs w;
+  const size_t need = carve_wgrad(ws, desc, g, &w);
+  if (ws_bytes < need) return LORACT_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int el = desc->dtype == LORACT_BF16 ? ELEM_BF16 : ELEM_F32;
+  const int r = desc->rank;
+  GemmDesc t;  // T = U^T G  (r x g), split over tokens
+  t.M = r; t.N = g; t.K = (int)desc->n_tokens; t.a_mn = true; t.b_mn = true; t.lda = r; t.ldb = ldg;
+  t.a_type = t.b_type = el;
+  t.terms[0] = {U, G};
+  t.out = OUT_F32; t.C0 = w.partials; t.ldc = g; t.splits = w.splits; t.split_stride = (int64_t)r * g;
+  uint32_t* status = (uint32_t*)ws;
+  cudaError_t e = cudaMemsetAsync(status, 0, 4, st);
+  if (e == cudaSuccess) e = run_gemm(t, status, st);
+  if (e == cudaSuccess)
+    e = reduce_partials_launch(w.partials, w.splits, t.split_stride, t.split_stride, w.T, nullptr, st);
+  if (e == cudaSuccess) {
+    GemmDesc q;  // dW = V^T T  (d x g)
+    q.M = (int)desc->d; q.N = g; q.K = r; q.a_mn = true; q.b_mn = true; q.lda = desc->d; q.ldb = g;
+    q.a_type = el; q.b_type = ELEM_F32;
+    q.terms[0] = {V, w.T};
+    q.out = OUT_F32; q.C0 = dW; q.ldc = g; q.accumulate = accumulate != 0;
+    e = gemm_simt_launch(q, st);
+  }
+  return from_cuda(e);
+}
+
+size_t loract_rsvd_workspace_bytes(const loract_desc_t* desc, int32_t oversample) {
+  if (check_desc(desc) != LORACT_OK || desc->dtype != LORACT_BF16) return 0;
+  const int l = desc->rank + oversample;
+  if (oversample < 0 || l % 16 || l > 512 || l > desc->n_tokens || l > desc->d) return 0;
+  Plan plan = make_plan(desc->n_tokens, desc->d, l, true);
+  Carver c(nullptr);
+  c.take(256);
+  c.take((size_t)l * desc->d * 2);  // test matrix / X^T Q
+  BasisWs b;
+  carve_basis(c, plan, &b);
+  return c.off;
+}
+
+loract_status_t loract_rsvd(const loract_desc_t* desc, int32_t oversample, const void* X, void* Uq, void* B,
+                            void* ws, size_t ws_bytes, void* stream) {
+  // t of Algorithm 1 is taken from desc->power_iters here, so validate a copy with t = 0
+  if (!desc) return LORACT_ERR_INVALID_ARG;
+  loract_desc_t d0 = *desc;
+  d0.power_iters = 0;
+  loract_status_t s = check_desc(&d0);
+  if (s != LORACT_OK) return s;
+  if (desc->dtype != LORACT_BF16) return LORACT_ERR_UNSUPPORTED;
+  if (desc->power_iters < 0 || desc->power_iters > 8) return LORACT_ERR_INVALID_ARG;
+  const size_t need = loract_rsvd_workspace_bytes(&d0, oversample);
+  if (need == 0) return LORACT_ERR_INVALID_ARG;
+  if (!X || !Uq || !B || !ws) return LORACT_ERR_INVALID_ARG;
+  if (misaligned(X) || misaligned(Uq) || misaligned(B) || ((uintptr_t)ws & 255)) return LORACT_ERR_ALIGNMENT;
+  if (ws_bytes < need) return LORACT_ERR_WORKSPACE_TOO_SMALL;
+  const int l = desc->rank + oversample;
+  Plan plan = make_plan(desc->n_tokens, desc->d, l, true);
+  Carver c(ws);
+  uint32_t* status = (uint32_t*)c.take(256);
+  __nv_bfloat16* Om = (__nv_bfloat16*)c.take((size_t)l * desc->d * 2);
+  BasisWs b;
+  carve_basis(c, plan, &b);
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMemsetAsync(status, 0, 4, st);
+  if (e == cudaSuccess) e = gaussian_rows_launch(desc->seed, desc->call_id, l, desc->d, Om, st);
+  if (e == cudaSuccess) e = range_basis(X, desc->ldx, plan, Om, Uq, b, status, st);
+  for (int it = 0; it < desc->power_iters && e == cudaSuccess; ++it) {
+    // Y = X (X^T Q): X^T Q is kept transposed (l x d), which is exactly the test-matrix layout
+    e = project(Uq, X, desc->ldx, plan, Om, b, status, st);
+    if (e == cudaSuccess) e = range_basis(X, desc->ldx, plan, Om, Uq, b, status, st);
+  }
+  if (e == cudaSuccess) e = project(Uq, X, desc->ldx, plan, B, b, status, st);
+  return from_cuda(e);
+}
+
+loract_status_t loract_read_device_status(const void* ws, uint32_t* out_host, void* stream) {
+  if (!ws || !out_host) return LORACT_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMemcpyAsync(out_host, ws, 4, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  return from_cuda(e);
+}
+
+const char* loract_status_string(loract_status_t s) {
+  switch (s) {
+    case LORACT_OK: return "ok";
+    case LORACT_ERR_INVALID_ARG: return "invalid argument";
+    case LORACT_ERR_UNSUPPORTED: return "unsupported";
+    case LORACT_ERR_ALIGNMENT: return "misaligned pointer or stride";
+    case LORACT_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case LORACT_ERR_CUDA: return "CUDA error";
+    case LORACT_ERR_NUMERIC: return "numerical breakdown";
+    case LORACT_ERR_TIMEOUT: return "device wait expired";
+  }
+  return "unknown status";
+}
+
+uint64_t loract_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+loract_status_t loract_debug_gemm(int32_t M, int32_t N, int32_t K, int32_t a_mn, int32_t b_mn,
+                                  const void* const* A, int64_t lda, const void* const* B, int64_t ldb,
+                                  int32_t a_type, int32_t b_type, int32_t n_terms, int32_t out_mode, void* C0,
+                                  void* C1, int64_t ldc, int32_t splits, int64_t split_stride, int32_t acc64,
+                                  int32_t engine, uint32_t* status_word, void* stream) {
+  if (!A || !B || !C0 || n_terms < 1 || n_terms > 3 || M < 1 || N < 1 || K < 1) return LORACT_ERR_INVALID_ARG;
+  GemmDesc g;
+  g.M = M; g.N = N; g.K = K; g.a_mn = a_mn != 0; g.b_mn = b_mn != 0; g.lda = lda; g.ldb = ldb;
+  g.a_type = a_type; g.b_type = b_type; g.n_terms = n_terms;
+  for (int t = 0; t < n_terms; ++t) g.terms[t] = {A[t], B[t]};
+  g.out = out_mode; g.C0 = C0; g.C1 = C1; g.ldc = ldc; g.splits = splits < 1 ? 1 : splits;
+  g.split_stride = split_stride; g.acc64 = acc64 != 0;
+  if (engine == 1) {
+    if (!gemm_tc_supported(g)) return LORACT_ERR_UNSUPPORTED;
+    return from_cuda(gemm_tc_launch(g, status_word, (cudaStream_t)stream));
+  }
+  return from_cuda(gemm_simt_launch(g, (cudaStream_t)stream));
+}
+
+loract_status_t loract_debug_small_block(int32_t r, const void* partials, int32_t partial_f64, int32_t n_partials,
+                                         int64_t partial_stride, int32_t use_f64, float shift_rel, void* scratch,
+                                         float* linv_f32, void* linv_hi, void* linv_lo, uint32_t* status_word,
+                                         void* stream) {
+  if (r < 16 || r > 512 || r % 16 || !partials || !scratch || n_partials < 1) return LORACT_ERR_INVALID_ARG;
+  SmallBlockArgs a;
+  a.r = r; a.partials = partials; a.partial_type = partial_f64 ? ELEM_F64 : ELEM_F32;
+  a.n_partials = n_partials; a.partial_stride = partial_stride; a.use_f64 = use_f64 != 0;
+  a.scratch = scratch; a.shift_rel = shift_rel; a.linv_f32 = linv_f32;
+  a.linv_hi = (__nv_bfloat16*)linv_hi; a.linv_lo = (__nv_bfloat16*)linv_lo; a.dev_status = status_word;
+  return from_cuda(small_block_launch(a, (cudaStream_t)stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,114 @@
+// Internal declarations shared by the translation units of libloract (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/loract.h"
+
+namespace loract {
+
+// ---------------------------------------------------------------- launch accounting
+void count_launch(int n = 1);
+
+#define LORACT_CUDA_TRY(expr)                          \
+  do {                                                 \
+    cudaError_t _e = (expr);                           \
+    if (_e != cudaSuccess) return _e;                  \
+  } while (0)
+
+// ---------------------------------------------------------------- generic contraction
+// C (M x N) = sum over terms of  A_t (M x K) * B_t (K x N), fp32 (or fp64) accumulation.
+// Operands are row-major arrays; a_mn / b_mn say which index is contiguous in memory:
+//   a_mn == false : A stored as [M][K]  (K-major)      a_mn == true : A stored as [K][M]  (M-major)
+//   b_mn == false : B stored as [N][K]  (K-major)      b_mn == true : B stored as [K][N]  (N-major)
+// Several terms share shapes and leading dimensions; they exist for split-precision products
+// (x = hi + lo in bf16: hi*hi + hi*lo + lo*hi).
+enum OutMode : int {
+  OUT_F32 = 0,    // C0: float
+  OUT_BF16 = 1,   // C0: bf16
+  OUT_SPLIT = 2,  // C0: bf16 hi, C1: bf16 lo  (hi = bf16(x), lo = bf16(x - hi))
+  OUT_F64 = 3     // C0: double (SIMT path only)
+};
+
+enum ElemType : int { ELEM_F32 = 0, ELEM_BF16 = 1, ELEM_F64 = 2 };
+
+struct GemmTerm {
+  const void* A;
+  const void* B;
+};
+
+struct GemmDesc {
+  int M = 0, N = 0, K = 0;
+  bool a_mn = false, b_mn = false;
+  int64_t lda = 0, ldb = 0;  // leading dimension (elements) of the stored arrays
+  int a_type = ELEM_BF16, b_type = ELEM_BF16;
+  int n_terms = 1;
+  GemmTerm terms[4];
+  int out = OUT_F32;
+  void* C0 = nullptr;
+  void* C1 = nullptr;
+  int64_t ldc = 0;
+  // split over K: split s handles a contiguous K range and writes C0 + s * split_stride (fp32/f64 out)
+  int splits = 1;
+  int64_t split_stride = 0;
+  bool acc64 = false;      // SIMT path: accumulate in double
+  bool accumulate = false; // SIMT path, OUT_F32, splits == 1: C += result
+  float alpha = 1.0f;      // SIMT path: C = alpha * sum
+};
+
+// tcgen05 engine: bf16 operands, fp32 accumulation in tensor memory.  Returns cudaErrorNotSupported
+// for shapes it does not take (the caller then uses the SIMT kernel).
+bool gemm_tc_supported(const GemmDesc& g);
+cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t stream);
+int gemm_tc_pick_splits(int M, int N, int K, bool a_mn, bool b_mn);
+
+// Plain CUDA-core kernel for any shape and type (fp32 path, small or odd shapes).
+cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t stream);
+
+// ---------------------------------------------------------------- sampler and gather
+cudaError_t sample_indices_launch(uint64_t seed, uint64_t call_id, uint32_t n_rows, int rank,
+                                  int32_t* idx_dev, uint32_t* dev_status, cudaStream_t stream);
+// dst (rank x d, stride d) = src[idx, :] (stride ld); 16-byte loads.  elem_bytes 2 or 4.
+cudaError_t gather_rows_launch(const void* src, int64_t ld, const int32_t* idx, int rank, int64_t d,
+                               int elem_bytes, void* dst, cudaStream_t stream);
+// Gaussian test matrix for the RSVD comparator: dst (l x d bf16, row-major) with
+// dst[c][j] = z(j * l + c), z the Philox + Box-Muller stream (counter word 1 = 1).
+cudaError_t gaussian_rows_launch(uint64_t seed, uint64_t call_id, int l, int64_t d,
+                                 __nv_bfloat16* dst, cudaStream_t stream);
+
+// ---------------------------------------------------------------- small-block factorisation
+// From the symmetric positive semi-definite r x r matrix  W = sum_s P_s  (P_s fp32 or fp64, row-major,
+// stride r, consecutive partials `partial_stride` elements apart) computes the inverse of the
+// Cholesky factor of  W + shift_rel * mean(diag W) * I :  Linv = L^{-1} (lower triangular), so that
+// (Y Linv^T) has orthonormal columns when W = Y^T Y.  Outputs (any may be null): Linv as an fp32 or
+// fp64 matrix, and as a bf16 hi/lo pair.  `scratch` holds 2 r*r elements of the compute type.
+struct SmallBlockArgs {
+  int r = 0;
+  const void* partials = nullptr;
+  int partial_type = ELEM_F32;
+  int n_partials = 1;
+  int64_t partial_stride = 0;
+  bool use_f64 = false;  // compute type
+  void* scratch = nullptr;
+  float shift_rel = 0.f;
+  void* linv_full = nullptr;  // fp32 (use_f64 == false) or fp64 (use_f64 == true), r x r
+  float* linv_f32 = nullptr;  // fp32 copy, r x r
+  __nv_bfloat16* linv_hi = nullptr;
+  __nv_bfloat16* linv_lo = nullptr;
+  uint32_t* dev_status = nullptr;
+};
+cudaError_t small_block_launch(const SmallBlockArgs& a, cudaStream_t stream);
+
+// ---------------------------------------------------------------- elementwise helpers
+// out = sum_s partials[s] (fixed order), written as fp32 and/or bf16.
+cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_t stride,
+                                   int64_t count, float* out_f32, __nv_bfloat16* out_bf16,
+                                   cudaStream_t stream);
+// Section 3.3 forward: A = Norm(X); per-row rstd (and mean for LayerNorm).  One warp per row.
+cudaError_t norm_forward_launch(const void* X, int64_t n, int64_t d, int64_t ldx, int elem_type,
+                                const void* gamma, const void* beta, float eps, int kind, void* A,
+                                int64_t lda, float* rstd, float* mean, cudaStream_t stream);
+
+}  // namespace loract

@@ -1,0 +1,443 @@
+// Tensor-core engine for the dense contractions of the path (Algorithm 1 lines 2 and 8, the Gram
+// matrices of the orthonormalisation, the application of the triangular factors, Reconstruct).
+//
+// One kernel, written for sm_100a: TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) fills a
+// 4-stage shared-memory ring, one thread issues tcgen05.mma (kind::f16, bf16 operands, M = 128,
+// N <= 256, K = 16 per instruction) into an fp32 accumulator in tensor memory, four warps read the
+// accumulator back with tcgen05.ld and write the result.  Operands may be K-major or MN-major, which
+// covers X Omega^T (K/K), U^T X and Y^T Y (MN/MN) and U V (K/MN) without transposing anything in memory.
+// A contraction can be the sum of up to three products over the same shapes (split-precision terms),
+// and can be split over K into partial results that a later kernel adds in a fixed order.
+//
+// Every wait on an mbarrier is bounded by a wall-clock limit; on expiry the kernel records
+// LORACT_DEV_WAIT_EXPIRED, stops issuing work, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include <map>
+#include <mutex>
+#include <tuple>
+
+#include "common.cuh"
+
+namespace loract {
+
+namespace {
+
+constexpr int kBM = 128;
+constexpr int kBK = 64;          // bf16 elements = one 128-byte swizzle row
+constexpr int kStages = 4;
+constexpr int kThreads = 192;    // warp 0: TMA, warp 1: MMA + tensor memory, warps 2..5: epilogue
+constexpr uint32_t kABytes = kBM * kBK * 2;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
+
+struct alignas(64) TmapPack {
+  CUtensorMap a[3];
+  CUtensorMap b[3];
+};
+
+struct TcParams {
+  int M, N;
+  int bn;             // tile width, multiple of 16, <= 256
+  int kb_total;       // 64-wide K blocks per term
+  int kb_per_split;
+  int n_terms;
+  int out;
+  void* C0;
+  void* C1;
+  int64_t ldc;
+  int64_t split_stride;
+  uint32_t b_bytes;   // bytes of one B stage
+  uint32_t tmem_cols;
+  uint32_t* dev_status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false if the limit expired (or another role already gave up).
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t spin = 1;; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spin & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int x,
+                                            int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t v[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  K-major: rows of 128 bytes, groups of 8 rows
+// 1024 bytes apart (stride byte offset); the leading byte offset is not used.  MN-major: rows are K
+// indices, each 128 bytes = 64 elements along M/N; groups of 8 K rows 1024 bytes apart (stride byte
+// offset) and consecutive 64-element groups along M/N one TMA box (64 rows = 8192 bytes) apart
+// (leading byte offset).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, bool mn_major) {
+  const uint64_t lbo = mn_major ? (8192u >> 4) : 1u;
+  const uint64_t sbo = 1024u >> 4;
+  return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+
+template <bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  __shared__ __align__(8) uint64_t full_bar[kStages];
+  __shared__ __align__(8) uint64_t empty_bar[kStages];
+  __shared__ __align__(8) uint64_t accum_bar;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * p.bn, m0 = blockIdx.y * kBM, split = blockIdx.z;
+  const int kb_begin = split * p.kb_per_split;
+  const int kb_count = max(0, min(p.kb_total, kb_begin + p.kb_per_split) - kb_begin);
+  const int n_iter = kb_count * p.n_terms;
+  const uint32_t stage_bytes = kABytes + p.b_bytes;
+  // dynamic shared memory is declared 1024-aligned; round up anyway (swizzle atoms need it)
+  unsigned char* tiles = (unsigned char*)(((uintptr_t)smem + 1023) & ~(uintptr_t)1023);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    mbar_init(&accum_bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                 "r"(p.tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const uint32_t tx_bytes = stage_bytes;
+      for (int it = 0; it < n_iter; ++it) {
+        const int s = it % kStages;
+        if (!mbar_wait_bounded(&empty_bar[s], ((it / kStages) & 1) ^ 1, &abort_flag)) break;
+        const int term = it / kb_count;
+        const int k0 = (kb_begin + (it - term * kb_count)) * kBK;
+        unsigned char* a_dst = tiles + (size_t)s * stage_bytes;
+        unsigned char* b_dst = a_dst + kABytes;
+        mbar_arrive_expect_tx(&full_bar[s], tx_bytes);
+        if (A_MN) {
+          tma_load_2d(a_dst, &maps.a[term], &full_bar[s], m0, k0);
+          tma_load_2d(a_dst + 8192, &maps.a[term], &full_bar[s], m0 + 64, k0);
+        } else {
+          tma_load_2d(a_dst, &maps.a[term], &full_bar[s], k0, m0);
+        }
+        if (B_MN) {
+          for (uint32_t q = 0; q * 8192u < p.b_bytes; ++q)
+            tma_load_2d(b_dst + q * 8192u, &maps.b[term], &full_bar[s], n0 + (int)q * 64, k0);
+        } else {
+          tma_load_2d(b_dst, &maps.b[term], &full_bar[s], k0, n0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // instruction descriptor: fp32 accumulator, bf16 A and B, operand majors, N >> 3, M >> 4
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
+                             ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(p.bn >> 3) << 17) |
+                             ((uint32_t)(kBM >> 4) << 24);
+      bool ok = true;
+      for (int it = 0; it < n_iter && ok; ++it) {
+        const int s = it % kStages;
+        ok = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1, &abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(tiles + (size_t)s * stage_bytes);
+        const uint32_t b_addr = a_addr + kABytes;
+        const uint64_t a_desc = make_smem_desc(a_addr, A_MN);
+        const uint64_t b_desc = make_smem_desc(b_addr, B_MN);
+#pragma unroll
+        for (int k = 0; k < kBK / 16; ++k) {
+          // 16 elements along K: 32 bytes inside the swizzled row (K-major) or 16 rows (MN-major)
+          const uint64_t a_k = a_desc + (uint64_t)((A_MN ? 2048u : 32u) >> 4) * k;
+          const uint64_t b_k = b_desc + (uint64_t)((B_MN ? 2048u : 32u) >> 4) * k;
+          tc_mma_bf16(tmem_base, a_k, b_k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+        }
+        tc_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+      }
+      tc_commit(&accum_bar);       // accumulator complete (or nothing was issued)
+    }
+  } else {
+    // epilogue: warp w may touch tensor-memory lanes 32 * (w % 4) .. + 31
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    const int m = m0 + row;
+    bool ok = mbar_wait_bounded(&accum_bar, 0, &abort_flag);
+    ok = __all_sync(0xffffffffu, ok);
+    tc_fence_after();
+    if (ok && n_iter > 0) {
+      for (int c0 = 0; c0 < p.bn; c0 += 32) {
+        uint32_t v[32];
+        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
+        tc_wait_ld();
+        const int n = n0 + c0;
+        if (m >= p.M) continue;
+        const int valid = min(32, min(p.bn - c0, p.N - n));
+        if (valid <= 0) continue;
+        if (p.out == OUT_F32) {
+          float* dst = (float*)p.C0 + (int64_t)split * p.split_stride + (int64_t)m * p.ldc + n;
+          if (valid == 32 && ((((uintptr_t)dst) & 15) == 0)) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              reinterpret_cast<uint4*>(dst)[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+          } else {
+            for (int q = 0; q < valid; ++q) dst[q] = __uint_as_float(v[q]);
+          }
+        } else {
+          __nv_bfloat16* dst_hi = (__nv_bfloat16*)p.C0 + (int64_t)m * p.ldc + n;
+          __nv_bfloat16* dst_lo = (p.out == OUT_SPLIT) ? (__nv_bfloat16*)p.C1 + (int64_t)m * p.ldc + n : nullptr;
+          if (valid == 32 && ((((uintptr_t)dst_hi) & 15) == 0)) {
+            uint32_t hi[16], lo[16];
+#pragma unroll
+            for (int q = 0; q < 16; ++q) {
+              const float x0 = __uint_as_float(v[2 * q]), x1 = __uint_as_float(v[2 * q + 1]);
+              const __nv_bfloat16 h0 = __float2bfloat16(x0), h1 = __float2bfloat16(x1);
+              hi[q] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+              lo[q] = pack_bf16x2(x0 - __bfloat162float(h0), x1 - __bfloat162float(h1));
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              reinterpret_cast<uint4*>(dst_hi)[q] = make_uint4(hi[4 * q], hi[4 * q + 1], hi[4 * q + 2], hi[4 * q + 3]);
+            if (dst_lo) {
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                reinterpret_cast<uint4*>(dst_lo)[q] = make_uint4(lo[4 * q], lo[4 * q + 1], lo[4 * q + 2], lo[4 * q + 3]);
+            }
+          } else {
+            for (int q = 0; q < valid; ++q) {
+              const float x = __uint_as_float(v[q]);
+              const __nv_bfloat16 h = __float2bfloat16(x);
+              dst_hi[q] = h;
+              if (dst_lo) dst_lo[q] = __float2bfloat16(x - __bfloat162float(h));
+            }
+          }
+        }
+      }
+    } else if (ok && n_iter == 0 && m < p.M && p.out == OUT_F32) {
+      // an empty K range still owns its partial: write zeros
+      float* dst = (float*)p.C0 + (int64_t)split * p.split_stride + (int64_t)m * p.ldc + n0;
+      for (int q = 0; q < min(p.bn, p.N - n0); ++q) dst[q] = 0.f;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols)
+                 : "memory");
+  }
+  if (threadIdx.x == 0 && abort_flag && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_WAIT_EXPIRED);
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)sym;
+  });
+  return fn;
+}
+
+// Tensor maps depend only on (pointer, extents, stride, box); they are cached so that a repeated call
+// on the same buffers encodes nothing.
+typedef std::tuple<const void*, uint64_t, uint64_t, uint64_t, uint32_t, uint32_t> TmapKey;
+std::mutex g_tmap_mutex;
+std::map<TmapKey, CUtensorMap> g_tmap_cache;
+
+// 2-D bf16 tensor: `inner` contiguous elements, `outer` rows `ld` elements apart; box inner x outer.
+cudaError_t get_tmap(const void* ptr, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_inner,
+                     uint32_t box_outer, CUtensorMap* out) {
+  const TmapKey key(ptr, inner, outer, ld, box_inner, box_outer);
+  {
+    std::lock_guard<std::mutex> lock(g_tmap_mutex);
+    auto it = g_tmap_cache.find(key);
+    if (it != g_tmap_cache.end()) { *out = it->second; return cudaSuccess; }
+  }
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return cudaErrorNotSupported;
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t elem[2] = {1, 1};
+  CUtensorMap m;
+  const CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box,
+                        elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  {
+    std::lock_guard<std::mutex> lock(g_tmap_mutex);
+    if (g_tmap_cache.size() > 4096) g_tmap_cache.clear();
+    g_tmap_cache[key] = m;
+  }
+  *out = m;
+  return cudaSuccess;
+}
+
+int pick_bn(int N) {
+  const int n16 = (N + 15) / 16 * 16;
+  if (n16 <= 256) return n16;
+  // widest tile <= 256 that leaves the least padding
+  int best = 256, best_pad = ((N + 255) / 256) * 256 - N;
+  for (int bn = 256; bn >= 128; bn -= 16) {
+    const int pad = ((N + bn - 1) / bn) * bn - N;
+    if (pad < best_pad) { best = bn; best_pad = pad; }
+  }
+  return best;
+}
+
+template <bool A_MN, bool B_MN>
+cudaError_t launch_variant(const TmapPack& maps, const TcParams& p, dim3 grid, size_t smem, cudaStream_t stream) {
+  static bool configured[64] = {};
+  int dev = 0;
+  LORACT_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    LORACT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kStages * (kABytes + 32768) + 1024));
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
+  gemm_tc_kernel<A_MN, B_MN><<<grid, kThreads, smem, stream>>>(maps, p);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool gemm_tc_supported(const GemmDesc& g) {
+  if (g.a_type != ELEM_BF16 || g.b_type != ELEM_BF16) return false;
+  if (!(g.out == OUT_F32 || g.out == OUT_BF16 || g.out == OUT_SPLIT)) return false;
+  if (g.M < 1 || g.N < 1 || g.K < 1 || g.n_terms < 1 || g.n_terms > 3) return false;
+  if (g.lda % 8 || g.ldb % 8) return false;
+  if (g.splits > 1 && g.out != OUT_F32) return false;
+  if (g.accumulate || g.alpha != 1.0f) return false;
+  for (int t = 0; t < g.n_terms; ++t)
+    if (((uintptr_t)g.terms[t].A & 15) || ((uintptr_t)g.terms[t].B & 15)) return false;
+  return true;
+}
+
+int gemm_tc_pick_splits(int M, int N, int K, bool, bool) {
+  const int tiles = ((M + kBM - 1) / kBM) * ((N + pick_bn(N) - 1) / pick_bn(N));
+  const int kb = (K + kBK - 1) / kBK;
+  if (tiles >= 96) return 1;
+  int s = 148 / tiles;
+  if (s > kb / 4) s = kb / 4;  // at least four K blocks per split
+  if (s > 32) s = 32;
+  return s < 1 ? 1 : s;
+}
+
+cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t stream) {
+  if (!gemm_tc_supported(g)) return cudaErrorNotSupported;
+  TcParams p;
+  p.M = g.M; p.N = g.N;
+  p.bn = pick_bn(g.N);
+  p.kb_total = (g.K + kBK - 1) / kBK;
+  const int splits = g.splits < 1 ? 1 : g.splits;
+  p.kb_per_split = (p.kb_total + splits - 1) / splits;
+  p.n_terms = g.n_terms;
+  p.out = g.out; p.C0 = g.C0; p.C1 = g.C1; p.ldc = g.ldc; p.split_stride = g.split_stride;
+  p.b_bytes = g.b_mn ? (uint32_t)((p.bn + 63) / 64) * 8192u : (uint32_t)p.bn * 128u;
+  p.tmem_cols = 32;
+  while ((int)p.tmem_cols < p.bn) p.tmem_cols *= 2;
+  p.dev_status = dev_status;
+
+  TmapPack maps;
+  for (int t = 0; t < g.n_terms; ++t) {
+    if (g.a_mn) LORACT_CUDA_TRY(get_tmap(g.terms[t].A, g.M, g.K, g.lda, 64, 64, &maps.a[t]));
+    else LORACT_CUDA_TRY(get_tmap(g.terms[t].A, g.K, g.M, g.lda, 64, kBM, &maps.a[t]));
+    if (g.b_mn) LORACT_CUDA_TRY(get_tmap(g.terms[t].B, g.N, g.K, g.ldb, 64, 64, &maps.b[t]));
+    else LORACT_CUDA_TRY(get_tmap(g.terms[t].B, g.K, g.N, g.ldb, 64, (uint32_t)p.bn, &maps.b[t]));
+  }
+  for (int t = g.n_terms; t < 3; ++t) { maps.a[t] = maps.a[0]; maps.b[t] = maps.b[0]; }
+
+  dim3 grid((g.N + p.bn - 1) / p.bn, (g.M + kBM - 1) / kBM, splits);
+  const size_t smem = (size_t)kStages * (kABytes + p.b_bytes) + 1024;
+  if (g.a_mn && g.b_mn) return launch_variant<true, true>(maps, p, grid, smem, stream);
+  if (g.a_mn && !g.b_mn) return launch_variant<true, false>(maps, p, grid, smem, stream);
+  if (!g.a_mn && g.b_mn) return launch_variant<false, true>(maps, p, grid, smem, stream);
+  return launch_variant<false, false>(maps, p, grid, smem, stream);
+}
+
+}  // namespace loract

@@ -1,0 +1,226 @@
+// CUDA-core kernels: the generic contraction used by the fp32 path and for shapes the tensor-core
+// engine does not take, the fixed-order reduction of split-K partials, and the pre-norm forward.
+#include "common.cuh"
+
+namespace loract {
+
+namespace {
+
+template <typename T> __device__ __forceinline__ float load_as_float(const T* p);
+template <> __device__ __forceinline__ float load_as_float<float>(const float* p) { return *p; }
+template <> __device__ __forceinline__ float load_as_float<__nv_bfloat16>(const __nv_bfloat16* p) {
+  return __bfloat162float(*p);
+}
+
+struct SimtParams {
+  int M, N, K;
+  int64_t sam, sak;  // element strides of A(m, k)
+  int64_t sbk, sbn;  // element strides of B(k, n)
+  int n_terms;
+  const void* A[4];
+  const void* B[4];
+  int out;
+  void* C0;
+  void* C1;
+  int64_t ldc;
+  int splits;
+  int64_t split_stride;
+  int accumulate;
+  float alpha;
+};
+
+constexpr int kTile = 64;   // output tile 64 x 64, 256 threads, 4 x 4 outputs per thread
+constexpr int kTileK = 16;
+
+template <typename TA, typename TB, typename TAcc>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(SimtParams p) {
+  __shared__ float As[kTileK][kTile + 1];
+  __shared__ float Bs[kTileK][kTile + 1];
+  const int tid = threadIdx.x;
+  const int tx = tid & 15, ty = tid >> 4;
+  const int m0 = blockIdx.y * kTile, n0 = blockIdx.x * kTile;
+  const int split = blockIdx.z;
+  const int k_per = ((p.K + p.splits - 1) / p.splits + kTileK - 1) / kTileK * kTileK;
+  const int k_begin = split * k_per;
+  const int k_end = min(p.K, k_begin + k_per);
+  TAcc acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = (TAcc)0;
+
+  for (int term = 0; term < p.n_terms; ++term) {
+    const TA* A = (const TA*)p.A[term];
+    const TB* B = (const TB*)p.B[term];
+    for (int k0 = k_begin; k0 < k_end; k0 += kTileK) {
+      // each thread loads 4 elements of each tile; the faster-varying thread index follows the
+      // contiguous dimension of the stored operand
+      for (int e = tid; e < kTile * kTileK; e += 256) {
+        int mm, kk;
+        if (p.sak == 1) { kk = e % kTileK; mm = e / kTileK; } else { mm = e % kTile; kk = e / kTile; }
+        const int m = m0 + mm, k = k0 + kk;
+        As[kk][mm] = (m < p.M && k < k_end) ? load_as_float(A + m * p.sam + k * p.sak) : 0.f;
+      }
+      for (int e = tid; e < kTile * kTileK; e += 256) {
+        int nn, kk;
+        if (p.sbk == 1) { kk = e % kTileK; nn = e / kTileK; } else { nn = e % kTile; kk = e / kTile; }
+        const int n = n0 + nn, k = k0 + kk;
+        Bs[kk][nn] = (n < p.N && k < k_end) ? load_as_float(B + k * p.sbk + n * p.sbn) : 0.f;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int kk = 0; kk < kTileK; ++kk) {
+        float a[4], b[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] += (TAcc)a[i] * (TAcc)b[j];
+      }
+      __syncthreads();
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + ty * 4 + i;
+    if (m >= p.M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n >= p.N) continue;
+      const int64_t off = (int64_t)m * p.ldc + n;
+      const TAcc v = acc[i][j] * (TAcc)p.alpha;
+      if (p.out == OUT_F32) {
+        float* c = (float*)p.C0 + (int64_t)split * p.split_stride + off;
+        *c = p.accumulate ? (*c + (float)v) : (float)v;
+      } else if (p.out == OUT_F64) {
+        ((double*)p.C0)[(int64_t)split * p.split_stride + off] = (double)v;
+      } else if (p.out == OUT_BF16) {
+        ((__nv_bfloat16*)p.C0)[off] = __float2bfloat16((float)v);
+      } else {
+        const float f = (float)v;
+        const __nv_bfloat16 hi = __float2bfloat16(f);
+        ((__nv_bfloat16*)p.C0)[off] = hi;
+        ((__nv_bfloat16*)p.C1)[off] = __float2bfloat16(f - __bfloat162float(hi));
+      }
+    }
+  }
+}
+
+__global__ void reduce_partials_kernel(const float* __restrict__ partials, int n_partials,
+                                       int64_t stride, int64_t count, float* __restrict__ out_f32,
+                                       __nv_bfloat16* __restrict__ out_bf16) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    float s = 0.f;
+    for (int q = 0; q < n_partials; ++q) s += partials[(int64_t)q * stride + i];
+    if (out_f32) out_f32[i] = s;
+    if (out_bf16) out_bf16[i] = __float2bfloat16(s);
+  }
+}
+
+// One warp per row.  RMS: rstd = 1/sqrt(mean x^2 + eps).  LayerNorm: mean first, then the centred
+// second moment (two passes over the row, which stays in L1/L2), A = (x - mean) rstd gamma + beta.
+template <typename T>
+__global__ void __launch_bounds__(256) norm_forward_kernel(const T* __restrict__ X, int64_t n, int64_t d,
+                                                           int64_t ldx, const T* __restrict__ gamma,
+                                                           const T* __restrict__ beta, float eps, int kind,
+                                                           T* __restrict__ A, int64_t lda,
+                                                           float* __restrict__ rstd_out,
+                                                           float* __restrict__ mean_out) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= n) return;
+  const T* x = X + row * ldx;
+  float mean = 0.f;
+  if (kind == LORACT_NORM_LAYER) {
+    float s = 0.f;
+    for (int64_t j = lane; j < d; j += 32) s += load_as_float(x + j);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    mean = s / (float)d;
+  }
+  float ss = 0.f;
+  for (int64_t j = lane; j < d; j += 32) {
+    const float v = load_as_float(x + j) - mean;
+    ss += v * v;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float rstd = rsqrtf(ss / (float)d + eps);
+  if (lane == 0) {
+    rstd_out[row] = rstd;
+    if (mean_out) mean_out[row] = mean;
+  }
+  T* a = A + row * lda;
+  for (int64_t j = lane; j < d; j += 32) {
+    float v = (load_as_float(x + j) - mean) * rstd * load_as_float(gamma + j);
+    if (beta) v += load_as_float(beta + j);
+    if constexpr (sizeof(T) == 2) a[j] = __float2bfloat16(v); else a[j] = v;
+  }
+}
+
+template <typename TA, typename TB>
+cudaError_t launch_simt_typed(const SimtParams& p, bool acc64, cudaStream_t stream) {
+  dim3 grid((p.N + kTile - 1) / kTile, (p.M + kTile - 1) / kTile, p.splits);
+  if (acc64) gemm_simt_kernel<TA, TB, double><<<grid, 256, 0, stream>>>(p);
+  else gemm_simt_kernel<TA, TB, float><<<grid, 256, 0, stream>>>(p);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t stream) {
+  SimtParams p;
+  p.M = g.M; p.N = g.N; p.K = g.K;
+  if (g.a_mn) { p.sam = 1; p.sak = g.lda; } else { p.sam = g.lda; p.sak = 1; }
+  if (g.b_mn) { p.sbn = 1; p.sbk = g.ldb; } else { p.sbn = g.ldb; p.sbk = 1; }
+  p.n_terms = g.n_terms;
+  for (int t = 0; t < 4; ++t) { p.A[t] = g.terms[t].A; p.B[t] = g.terms[t].B; }
+  p.out = g.out; p.C0 = g.C0; p.C1 = g.C1; p.ldc = g.ldc;
+  p.splits = g.splits < 1 ? 1 : g.splits;
+  p.split_stride = g.split_stride;
+  p.accumulate = g.accumulate ? 1 : 0;
+  p.alpha = g.alpha;
+  if (p.splits > 1 && !(g.out == OUT_F32 || g.out == OUT_F64)) return cudaErrorInvalidValue;
+  const bool a16 = g.a_type == ELEM_BF16, b16 = g.b_type == ELEM_BF16;
+  if (a16 && b16) return launch_simt_typed<__nv_bfloat16, __nv_bfloat16>(p, g.acc64, stream);
+  if (a16 && !b16) return launch_simt_typed<__nv_bfloat16, float>(p, g.acc64, stream);
+  if (!a16 && b16) return launch_simt_typed<float, __nv_bfloat16>(p, g.acc64, stream);
+  return launch_simt_typed<float, float>(p, g.acc64, stream);
+}
+
+cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_t stride,
+                                   int64_t count, float* out_f32, __nv_bfloat16* out_bf16,
+                                   cudaStream_t stream) {
+  int grid = (int)((count + 255) / 256);
+  if (grid > 148 * 16) grid = 148 * 16;
+  if (grid < 1) grid = 1;
+  reduce_partials_kernel<<<grid, 256, 0, stream>>>(partials, n_partials, stride, count, out_f32,
+                                                   out_bf16);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t norm_forward_launch(const void* X, int64_t n, int64_t d, int64_t ldx, int elem_type,
+                                const void* gamma, const void* beta, float eps, int kind, void* A,
+                                int64_t lda, float* rstd, float* mean, cudaStream_t stream) {
+  const int warps = 8;
+  const int grid = (int)((n + warps - 1) / warps);
+  if (elem_type == ELEM_BF16)
+    norm_forward_kernel<__nv_bfloat16><<<grid, warps * 32, 0, stream>>>(
+        (const __nv_bfloat16*)X, n, d, ldx, (const __nv_bfloat16*)gamma, (const __nv_bfloat16*)beta,
+        eps, kind, (__nv_bfloat16*)A, lda, rstd, mean);
+  else
+    norm_forward_kernel<float><<<grid, warps * 32, 0, stream>>>(
+        (const float*)X, n, d, ldx, (const float*)gamma, (const float*)beta, eps, kind, (float*)A, lda,
+        rstd, mean);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace loract
