@@ -1,0 +1,316 @@
+#!/usr/bin/env python
+"""Benchmark of the LoRAct hot path: one step = loract_compress + loract_weight_grad on one batch.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line.  `value` is GB/s of X (bytes of the activation matrix compressed and consumed
+per second, whole job).  With N > 1 (launched by torch.distributed.run) every rank runs its own batch
+-- data-parallel fine-tuning needs no collective on this path -- and the time is the max over ranks.
+`--impl reference` times the float64 CPU oracle on the same workload instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "compress+weight-grad GB/s of X"
+DEFAULT_WORKLOAD = "llama7b_block"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); smax = float(f[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": smax,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def oracle_step(Xd, Gd, w):
+    """One pass of the hot path in the float64 oracle: Algorithm 1 + the factor-form weight gradient."""
+    from oracle import loract_oracle as orc
+    U, V, _ = orc.decompose(Xd, w.rank, seed=w.seed)
+    return orc.weight_grad(U, V, Gd)
+
+
+def run_reference(args):
+    import numpy as np
+    import torch
+    from paper_2509_23472_b200 import synth
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = synth.get_workload(args.workload)
+    # bounded sample: the first n_sample token rows of the same workload (all of them when that is fast)
+    n_sample = min(w.n_tokens, 4096)
+    ws = synth.scaled(w, n_tokens=n_sample, name=w.name)
+    inp = synth.make_inputs(ws)
+    Xd, Gd = inp["X"].double().numpy(), inp["G"].double().numpy()
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(Xd, Gd, ws)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(Xd, Gd, ws)
+    dt = (time.perf_counter() - t0) / args.steps
+    gbs = n_sample * w.d * w.elem_bytes / dt / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "n_tokens": w.n_tokens, "d": w.d, "rank": w.rank, "g": w.g},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cpu_threads(), "kind": "oracle",
+                         "sample": f"first {n_sample} of {w.n_tokens} token rows, every step"},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "tokens_per_s": n_sample / dt,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--impl", default="loract", choices=["loract", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "loract" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import __graft_entry__ as entry
+    from paper_2509_23472_b200 import binding as B
+    from paper_2509_23472_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        entry.build()
+    if dist is not None:
+        dist.barrier()
+    B.lib()
+
+    w = synth.get_workload(args.workload)
+    # data-parallel replicas: every rank draws its own batch and samples its own rows
+    w_rank = synth.scaled(w, name=w.name) if rank == 0 else \
+        synth.Workload(**{**w.__dict__, "seed": w.seed + 7919 * rank})
+    inp = synth.make_inputs(w_rank, device=dev)
+    X, G = inp["X"], inp["G"]
+    N, d, r, g = w.n_tokens, w.d, w.rank, w.g
+    es = w.elem_bytes
+    desc = B.make_desc(X, r, seed=w_rank.seed, call_id=rank)
+    ws = B.alloc_workspace(desc, dev)
+    U = torch.empty(N, r, dtype=X.dtype, device=dev)
+    V = torch.empty(r, d, dtype=X.dtype, device=dev)
+    idx = torch.empty(r, dtype=torch.int32, device=dev)
+    dW = torch.empty(d, g, dtype=torch.float32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def step(Xin, Gin):
+        B.compress(Xin, r, ws=ws, out=(U, V, idx), desc=desc)
+        B.weight_grad(U, V, Gin, dW=dW, ws=ws)
+
+    def timed(fn, steps):
+        """Sum of per-step device times; L2 is flushed (256 MiB memset) before every step, outside the events."""
+        evs = []
+        for _ in range(steps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in evs]
+
+    for _ in range(args.warmup):
+        step(X, G)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = B.kernel_launch_count()
+    torch.cuda.synchronize()
+    times = timed(lambda: step(X, G), args.steps)
+    torch.cuda.synchronize()
+    launches = B.kernel_launch_count() - launches0
+    if dist is not None:
+        dist.barrier()
+    total_ms = sum(times)
+    status = B.read_device_status(ws)
+
+    # ---- end to end: inputs start in pinned host memory, the gradient is read back to the host
+    Xh, Gh = X.cpu().pin_memory(), G.cpu().pin_memory()
+    Xd2, Gd2 = torch.empty_like(X), torch.empty_like(G)
+    dWh = torch.empty(d, g, dtype=torch.float32).pin_memory()
+
+    def step_e2e():
+        Xd2.copy_(Xh, non_blocking=True)
+        Gd2.copy_(Gh, non_blocking=True)
+        step(Xd2, Gd2)
+        dWh.copy_(dW, non_blocking=True)
+
+    for _ in range(2):
+        step_e2e()
+    torch.cuda.synchronize()
+    e2e_steps = max(3, args.steps // 3)
+    e2e_ms = sum(timed(step_e2e, e2e_steps))
+    clocks = sampler.stop()
+
+    # ---- the dominant kernel alone: pass 1 of Algorithm 1, Y = X Omega^T (TMA + tcgen05), same launch shape
+    Om = torch.randn(r, d, device=dev).to(X.dtype)
+    k_ms = None
+    if X.dtype == torch.bfloat16:
+        def pass1():
+            B.debug_gemm([X], [Om], N, r, d, False, False, out_mode=B.OUT_SPLIT, engine=1)
+        for _ in range(3):
+            pass1()
+        k_times = timed(pass1, 20)
+        k_ms = statistics.mean(k_times)
+
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(t[0]), float(t[1])
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    ms_per_step = total_ms / args.steps
+    x_bytes = N * d * es
+    value = world * x_bytes / (ms_per_step * 1e-3) / 1e9
+    e2e_value = world * x_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9
+    # algorithmic bytes of pass 1: X read once, the test matrix read once, Y written once as a bf16 pair
+    k_bytes = N * d * es + r * d * es + N * r * 4
+    roofline = None
+    if k_ms is not None:
+        achieved = k_bytes / (k_ms * 1e-3) / 1e9
+        roofline = {"kernel": "gemm_tc_kernel<K-major,K-major> (Y = X Omega^T)", "bound": "hbm",
+                    "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                    "traffic": None, "ms_per_launch": k_ms, "algorithmic_bytes": k_bytes,
+                    "tflops": 2.0 * N * d * r / (k_ms * 1e-3) / 1e12}
+    # whole-step floor: X once + factors + gathered rows (strict), against measured HBM bandwidth
+    strict_bytes = x_bytes + (N * r + 2 * r * d) * es + (N * r + N * g + r * d) * es + 4 * d * g
+    step_floor_ms = max(strict_bytes / (peaks["hbm_gbs"] * 1e9), 4.0 * N * d * r / (peaks["bf16_tflops"] * 1e12)) * 1e3
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        n_sample = min(N, 4096)
+        wsmp = synth.scaled(w, n_tokens=n_sample, name=w.name)
+        Xc = X[:n_sample].double().cpu().numpy()
+        Gc = G[:n_sample].double().cpu().numpy()
+        t0 = time.perf_counter()
+        reps = 0
+        while reps < 1 or (time.perf_counter() - t0 < 10.0 and reps < 50):
+            oracle_step(Xc, Gc, wsmp)
+            reps += 1
+        dt = (time.perf_counter() - t0) / reps
+        cpu = {"value": n_sample * d * es / dt / 1e9, "unit": "GB/s", "cores": cpu_threads(), "kind": "oracle",
+               "sample": f"first {n_sample} of {N} token rows, {reps} repetitions, float64 numpy"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "n_tokens": N, "d": d, "rank": r, "g": g,
+                   "l2": "flushed with a 256 MiB memset before every timed step",
+                   "step": "loract_compress + one loract_weight_grad (all consumers' G concatenated)",
+                   "parallelism": f"dp{world} (independent batches, no collective)"},
+        "tokens_per_s": world * N / (ms_per_step * 1e-3),
+        "step_roofline_frac": step_floor_ms / ms_per_step,
+        "ms_min": min(times), "ms_median": statistics.median(times),
+        "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": X.numel() * es + G.numel() * es,
+                "d2h_bytes_per_step": dW.numel() * 4, "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": int(launches), "device_status": status, "clocks": clocks,
+        "roofline": roofline, "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

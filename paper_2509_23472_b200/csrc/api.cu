@@ -89,7 +89,7 @@ void carve_basis(Carver& c, const Plan& p, BasisWs* w) {
   if (p.bf16) {
     w->Lh = (__nv_bfloat16*)c.take(l * l * 2);
     w->Ll = (__nv_bfloat16*)c.take(l * l * 2);
-    w->sb_scratch = c.take((l * l + l * 32) * sizeof(float));
+    w->sb_scratch = c.take((l * l + (l + 31) / 32 * 1024) * sizeof(float));
     const size_t gs = (size_t)(p.splits_gs > p.splits_w ? p.splits_gs : p.splits_w);
     w->gram_partials = (float*)c.take(gs * l * l * 4);
     w->Yh = (__nv_bfloat16*)c.take(n * l * 2);
@@ -99,7 +99,7 @@ void carve_basis(Carver& c, const Plan& p, BasisWs* w) {
     w->v_partials = (float*)c.take((p.splits_v > 1 ? (size_t)p.splits_v : 0) * l * d * 4);
   } else {
     w->Linv32 = (float*)c.take(l * l * 4);
-    w->sb_scratch = c.take((l * l + l * 32) * sizeof(double));
+    w->sb_scratch = c.take((l * l + (l + 31) / 32 * 1024) * sizeof(double));
     w->gram64 = (double*)c.take(l * l * 8);
     w->Y32 = (float*)c.take(n * l * 4);
     w->Q32 = (float*)c.take(n * l * 4);

@@ -83,7 +83,7 @@ cudaError_t gaussian_rows_launch(uint64_t seed, uint64_t call_id, int l, int64_t
 // stride r, consecutive partials `partial_stride` elements apart) computes the inverse of the
 // Cholesky factor of  W + shift_rel * mean(diag W) * I :  Linv = L^{-1} (lower triangular), so that
 // (Y Linv^T) has orthonormal columns when W = Y^T Y.  Outputs (any may be null): Linv as an fp32 or
-// fp64 matrix, and as a bf16 hi/lo pair.  `scratch` holds 2 r*r elements of the compute type.
+// fp64 matrix, and as a bf16 hi/lo pair.  `scratch` holds r*r + 1024*ceil(r/32) elements of the compute type.
 struct SmallBlockArgs {
   int r = 0;
   const void* partials = nullptr;

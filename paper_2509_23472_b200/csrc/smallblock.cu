@@ -29,7 +29,7 @@ struct SBParams {
   int partial_is_f64;
   int n_partials;
   int64_t partial_stride;
-  void* scratch;       // T[r*r] (W, then L in its lower triangle) + T[r*32] (inverses of diagonal blocks)
+  void* scratch;       // T[r*r] (W, then L in its lower triangle) + T[1024*ceil(r/32)] (inverses of diagonal blocks)
   float shift_rel;
   void* linv_full;     // T, r x r, or null
   float* linv_f32;
