@@ -141,6 +141,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="loract", choices=["loract", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="run only the dominant kernel (pass 1) a few times: the small case for profiler captures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "loract" else args.warmup
     if args.impl == "reference":
@@ -201,6 +203,15 @@ def main():
             evs.append((e0, e1))
         torch.cuda.synchronize()
         return [a.elapsed_time(b) for a, b in evs]
+
+    if args.kernel_only:
+        Om = torch.randn(r, d, device=dev).to(X.dtype)
+        for _ in range(args.warmup + args.steps):
+            flush.zero_()
+            B.debug_gemm([X], [Om], N, r, d, False, False, out_mode=B.OUT_SPLIT, engine=1)
+        torch.cuda.synchronize()
+        print(json.dumps({"kernel_only": True, "launches": args.warmup + args.steps}))
+        return
 
     for _ in range(args.warmup):
         step(X, G)
