@@ -109,6 +109,27 @@ loract_status_t loract_compress_prenorm(const loract_desc_t* desc, const void* X
                                         float* rstd, float* mean, void* U, void* V, int32_t* idx_out,
                                         void* ws, size_t ws_bytes, void* stream);
 
+/* The same result as loract_weight_grad, for callers that cannot allocate device memory and so cannot
+ * provide `ws`.  (The paper has no counterpart: this is a property of the library, not of the method.)
+ * Typical callers: a backward hook running while the framework's caching allocator is locked or out of
+ * memory, a runtime with a memory plan fixed ahead of time, a process in which another component owns
+ * cudaMalloc.  The intermediate T = U^T G lives in a fixed 1 MiB array inside the library image, which
+ * every GPU that loads the library holds until the process exits.  The call itself allocates nothing: no
+ * cudaMalloc, no cudaFree, no allocating library routine.
+ *   - Limit: 256 + 2 * (4 * rank * g rounded up to 256) bytes must fit in the 1 MiB, i.e. rank * g <= 131040
+ *     (every valid rank <= 512 with g <= 255; rank 512 with g = 256 does not fit).  Beyond it the call
+ *     returns LORACT_ERR_UNSUPPORTED and launches nothing.  Other argument rules as loract_weight_grad.
+ *   - The first call on each device looks up the array's device address (the device must be current);
+ *     make that first call before any stream capture begins.
+ *   - All calls share the one array, which keeps the previous call's contents; the call clears what must
+ *     start at zero.  Two calls that overlap on the GPU (different streams, or different threads) race
+ *     on it: serialise them.
+ *   - The device status word of this entry point is the first word of that array; it is not readable
+ *     through loract_read_device_status. */
+loract_status_t loract_weight_grad_static(const loract_desc_t* desc, const void* U, const void* V,
+                                          const void* G, int32_t g, int64_t ldg, float* dW, int accumulate,
+                                          void* stream);
+
 /* Comparator of Section 3.2: randomized SVD at the same rank -- Algorithm 1 with a Gaussian test matrix
  * of rank + oversample columns (Philox + Box-Muller, counter word 1 set to 1) and `power_iters`
  * iterations of Y = X (X^T Q).  Writes the un-truncated pair: Uq (n_tokens x l), B (l x d), l = rank +

@@ -21,7 +21,7 @@ DEV_PIVOT_CLAMPED, DEV_WAIT_EXPIRED, DEV_SAMPLER_SHORT, DEV_NONFINITE = 1, 2, 4,
 
 EXPORTS = (
     "loract_workspace_bytes", "loract_sample_indices", "loract_compress", "loract_reconstruct",
-    "loract_weight_grad", "loract_compress_prenorm", "loract_rsvd_workspace_bytes", "loract_rsvd",
+    "loract_weight_grad", "loract_weight_grad_static", "loract_compress_prenorm", "loract_rsvd_workspace_bytes", "loract_rsvd",
     "loract_read_device_status", "loract_status_string", "loract_kernel_launch_count",
 )
 
@@ -60,6 +60,8 @@ def lib() -> ctypes.CDLL:
         l.loract_reconstruct.argtypes = [dp, vp, vp, vp, vp]
         l.loract_weight_grad.restype = ctypes.c_int
         l.loract_weight_grad.argtypes = [dp, vp, vp, vp, i32, i64, vp, ctypes.c_int, vp, sz, vp]
+        l.loract_weight_grad_static.restype = ctypes.c_int
+        l.loract_weight_grad_static.argtypes = [dp, vp, vp, vp, i32, i64, vp, ctypes.c_int, vp]
         l.loract_compress_prenorm.restype = ctypes.c_int
         l.loract_compress_prenorm.argtypes = [dp, vp, vp, vp, ctypes.c_float, i32, vp, vp, vp, vp, vp, vp,
                                               vp, sz, vp]
@@ -188,6 +190,24 @@ def weight_grad(U: torch.Tensor, V: torch.Tensor, G: torch.Tensor, dW: Optional[
     _check(lib().loract_weight_grad(ctypes.byref(desc), _ptr(U), _ptr(V), _ptr(G), g, G.stride(0), _ptr(dW),
                                     1 if accumulate else 0, _ptr(ws), ws.numel(), _stream(U.device)),
            "loract_weight_grad")
+    return dW
+
+
+def weight_grad_static(U: torch.Tensor, V: torch.Tensor, G: torch.Tensor, dW: torch.Tensor,
+                       accumulate: bool = False) -> torch.Tensor:
+    """dW = (U V)^T G without a workspace: for callers that cannot allocate device memory (a backward hook
+    under a locked or exhausted allocator, a fixed memory plan).  The caller passes the output too; the
+    intermediate lives in a fixed 1 MiB array inside the library, shared by all calls -- do not overlap
+    two of them on the GPU.  Raises LoractError(2) when rank * g exceeds what that array holds."""
+    _cuda(U, "U"); _cuda(V, "V"); _cuda(G, "G"); _cuda(dW, "dW")
+    n, r = U.shape
+    d = V.shape[1]
+    g = G.shape[1]
+    if G.stride(1) != 1 or dW.shape != (d, g) or dW.dtype != torch.float32 or not dW.is_contiguous():
+        raise ValueError("G must be row-major and dW a contiguous fp32 (d x g) tensor")
+    desc = Desc(n, d, d, r, 0, _dtype_code(U), 0, 0, 0)
+    _check(lib().loract_weight_grad_static(ctypes.byref(desc), _ptr(U), _ptr(V), _ptr(G), g, G.stride(0), _ptr(dW),
+                                           1 if accumulate else 0, _stream(U.device)), "loract_weight_grad_static")
     return dW
 
 
