@@ -12,7 +12,7 @@ CSRC = os.path.join(HERE, "csrc")
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libloract.so")
 OBJ_DIR = os.path.join(HERE, "_build")
-SOURCES = ["api.cu", "sampler.cu", "simt.cu", "smallblock.cu", "gemm_tc.cu", "static_scratch.cu"]
+SOURCES = ["api.cu", "sampler.cu", "simt.cu", "smallblock.cu", "smallblock_cluster.cu", "gemm_tc.cu", "static_scratch.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

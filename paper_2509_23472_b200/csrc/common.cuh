@@ -100,6 +100,10 @@ struct SmallBlockArgs {
   uint32_t* dev_status = nullptr;
 };
 cudaError_t small_block_launch(const SmallBlockArgs& a, cudaStream_t stream);
+// The same computation for r <= 256 in fp32 from fp32 partials, entirely in the shared memory of a
+// cluster of eight CTAs (no scratch).  small_block_launch uses it whenever it applies.
+bool small_block_cluster_supported(const SmallBlockArgs& a);
+cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t stream);
 
 // ---------------------------------------------------------------- elementwise helpers
 // out = sum_s partials[s] (fixed order), written as fp32 and/or bf16.

@@ -150,9 +150,11 @@ small_block_kernel(SBParams p) {
 #pragma unroll
       for (int k = 0; k < kNB; ++k) {
         T akk = __shfl_sync(0xffffffffu, a[k], k);
-        if (!(akk > pivot_floor)) { akk = pivot_floor; clamped = true; }
+        // a pivot that is not safely positive is replaced by the floor and its column is dropped
+        const bool bad = !(akk > pivot_floor);
+        if (bad) { akk = pivot_floor; clamped = true; }
         const T rinv = rsqrt_t<T>(akk);
-        const T lik = (lane == k) ? akk * rinv : ((lane > k) ? a[k] * rinv : (T)0);
+        const T lik = (lane == k) ? akk * rinv : ((lane > k && !bad) ? a[k] * rinv : (T)0);
         a[k] = lik;
 #pragma unroll
         for (int j = k + 1; j < kNB; ++j) {
@@ -271,6 +273,7 @@ cudaError_t launch_typed(const SBParams& p, cudaStream_t stream) {
 }  // namespace
 
 cudaError_t small_block_launch(const SmallBlockArgs& a, cudaStream_t stream) {
+  if (small_block_cluster_supported(a)) return small_block_cluster_launch(a, stream);
   SBParams p;
   p.r = a.r;
   p.partials = a.partials;

@@ -1,0 +1,519 @@
+// Small-block factorisation for r <= 256, fp32: Cholesky factor of an r x r Gram matrix and the inverse
+// of that factor (the serial part of the orthonormalisation, Algorithm 1 line 7 done through Gram
+// matrices), as one thread-block-cluster kernel whose working set never leaves shared memory.
+//
+// The matrix is cut into 32 x 32 blocks.  Eight CTAs form a cluster:
+//   * CTA 0 is the pivot chain.  For block column k one warp factors the diagonal block in registers
+//     (shuffles) and inverts it; the CTA then forms L(k+1,k) = A(k+1,k) D_k^{-T} and applies it to the next
+//     diagonal block itself, so the chain waits for nothing but the two blocks it needs next.
+//   * CTAs 1..7 own all blocks (dealt out column by column).  Half of their warps do the factorisation:
+//     for column k each forms its L(i,k), then updates its trailing blocks, A(i,j) -= L(i,k) L(j,k)^T; the
+//     two blocks the chain needs next, (k+2,k+1) and (k+2,k+2), are updated first and sent to CTA 0.
+//     The other half computes the inverse X = L^{-1} by block columns,
+//     X(i,j) = -D_i^{-1} sum_c L(i,c) X(c,j), one block row per step, behind the factorisation.
+//   * Every finished block (D_k^{-1}, L(i,k)) is written into the same slot of every worker's shared
+//     memory with asynchronous distributed-shared-memory stores that count bytes on an mbarrier of the
+//     receiving CTA (st.async ... mbarrier::complete_tx), so each worker ends up with a full copy of L
+//     without a global-memory round trip, a fence or a remote arrive.
+// Every wait is bounded by a wall-clock limit; on expiry the CTA records LORACT_DEV_WAIT_EXPIRED, stops
+// waiting and runs to its end (results are then invalid but every access stays in bounds).
+#include "common.cuh"
+
+namespace loract {
+
+namespace {
+
+constexpr int kB = 32;                   // block edge
+constexpr int kLd = 36;                  // padded row stride of a block slot (floats): rows 16-byte aligned
+constexpr int kSlot = kB * kLd;          // floats per slot
+constexpr int kSlotTx = kB * kB * 4;     // bytes one pushed block adds to a barrier's transaction count
+constexpr int kMaxBlk = 8;               // r <= 256
+constexpr int kCl = 8;                   // CTAs per cluster
+constexpr int kWorkers = kCl - 1;
+constexpr int kCThreads = 512;
+constexpr int kGroup = 256;              // threads of a warp group (8 warps, 4 block rows each)
+constexpr int kMaxTri = kMaxBlk * (kMaxBlk + 1) / 2;
+constexpr int kXSlots = kMaxBlk;         // inverse blocks of the block columns one CTA owns
+constexpr uint64_t kClusterWaitNs = 50000000ull;  // 50 ms
+
+struct SCParams {
+  int r;
+  const float* partials;
+  int n_partials;
+  int64_t partial_stride;
+  float shift_rel;
+  float* linv_f32;
+  __nv_bfloat16* linv_hi;
+  __nv_bfloat16* linv_lo;
+  uint32_t* dev_status;
+};
+
+__device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }
+
+// Worker (1..7) that owns block (i, j), i >= j: blocks are dealt out in column-major order, so the blocks
+// of one column sit on different CTAs.
+__device__ __forceinline__ int owner_of(int i, int j, int nblk) {
+  const int n = j * nblk - j * (j - 1) / 2 + (i - j);
+  return 1 + n % kWorkers;
+}
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, int rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float4 v) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z),
+               "f"(v.w)
+               : "memory");
+}
+// 16 bytes into another CTA's shared memory; on arrival 16 is taken off the transaction count of `bar`
+// (an mbarrier of the same CTA).
+__device__ __forceinline__ void st_async_v4(uint32_t addr, float4 v, uint32_t bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void bar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void bar_expect(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool bar_try(uint64_t* bar) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], 0;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_addr(bar))
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Every barrier of this kernel completes exactly once (phase 0).  Called by ONE thread of a warp group;
+// the others block on the named barrier that follows, so that waiting costs no issue slots.  Returns
+// false once the CTA has given up.
+__device__ __forceinline__ bool bar_wait(uint64_t* bar, volatile int* gave_up) {
+  if (bar_try(bar)) return true;
+  if (*gave_up) return false;
+  uint64_t t0 = 0;
+  for (uint32_t spin = 1;; ++spin) {
+    if (bar_try(bar)) return true;
+    __nanosleep(20);
+    if ((spin & 255u) == 0u) {
+      if (*gave_up) return false;
+      const uint64_t now = timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kClusterWaitNs) { *gave_up = 1; return false; }
+    }
+  }
+}
+__device__ __forceinline__ void group_sync(int id) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(kGroup) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// acc[rr] += sum_q A[rr][q] * B[lane][q], q < 32: R rows of a block against all 32 rows of another.
+template <int R>
+__device__ __forceinline__ void mac_nt(float (&acc)[R], const float* __restrict__ a_rows,
+                                       const float* __restrict__ b_row) {
+#pragma unroll
+  for (int q4 = 0; q4 < kB / 4; ++q4) {
+    const float4 b = *reinterpret_cast<const float4*>(b_row + 4 * q4);
+#pragma unroll
+    for (int rr = 0; rr < R; ++rr) {
+      const float4 a = *reinterpret_cast<const float4*>(a_rows + rr * kLd + 4 * q4);
+      acc[rr] = fmaf(a.x, b.x, acc[rr]);
+      acc[rr] = fmaf(a.y, b.y, acc[rr]);
+      acc[rr] = fmaf(a.z, b.z, acc[rr]);
+      acc[rr] = fmaf(a.w, b.w, acc[rr]);
+    }
+  }
+}
+
+// One warp holds rows [row0, row0 + 4) of a block (v[rr]: row row0 + rr, column = lane).  Writes them
+// into `slot_local` (if keep_local) and sends them to the same slot of the CTAs first_dst .. last_dst,
+// counting the bytes on each receiver's barrier `bar_local` (same address in every CTA).
+__device__ __forceinline__ void send_rows4(const float (&v)[4], float* stage /* 4 x 32 floats, warp-private */,
+                                           float* slot_local, int row0, const uint64_t* bar_local,
+                                           int first_dst, int last_dst, bool keep_local, int lane) {
+#pragma unroll
+  for (int rr = 0; rr < 4; ++rr) stage[rr * kB + lane] = v[rr];
+  __syncwarp();
+  // 4 rows x 8 float4: lane -> (row = lane / 8, quad = lane % 8)
+  const int rr = lane >> 3, q4 = lane & 7;
+  const float4 val = *reinterpret_cast<const float4*>(stage + rr * kB + 4 * q4);
+  float* dst_local = slot_local + (row0 + rr) * kLd + 4 * q4;
+  if (keep_local) *reinterpret_cast<float4*>(dst_local) = val;
+  const uint32_t dst_addr = smem_addr(dst_local), bar_addr = smem_addr(bar_local);
+  for (int c = first_dst; c <= last_dst; ++c) st_async_v4(map_to_cta(dst_addr, c), val, map_to_cta(bar_addr, c));
+  __syncwarp();
+}
+
+// Cholesky factor of one 32 x 32 diagonal block and the inverse of that factor, by one warp in registers:
+// lane i holds row i of the block and row i of the inverse.  Right-looking in both: once column k of L
+// is known, every later row takes its multiple of row k off -- no serial dot products.  Writes D^{-1}
+// (lower triangular, zeros above) into `slot`.  Returns true if a pivot was clamped.
+__device__ __forceinline__ bool factor_diag_block(float* slot, float pivot_floor, int lane) {
+  float a[kB], x[kB];
+#pragma unroll
+  for (int j = 0; j < kB; ++j) {
+    a[j] = (j < lane) ? slot[lane * kLd + j] : 0.f;
+    x[j] = (j == lane) ? 1.f : 0.f;
+  }
+  float diag = slot[lane * kLd + lane];
+  bool clamped = false;
+#pragma unroll
+  for (int k = 0; k < kB; ++k) {
+    float akk = __shfl_sync(0xffffffffu, diag, k);
+    // a pivot that is not safely positive is replaced by the floor and its column is dropped (entries
+    // below such a pivot are rounding noise; dividing them by the tiny pivot would overflow later columns)
+    const bool bad = !(akk > pivot_floor);
+    if (bad) { akk = pivot_floor; clamped = true; }
+    const float rinv = rsqrtf(akk);
+    const float lik = (lane > k && !bad) ? a[k] * rinv : 0.f;   // L[lane][k]
+    diag = fmaf(-lik, lik, diag);
+    // row k of the inverse is final: X[k][j] = x_k[j] / L[k][k]; rows below take L[i][k] X[k][j] off
+#pragma unroll
+    for (int j = 0; j <= k; ++j) {
+      const float xkj = __shfl_sync(0xffffffffu, x[j], k) * rinv;
+      x[j] = (lane == k) ? xkj : fmaf(-lik, xkj, x[j]);
+    }
+#pragma unroll
+    for (int j = k + 1; j < kB; ++j) {
+      const float ljk = __shfl_sync(0xffffffffu, lik, j);
+      a[j] = fmaf(-lik, ljk, a[j]);
+    }
+  }
+  __syncwarp();
+#pragma unroll
+  for (int j = 0; j < kB; ++j) slot[lane * kLd + j] = x[j];
+  __syncwarp();
+  return clamped;
+}
+
+__global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCParams p) {
+  extern __shared__ __align__(16) unsigned char sc_smem[];
+  // all barriers complete once; the same layout in every CTA, so a local address maps to any peer
+  __shared__ __align__(8) uint64_t dinv_bar[kMaxBlk];    // workers: D_k^{-1} has arrived
+  __shared__ __align__(8) uint64_t panel_bar[kMaxBlk];   // workers: every L(i,k), i > k, has arrived
+  __shared__ __align__(8) uint64_t chain_bar[kMaxBlk];   // CTA 0: blocks (j, j-1) and (j, j) have arrived
+  __shared__ float s_red[kCThreads / 32];
+  __shared__ float s_shift, s_floor;
+  __shared__ int s_gave_up;
+  __shared__ int s_clamped;
+  // blocks (i, j) owned by this CTA, in column-major order
+  __shared__ unsigned char s_mine_i[kMaxTri], s_mine_j[kMaxTri];
+  __shared__ int s_n_mine;
+
+  float* slots = reinterpret_cast<float*>(sc_smem);        // kMaxTri slots: the matrix, then L / D^{-1}
+  float* xt = slots + kMaxTri * kSlot;                      // kXSlots slots: transposed inverse blocks
+  float* tt = xt + kXSlots * kSlot;                         // 2 slots: transposed partial sums
+  float* stage = tt + 2 * kSlot;                            // 16 warps x 128 floats
+
+  uint32_t rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+  const int cta = (int)rank;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int r = p.r;
+  const int nblk = (r + kB - 1) / kB;
+  const int ntri = nblk * (nblk + 1) / 2;
+  float* my_stage = stage + warp * 4 * kB;
+
+  if (tid == 0) {
+    for (int k = 0; k < kMaxBlk; ++k) {
+      bar_init(&dinv_bar[k], 1);
+      bar_init(&panel_bar[k], 1);
+      bar_init(&chain_bar[k], 1);
+    }
+    s_gave_up = 0;
+    s_clamped = 0;
+    int n = 0;
+    for (int bj = 0; bj < nblk; ++bj)
+      for (int bi = bj; bi < nblk; ++bi)
+        if (owner_of(bi, bj, nblk) == cta) { s_mine_i[n] = (unsigned char)bi; s_mine_j[n] = (unsigned char)bj; ++n; }
+    s_n_mine = n;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // the byte counts every barrier will receive are known up front
+    for (int k = 0; k < nblk; ++k) {
+      if (cta != 0) {
+        bar_expect(&dinv_bar[k], kSlotTx);
+        if (k + 1 < nblk) bar_expect(&panel_bar[k], (uint32_t)(nblk - 1 - k) * kSlotTx);
+      } else if (k >= 2) {
+        bar_expect(&chain_bar[k], 2 * kSlotTx);
+      }
+    }
+  }
+
+  // ---- trace of W (every CTA, same order of additions) -> diagonal shift and pivot floor
+  {
+    float t = 0.f;
+    for (int i = tid; i < r; i += kCThreads) {
+      float d = 0.f;
+      for (int q = 0; q < p.n_partials; ++q) d += __ldg(p.partials + (int64_t)q * p.partial_stride + (int64_t)i * r + i);
+      t += d;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    if (lane == 0) s_red[warp] = t;
+    __syncthreads();
+    if (tid == 0) {
+      float tr = 0.f;
+      for (int q = 0; q < kCThreads / 32; ++q) tr += s_red[q];
+      float mean_diag = tr / (float)r;
+      if (!(mean_diag == mean_diag) || mean_diag > 3.0e38f || mean_diag < 0.f) {
+        if (p.dev_status && cta == 0) atomicOr(p.dev_status, LORACT_DEV_NONFINITE);
+        mean_diag = 1.f;
+      }
+      if (mean_diag == 0.f) mean_diag = 1.f;
+      s_shift = p.shift_rel * mean_diag;
+      s_floor = mean_diag * 1e-7f;
+    }
+    __syncthreads();
+  }
+
+  // ---- load: block t is summed over the partials by CTA t mod 8 and written into the slot of the CTA
+  // that works on it first (CTA 0 for block rows 0 and 1, the owner otherwise)
+  {
+    const float shift = s_shift;
+    for (int t = cta; t < ntri; t += kCl) {
+      int bi = 0;
+      while (tri(bi + 1, 0) <= t) ++bi;
+      const int bj = t - tri(bi, 0);
+      const int dst_cta = bi <= 1 ? 0 : owner_of(bi, bj, nblk);
+      const uint32_t dst = map_to_cta(smem_addr(slots + t * kSlot), dst_cta);
+      for (int e = tid; e < kB * (kB / 4); e += kCThreads) {
+        const int a = e >> 3, q4 = e & 7;
+        const int row = bi * kB + a, col = bj * kB + 4 * q4;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row < r && col < r) {
+          const float* src = p.partials + (int64_t)row * r + col;
+          for (int q = 0; q < p.n_partials; ++q) {
+            const float4 v = __ldg(reinterpret_cast<const float4*>(src + (int64_t)q * p.partial_stride));
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+          }
+        }
+        if (bi == bj) {
+          const int dcol = a - 4 * q4;  // position of the diagonal element inside this quad, if any
+          const float add = row < r ? shift : 1.f;  // padding rows of a ragged last block: identity
+          if (dcol == 0) s.x += add; else if (dcol == 1) s.y += add; else if (dcol == 2) s.z += add; else if (dcol == 3) s.w += add;
+        }
+        st_cluster_v4(dst + (uint32_t)((a * kLd + 4 * q4) * 4), s);
+      }
+    }
+  }
+  cluster_sync_all();
+
+  if (cta == 0) {
+    // =========================================================== pivot chain (warps 0..7)
+    if (warp < 8) {
+      for (int k = 0; k < nblk; ++k) {
+        float* dslot = slots + tri(k, k) * kSlot;
+        if (warp == 0) {
+          if (factor_diag_block(dslot, s_floor, lane) && lane == 0) s_clamped = 1;
+        } else if (tid == 32 && k + 1 < nblk && k >= 1) {
+          bar_wait(&chain_bar[k + 1], &s_gave_up);   // blocks (k+1, k) and (k+1, k+1)
+        }
+        group_sync(1);
+        const int row0 = warp * 4;
+        {  // D_k^{-1} to every worker
+          const int rr = lane >> 3, q4 = lane & 7;
+          const float* src = dslot + (row0 + rr) * kLd + 4 * q4;
+          const float4 val = *reinterpret_cast<const float4*>(src);
+          const uint32_t a0 = smem_addr(src), b0 = smem_addr(&dinv_bar[k]);
+          for (int c = 1; c < kCl; ++c) st_async_v4(map_to_cta(a0, c), val, map_to_cta(b0, c));
+        }
+        if (k + 1 < nblk) {
+          // L(k+1, k) = A(k+1, k) D_k^{-T}
+          float* sub = slots + tri(k + 1, k) * kSlot;
+          float acc[4] = {0.f, 0.f, 0.f, 0.f};
+          mac_nt<4>(acc, sub + row0 * kLd, dslot + lane * kLd);
+          __syncwarp();
+          send_rows4(acc, my_stage, sub, row0, &panel_bar[k], 1, kCl - 1, true, lane);
+          group_sync(1);
+          // next diagonal block: A(k+1, k+1) -= L(k+1, k) L(k+1, k)^T
+          float acc2[4] = {0.f, 0.f, 0.f, 0.f};
+          mac_nt<4>(acc2, sub + row0 * kLd, sub + lane * kLd);
+          float* dst = slots + tri(k + 1, k + 1) * kSlot + row0 * kLd + lane;
+#pragma unroll
+          for (int rr = 0; rr < 4; ++rr) dst[rr * kLd] -= acc2[rr];
+          group_sync(1);
+        }
+      }
+      if (tid == 0 && s_clamped && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_PIVOT_CLAMPED);
+    }
+  } else if (warp < 8) {
+    // =========================================================== workers, factorisation half
+    const int row0 = warp * 4;
+    const int n_mine = s_n_mine;
+    for (int k = 0; k < nblk; ++k) {
+      if (tid == 0) bar_wait(&dinv_bar[k], &s_gave_up);
+      group_sync(1);
+      const float* dk = slots + tri(k, k) * kSlot;
+      // L(i, k) = A(i, k) D_k^{-T} for the blocks of column k this CTA owns (CTA 0 does block k + 1)
+      for (int q = 0; q < n_mine; ++q) {
+        const int bi = s_mine_i[q], bj = s_mine_j[q];
+        if (bj != k || bi < k + 2) continue;
+        float* blk = slots + tri(bi, k) * kSlot;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        mac_nt<4>(acc, blk + row0 * kLd, dk + lane * kLd);
+        __syncwarp();
+        send_rows4(acc, my_stage, blk, row0, &panel_bar[k], 1, kCl - 1, false, lane);
+      }
+      if (k + 1 >= nblk) break;
+      if (tid == 0) bar_wait(&panel_bar[k], &s_gave_up);
+      group_sync(1);
+      // trailing update with column k.  Pass 0: the two blocks CTA 0 needs next, sent on as soon as they
+      // are done.  Pass 1: the rest.  A diagonal block (j, j) takes columns k <= j - 2 here (CTA 0 applies
+      // column j - 1 itself), every other block (i, j) columns k <= j - 1.
+      for (int pass = 0; pass < 2; ++pass) {
+        for (int q = 0; q < n_mine; ++q) {
+          const int bi = s_mine_i[q], bj = s_mine_j[q];
+          if (bi < 2) continue;
+          const bool active = (bi == bj) ? (k <= bj - 2) : (k <= bj - 1);
+          if (!active) continue;
+          const bool urgent = (bi == k + 2) && (bj == k + 1 || bj == k + 2);
+          if (urgent != (pass == 0)) continue;
+          float acc[4] = {0.f, 0.f, 0.f, 0.f};
+          mac_nt<4>(acc, slots + tri(bi, k) * kSlot + row0 * kLd, slots + tri(bj, k) * kSlot + lane * kLd);
+          float* blk = slots + tri(bi, bj) * kSlot;
+          float v[4];
+#pragma unroll
+          for (int rr = 0; rr < 4; ++rr) v[rr] = blk[(row0 + rr) * kLd + lane] - acc[rr];
+          if (urgent) {
+            __syncwarp();
+            send_rows4(v, my_stage, blk, row0, &chain_bar[k + 2], 0, 0, false, lane);
+          } else {
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr) blk[(row0 + rr) * kLd + lane] = v[rr];
+          }
+        }
+      }
+    }
+  } else {
+    // =========================================================== workers, inverse half (warps 8..15)
+    const int w = warp - 8;
+    const int row0 = w * 4;
+    // block columns of the inverse this CTA computes: j0 = cta - 1, and 7 as well on the last worker
+    const int j0 = cta - 1;
+    const int n_cols = (j0 < nblk ? 1 : 0) + ((cta == kWorkers && kWorkers < nblk) ? 1 : 0);
+    for (int k = 0; k < nblk; ++k) {
+      if (tid == kGroup) {
+        bar_wait(&dinv_bar[k], &s_gave_up);
+        if (k >= 1) bar_wait(&panel_bar[k - 1], &s_gave_up);
+      }
+      group_sync(2);
+      const float* dk = slots + tri(k, k) * kSlot;
+      // first half: tt[b][a] = sum_{j <= c < k} sum_q Xt(c,j)[b][q] L(k,c)[a][q]
+      for (int cidx = 0; cidx < n_cols; ++cidx) {
+        const int j = j0 + cidx;
+        if (j >= k) continue;
+        const float* xcol = xt + (cidx == 0 ? 0 : (nblk - j0)) * kSlot;  // block (c, j) at xcol + (c - j) slots
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int c = j; c < k; ++c)
+          mac_nt<4>(acc, xcol + (c - j) * kSlot + row0 * kLd, slots + tri(k, c) * kSlot + lane * kLd);
+#pragma unroll
+        for (int rr = 0; rr < 4; ++rr) tt[cidx * kSlot + (row0 + rr) * kLd + lane] = acc[rr];
+      }
+      group_sync(2);
+      // second half: Xt(k,j)[b][a] = -sum_q tt[b][q] D_k^{-1}[a][q];  Xt(k,k) = D_k^{-T}
+      for (int cidx = 0; cidx < n_cols; ++cidx) {
+        const int j = j0 + cidx;
+        if (j > k) continue;
+        float* dst = xt + ((cidx == 0 ? 0 : (nblk - j0)) + (k - j)) * kSlot;
+        if (j == k) {
+          for (int e = tid - kGroup; e < kB * kB; e += kGroup) {
+            const int b = e >> 5, a = e & 31;
+            dst[b * kLd + a] = dk[a * kLd + b];
+          }
+        } else {
+          float acc[4] = {0.f, 0.f, 0.f, 0.f};
+          mac_nt<4>(acc, tt + cidx * kSlot + row0 * kLd, dk + lane * kLd);
+#pragma unroll
+          for (int rr = 0; rr < 4; ++rr) dst[(row0 + rr) * kLd + lane] = -acc[rr];
+        }
+      }
+    }
+    group_sync(2);
+    // ---- output: Linv[i*32 + a][j*32 + b] = Xt(i,j)[b][a]; zeros above the diagonal blocks
+    for (int cidx = 0; cidx < n_cols; ++cidx) {
+      const int j = j0 + cidx;
+      const float* xcol = xt + (cidx == 0 ? 0 : (nblk - j0)) * kSlot;
+      const int ncol = min(kB, r - j * kB);
+      for (int e = tid - kGroup; e < r * kB; e += kGroup) {
+        const int row = e >> 5, b = e & 31;
+        if (b >= ncol) continue;
+        const int bi = row / kB, a = row - bi * kB;
+        const float v = (bi >= j) ? xcol[(bi - j) * kSlot + b * kLd + a] : 0.f;
+        const int64_t off = (int64_t)row * r + j * kB + b;
+        if (p.linv_f32) p.linv_f32[off] = v;
+        if (p.linv_hi) {
+          const __nv_bfloat16 hi = __float2bfloat16(v);
+          p.linv_hi[off] = hi;
+          if (p.linv_lo) p.linv_lo[off] = __float2bfloat16(v - __bfloat162float(hi));
+        }
+      }
+    }
+  }
+  __syncthreads();
+  if (tid == 0 && s_gave_up && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_WAIT_EXPIRED);
+  // no CTA leaves while another may still write into its shared memory
+  cluster_sync_all();
+}
+
+}  // namespace
+
+bool small_block_cluster_supported(const SmallBlockArgs& a) {
+  return !a.use_f64 && a.partial_type == ELEM_F32 && a.r <= kMaxBlk * kB && a.r % 4 == 0 &&
+         a.linv_full == nullptr && (((uintptr_t)a.partials & 15) == 0) && (a.partial_stride % 4 == 0);
+}
+
+cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t stream) {
+  SCParams p;
+  p.r = a.r;
+  p.partials = (const float*)a.partials;
+  p.n_partials = a.n_partials;
+  p.partial_stride = a.partial_stride;
+  p.shift_rel = a.shift_rel;
+  p.linv_f32 = a.linv_f32;
+  p.linv_hi = a.linv_hi;
+  p.linv_lo = a.linv_lo;
+  p.dev_status = a.dev_status;
+  const size_t smem = (size_t)(kMaxTri + kXSlots + 2) * kSlot * sizeof(float) + (size_t)(kCThreads / 32) * 4 * kB * sizeof(float);
+  static bool configured[64] = {};
+  int dev = 0;
+  LORACT_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    LORACT_CUDA_TRY(cudaFuncSetAttribute(small_block_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem));
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kCl, 1, 1);
+  cfg.blockDim = dim3(kCThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kCl;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  LORACT_CUDA_TRY(cudaLaunchKernelEx(&cfg, small_block_cluster_kernel, p));
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace loract
