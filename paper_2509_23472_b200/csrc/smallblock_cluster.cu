@@ -161,17 +161,19 @@ __device__ __forceinline__ void send_rows4(const float (&v)[4], float* stage /* 
   __syncwarp();
 }
 
-// Cholesky factor of one 32 x 32 diagonal block and the inverse of that factor, by one warp in registers:
-// lane i holds row i of the block and row i of the inverse.  Right-looking in both: once column k of L
-// is known, every later row takes its multiple of row k off -- no serial dot products.  Writes D^{-1}
-// (lower triangular, zeros above) into `slot`.  Returns true if a pivot was clamped.
-__device__ __forceinline__ bool factor_diag_block(float* slot, float pivot_floor, int lane) {
-  float a[kB], x[kB];
+// The 32 x 32 diagonal block is handled by two warps that run side by side.
+//
+// factor_diag_block (one warp, lane i holds row i): right-looking Cholesky in registers.  As soon as
+// column k of L is known it is published to `lcol` (lcol[k][i] = L[i][k] for i > k, 1 / L[k][k] for i = k,
+// 0 above), whose words start out as kUnset -- the consumer needs no flag and no fence, it waits for
+// each word to change.  Returns true if a pivot was clamped.
+constexpr uint32_t kUnset = 0xFFFFFFFFu;   // a NaN pattern arithmetic does not produce
+constexpr int kLcolLd = kB + 1;
+
+__device__ __forceinline__ bool factor_diag_block(const float* slot, float* lcol, float pivot_floor, int lane) {
+  float a[kB];
 #pragma unroll
-  for (int j = 0; j < kB; ++j) {
-    a[j] = (j < lane) ? slot[lane * kLd + j] : 0.f;
-    x[j] = (j == lane) ? 1.f : 0.f;
-  }
+  for (int j = 0; j < kB; ++j) a[j] = (j < lane) ? slot[lane * kLd + j] : 0.f;
   float diag = slot[lane * kLd + lane];
   bool clamped = false;
 #pragma unroll
@@ -183,24 +185,47 @@ __device__ __forceinline__ bool factor_diag_block(float* slot, float pivot_floor
     if (bad) { akk = pivot_floor; clamped = true; }
     const float rinv = rsqrtf(akk);
     const float lik = (lane > k && !bad) ? a[k] * rinv : 0.f;   // L[lane][k]
+    float pub = (lane == k) ? rinv : lik;
+    if (__float_as_uint(pub) == kUnset) pub = 0.f;
+    lcol[k * kLcolLd + lane] = pub;
     diag = fmaf(-lik, lik, diag);
-    // row k of the inverse is final: X[k][j] = x_k[j] / L[k][k]; rows below take L[i][k] X[k][j] off
-#pragma unroll
-    for (int j = 0; j <= k; ++j) {
-      const float xkj = __shfl_sync(0xffffffffu, x[j], k) * rinv;
-      x[j] = (lane == k) ? xkj : fmaf(-lik, xkj, x[j]);
-    }
 #pragma unroll
     for (int j = k + 1; j < kB; ++j) {
       const float ljk = __shfl_sync(0xffffffffu, lik, j);
       a[j] = fmaf(-lik, ljk, a[j]);
     }
   }
-  __syncwarp();
-#pragma unroll
-  for (int j = 0; j < kB; ++j) slot[lane * kLd + j] = x[j];
-  __syncwarp();
   return clamped;
+}
+
+// invert_diag_block (a second warp, lane i holds row i of the inverse): takes the columns of L as they
+// appear in `lcol` and forms X = L^{-1} right-looking: once column k is known, row k of X is final up to
+// its scale 1 / L[k][k], and every later row takes its multiple of it off -- no serial dot products.
+// Writes X (lower triangular, zeros above) into `slot`.  The wait for a column is bounded.
+__device__ __forceinline__ void invert_diag_block(float* slot, const float* lcol, volatile int* gave_up, int lane) {
+  float x[kB];
+#pragma unroll
+  for (int j = 0; j < kB; ++j) x[j] = (j == lane) ? 1.f : 0.f;
+  float my_rinv = 1.f;
+#pragma unroll
+  for (int k = 0; k < kB; ++k) {
+    const volatile uint32_t* src = reinterpret_cast<const volatile uint32_t*>(lcol + k * kLcolLd + lane);
+    uint32_t bits = *src;
+    for (uint32_t spin = 0; bits == kUnset; ++spin) {
+      if (spin > (1u << 22) || *gave_up) { *gave_up = 1; bits = 0u; break; }
+      bits = *src;
+    }
+    const float v = __uint_as_float(bits);
+    const float rinv = __shfl_sync(0xffffffffu, v, k);
+    if (lane == k) my_rinv = rinv;
+    // rows below take (L[i][k] / L[k][k]) times the unscaled row k off; rows up to k are left alone
+    const float m = (lane > k) ? v * rinv : 0.f;
+#pragma unroll
+    for (int j = 0; j <= k; ++j) x[j] = fmaf(-m, __shfl_sync(0xffffffffu, x[j], k), x[j]);
+  }
+#pragma unroll
+  for (int j = 0; j < kB; ++j) slot[lane * kLd + j] = x[j] * my_rinv;
+  __syncwarp();
 }
 
 __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCParams p) {
@@ -219,8 +244,8 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
 
   float* slots = reinterpret_cast<float*>(sc_smem);        // kMaxTri slots: the matrix, then L / D^{-1}
   float* xt = slots + kMaxTri * kSlot;                      // kXSlots slots: transposed inverse blocks
-  float* tt = xt + kXSlots * kSlot;                         // 2 slots: transposed partial sums
-  float* stage = tt + 2 * kSlot;                            // 16 warps x 128 floats
+  float* stage = xt + kXSlots * kSlot;                            // 16 warps x 128 floats
+  float* lcol = stage + (kCThreads / 32) * 4 * kB;          // columns of the diagonal block's factor
 
   uint32_t rank;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
@@ -231,22 +256,15 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
   const int ntri = nblk * (nblk + 1) / 2;
   float* my_stage = stage + warp * 4 * kB;
 
-  if (tid == 0) {
-    for (int k = 0; k < kMaxBlk; ++k) {
-      bar_init(&dinv_bar[k], 1);
-      bar_init(&panel_bar[k], 1);
-      bar_init(&chain_bar[k], 1);
-    }
-    s_gave_up = 0;
-    s_clamped = 0;
-    int n = 0;
-    for (int bj = 0; bj < nblk; ++bj)
-      for (int bi = bj; bi < nblk; ++bi)
-        if (owner_of(bi, bj, nblk) == cta) { s_mine_i[n] = (unsigned char)bi; s_mine_j[n] = (unsigned char)bj; ++n; }
-    s_n_mine = n;
+  // ---- set-up, spread over threads: barriers (with the byte counts they will receive, known up front),
+  // this CTA's block list, the sentinel words of the diagonal-block column buffer
+  if (tid < kMaxBlk) {
+    const int k = tid;
+    bar_init(&dinv_bar[k], 1);
+    bar_init(&panel_bar[k], 1);
+    bar_init(&chain_bar[k], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    // the byte counts every barrier will receive are known up front
-    for (int k = 0; k < nblk; ++k) {
+    if (k < nblk) {
       if (cta != 0) {
         bar_expect(&dinv_bar[k], kSlotTx);
         if (k + 1 < nblk) bar_expect(&panel_bar[k], (uint32_t)(nblk - 1 - k) * kSlotTx);
@@ -254,15 +272,51 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
         bar_expect(&chain_bar[k], 2 * kSlotTx);
       }
     }
+  } else if (tid == 32) {
+    s_gave_up = 0;
+    s_clamped = 0;
+    int n = 0;
+    for (int bj = 0; bj < nblk; ++bj)
+      for (int bi = bj; bi < nblk; ++bi)
+        if (owner_of(bi, bj, nblk) == cta) { s_mine_i[n] = (unsigned char)bi; s_mine_j[n] = (unsigned char)bj; ++n; }
+    s_n_mine = n;
   }
+  for (int e = tid; e < kB * kLcolLd; e += kCThreads) reinterpret_cast<uint32_t*>(lcol)[e] = kUnset;
 
-  // ---- trace of W (every CTA, same order of additions) -> diagonal shift and pivot floor
+  // ---- load.  Block t is summed over the partials by CTA t mod 8 and written into the slot of the CTA
+  // that works on it first (CTA 0 for block rows 0 and 1, the owner otherwise).  All global loads of a
+  // thread are issued before the first use; the trace of W (same order of additions in every CTA) gives
+  // the diagonal shift and the pivot floor.
   {
     float t = 0.f;
     for (int i = tid; i < r; i += kCThreads) {
       float d = 0.f;
       for (int q = 0; q < p.n_partials; ++q) d += __ldg(p.partials + (int64_t)q * p.partial_stride + (int64_t)i * r + i);
       t += d;
+    }
+    constexpr int kMaxMine = (kMaxTri + kCl - 1) / kCl;          // blocks one CTA loads
+    constexpr int kPerThread = kMaxMine * (kB * kB / 4) / kCThreads + 1;
+    float4 acc[kPerThread];
+    const int n_load = (ntri - cta + kCl - 1) / kCl;              // blocks cta, cta + 8, ...
+#pragma unroll
+    for (int u = 0; u < kPerThread; ++u) {
+      acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      const int e = tid + u * kCThreads;
+      const int lb = e >> 8;                                      // 256 quads per block
+      if (lb >= n_load) continue;
+      const int blk = cta + lb * kCl;
+      int bi = 0;
+      while (tri(bi + 1, 0) <= blk) ++bi;
+      const int bj = blk - tri(bi, 0);
+      const int a = (e & 255) >> 3, q4 = e & 7;
+      const int row = bi * kB + a, col = bj * kB + 4 * q4;
+      if (row < r && col < r) {
+        const float* src = p.partials + (int64_t)row * r + col;
+        for (int q = 0; q < p.n_partials; ++q) {
+          const float4 v = __ldg(reinterpret_cast<const float4*>(src + (int64_t)q * p.partial_stride));
+          acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
+        }
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
@@ -281,78 +335,86 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
       s_floor = mean_diag * 1e-7f;
     }
     __syncthreads();
-  }
-
-  // ---- load: block t is summed over the partials by CTA t mod 8 and written into the slot of the CTA
-  // that works on it first (CTA 0 for block rows 0 and 1, the owner otherwise)
-  {
     const float shift = s_shift;
-    for (int t = cta; t < ntri; t += kCl) {
+#pragma unroll
+    for (int u = 0; u < kPerThread; ++u) {
+      const int e = tid + u * kCThreads;
+      const int lb = e >> 8;
+      if (lb >= n_load) continue;
+      const int blk = cta + lb * kCl;
       int bi = 0;
-      while (tri(bi + 1, 0) <= t) ++bi;
-      const int bj = t - tri(bi, 0);
-      const int dst_cta = bi <= 1 ? 0 : owner_of(bi, bj, nblk);
-      const uint32_t dst = map_to_cta(smem_addr(slots + t * kSlot), dst_cta);
-      for (int e = tid; e < kB * (kB / 4); e += kCThreads) {
-        const int a = e >> 3, q4 = e & 7;
-        const int row = bi * kB + a, col = bj * kB + 4 * q4;
-        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (row < r && col < r) {
-          const float* src = p.partials + (int64_t)row * r + col;
-          for (int q = 0; q < p.n_partials; ++q) {
-            const float4 v = __ldg(reinterpret_cast<const float4*>(src + (int64_t)q * p.partial_stride));
-            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
-          }
-        }
-        if (bi == bj) {
-          const int dcol = a - 4 * q4;  // position of the diagonal element inside this quad, if any
-          const float add = row < r ? shift : 1.f;  // padding rows of a ragged last block: identity
-          if (dcol == 0) s.x += add; else if (dcol == 1) s.y += add; else if (dcol == 2) s.z += add; else if (dcol == 3) s.w += add;
-        }
-        st_cluster_v4(dst + (uint32_t)((a * kLd + 4 * q4) * 4), s);
+      while (tri(bi + 1, 0) <= blk) ++bi;
+      const int bj = blk - tri(bi, 0);
+      const int a = (e & 255) >> 3, q4 = e & 7;
+      float4 sv = acc[u];
+      if (bi == bj) {
+        const int dcol = a - 4 * q4;  // position of the diagonal element inside this quad, if any
+        const float add = (bi * kB + a) < r ? shift : 1.f;  // padding rows of a ragged last block: identity
+        if (dcol == 0) sv.x += add; else if (dcol == 1) sv.y += add; else if (dcol == 2) sv.z += add; else if (dcol == 3) sv.w += add;
       }
+      const int dst_cta = bi <= 1 ? 0 : owner_of(bi, bj, nblk);
+      const uint32_t dst = map_to_cta(smem_addr(slots + blk * kSlot), dst_cta);
+      st_cluster_v4(dst + (uint32_t)((a * kLd + 4 * q4) * 4), sv);
     }
   }
   cluster_sync_all();
 
   if (cta == 0) {
-    // =========================================================== pivot chain (warps 0..7)
-    if (warp < 8) {
-      for (int k = 0; k < nblk; ++k) {
-        float* dslot = slots + tri(k, k) * kSlot;
-        if (warp == 0) {
-          if (factor_diag_block(dslot, s_floor, lane) && lane == 0) s_clamped = 1;
-        } else if (tid == 32 && k + 1 < nblk && k >= 1) {
-          bar_wait(&chain_bar[k + 1], &s_gave_up);   // blocks (k+1, k) and (k+1, k+1)
-        }
-        group_sync(1);
-        const int row0 = warp * 4;
-        {  // D_k^{-1} to every worker
-          const int rr = lane >> 3, q4 = lane & 7;
-          const float* src = dslot + (row0 + rr) * kLd + 4 * q4;
-          const float4 val = *reinterpret_cast<const float4*>(src);
-          const uint32_t a0 = smem_addr(src), b0 = smem_addr(&dinv_bar[k]);
-          for (int c = 1; c < kCl; ++c) st_async_v4(map_to_cta(a0, c), val, map_to_cta(b0, c));
-        }
+    // =========================================================== pivot chain
+    // Phase A: warp 0 factors the diagonal block, warp 1 inverts it alongside, one thread waits for the
+    // two blocks of the next step.  Phase B: warps 0..7 form L(k+1, k); warps 8..15 send D_k^{-1} out.
+    // Phase C: warps 0..7 update the next diagonal block; warps 8..15 send L(k+1, k) out.  Sending is
+    // kept off the warps the next pivot waits for.
+    const int row0 = (warp & 7) * 4;
+    for (int k = 0; k < nblk; ++k) {
+      float* dslot = slots + tri(k, k) * kSlot;
+      if (warp == 0) {
+        if (factor_diag_block(dslot, lcol, s_floor, lane) && lane == 0) s_clamped = 1;
+      } else if (warp == 1) {
+        invert_diag_block(dslot, lcol, &s_gave_up, lane);
+      } else if (tid == 64 && k + 1 < nblk && k >= 1) {
+        bar_wait(&chain_bar[k + 1], &s_gave_up);   // blocks (k+1, k) and (k+1, k+1)
+      }
+      __syncthreads();
+      float* sub = slots + tri(k + 1 < nblk ? k + 1 : k, k) * kSlot;
+      if (warp < 8) {
         if (k + 1 < nblk) {
-          // L(k+1, k) = A(k+1, k) D_k^{-T}
-          float* sub = slots + tri(k + 1, k) * kSlot;
+          // L(k+1, k) = A(k+1, k) D_k^{-T}, in place (a warp reads only the rows it writes)
           float acc[4] = {0.f, 0.f, 0.f, 0.f};
           mac_nt<4>(acc, sub + row0 * kLd, dslot + lane * kLd);
           __syncwarp();
-          send_rows4(acc, my_stage, sub, row0, &panel_bar[k], 1, kCl - 1, true, lane);
-          group_sync(1);
-          // next diagonal block: A(k+1, k+1) -= L(k+1, k) L(k+1, k)^T
-          float acc2[4] = {0.f, 0.f, 0.f, 0.f};
-          mac_nt<4>(acc2, sub + row0 * kLd, sub + lane * kLd);
-          float* dst = slots + tri(k + 1, k + 1) * kSlot + row0 * kLd + lane;
 #pragma unroll
-          for (int rr = 0; rr < 4; ++rr) dst[rr * kLd] -= acc2[rr];
-          group_sync(1);
+          for (int rr = 0; rr < 4; ++rr) sub[(row0 + rr) * kLd + lane] = acc[rr];
         }
+      } else {
+        // D_k^{-1} to every worker
+        const int rr = lane >> 3, q4 = lane & 7;
+        const float* src = dslot + (row0 + rr) * kLd + 4 * q4;
+        const float4 val = *reinterpret_cast<const float4*>(src);
+        const uint32_t a0 = smem_addr(src), b0 = smem_addr(&dinv_bar[k]);
+        for (int c = 1; c < kCl; ++c) st_async_v4(map_to_cta(a0, c), val, map_to_cta(b0, c));
       }
-      if (tid == 0 && s_clamped && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_PIVOT_CLAMPED);
+      if (k + 1 >= nblk) break;
+      __syncthreads();
+      if (warp < 8) {
+        // next diagonal block: A(k+1, k+1) -= L(k+1, k) L(k+1, k)^T
+        float acc2[4] = {0.f, 0.f, 0.f, 0.f};
+        mac_nt<4>(acc2, sub + row0 * kLd, sub + lane * kLd);
+        float* dst = slots + tri(k + 1, k + 1) * kSlot + row0 * kLd + lane;
+#pragma unroll
+        for (int rr = 0; rr < 4; ++rr) dst[rr * kLd] -= acc2[rr];
+        for (int e = tid; e < kB * kLcolLd; e += kGroup) reinterpret_cast<uint32_t*>(lcol)[e] = kUnset;
+      } else {
+        // L(k+1, k) to every worker
+        const int rr = lane >> 3, q4 = lane & 7;
+        const float* src = sub + (row0 + rr) * kLd + 4 * q4;
+        const float4 val = *reinterpret_cast<const float4*>(src);
+        const uint32_t a0 = smem_addr(src), b0 = smem_addr(&panel_bar[k]);
+        for (int c = 1; c < kCl; ++c) st_async_v4(map_to_cta(a0, c), val, map_to_cta(b0, c));
+      }
+      __syncthreads();
     }
+    if (tid == 0 && s_clamped && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_PIVOT_CLAMPED);
   } else if (warp < 8) {
     // =========================================================== workers, factorisation half
     const int row0 = warp * 4;
@@ -403,65 +465,91 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
     }
   } else {
     // =========================================================== workers, inverse half (warps 8..15)
-    const int w = warp - 8;
-    const int row0 = w * 4;
+    // Right-looking by block rows, in transposed storage Xt(i,j)[b][a] = X(i,j)[a][b]: at step k block row
+    // k of the inverse becomes final, X(k,j) = -D_k^{-1} T(k,j) (X(k,k) = D_k^{-1}), is written out, and is
+    // added into the sums of all later rows, T(i,j) += L(i,k) X(k,j).  A warp only ever touches its own
+    // four rows b of every block (the columns of X are independent), except for the transposed copy.
+    const int gt = tid - kGroup;
+    const int row0 = (warp - 8) * 4;
     // block columns of the inverse this CTA computes: j0 = cta - 1, and 7 as well on the last worker
     const int j0 = cta - 1;
     const int n_cols = (j0 < nblk ? 1 : 0) + ((cta == kWorkers && kWorkers < nblk) ? 1 : 0);
-    for (int k = 0; k < nblk; ++k) {
-      if (tid == kGroup) {
-        bar_wait(&dinv_bar[k], &s_gave_up);
-        if (k >= 1) bar_wait(&panel_bar[k - 1], &s_gave_up);
+    // zeros above the diagonal blocks
+    for (int cidx = 0; cidx < n_cols; ++cidx) {
+      const int j = j0 + cidx;
+      const int ncol = min(kB, r - j * kB);
+      for (int e = gt; e < j * kB * kB; e += kGroup) {
+        const int row = e >> 5, b = e & 31;
+        if (b >= ncol) continue;
+        const int64_t off = (int64_t)row * r + j * kB + b;
+        if (p.linv_f32) p.linv_f32[off] = 0.f;
+        if (p.linv_hi) p.linv_hi[off] = __float2bfloat16(0.f);
+        if (p.linv_lo) p.linv_lo[off] = __float2bfloat16(0.f);
       }
+    }
+    for (int k = 0; k < nblk; ++k) {
+      if (gt == 0) bar_wait(&dinv_bar[k], &s_gave_up);
       group_sync(2);
       const float* dk = slots + tri(k, k) * kSlot;
-      // first half: tt[b][a] = sum_{j <= c < k} sum_q Xt(c,j)[b][q] L(k,c)[a][q]
-      for (int cidx = 0; cidx < n_cols; ++cidx) {
-        const int j = j0 + cidx;
-        if (j >= k) continue;
-        const float* xcol = xt + (cidx == 0 ? 0 : (nblk - j0)) * kSlot;  // block (c, j) at xcol + (c - j) slots
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int c = j; c < k; ++c)
-          mac_nt<4>(acc, xcol + (c - j) * kSlot + row0 * kLd, slots + tri(k, c) * kSlot + lane * kLd);
-#pragma unroll
-        for (int rr = 0; rr < 4; ++rr) tt[cidx * kSlot + (row0 + rr) * kLd + lane] = acc[rr];
-      }
-      group_sync(2);
-      // second half: Xt(k,j)[b][a] = -sum_q tt[b][q] D_k^{-1}[a][q];  Xt(k,k) = D_k^{-T}
       for (int cidx = 0; cidx < n_cols; ++cidx) {
         const int j = j0 + cidx;
         if (j > k) continue;
         float* dst = xt + ((cidx == 0 ? 0 : (nblk - j0)) + (k - j)) * kSlot;
         if (j == k) {
-          for (int e = tid - kGroup; e < kB * kB; e += kGroup) {
+          for (int e = gt; e < kB * kB; e += kGroup) {
             const int b = e >> 5, a = e & 31;
             dst[b * kLd + a] = dk[a * kLd + b];
           }
         } else {
+          // Xt(k,j)[b][a] = -sum_q Tt(k,j)[b][q] D_k^{-1}[a][q], in place
           float acc[4] = {0.f, 0.f, 0.f, 0.f};
-          mac_nt<4>(acc, tt + cidx * kSlot + row0 * kLd, dk + lane * kLd);
+          mac_nt<4>(acc, dst + row0 * kLd, dk + lane * kLd);
+          __syncwarp();
 #pragma unroll
           for (int rr = 0; rr < 4; ++rr) dst[(row0 + rr) * kLd + lane] = -acc[rr];
         }
       }
-    }
-    group_sync(2);
-    // ---- output: Linv[i*32 + a][j*32 + b] = Xt(i,j)[b][a]; zeros above the diagonal blocks
-    for (int cidx = 0; cidx < n_cols; ++cidx) {
-      const int j = j0 + cidx;
-      const float* xcol = xt + (cidx == 0 ? 0 : (nblk - j0)) * kSlot;
-      const int ncol = min(kB, r - j * kB);
-      for (int e = tid - kGroup; e < r * kB; e += kGroup) {
-        const int row = e >> 5, b = e & 31;
-        if (b >= ncol) continue;
-        const int bi = row / kB, a = row - bi * kB;
-        const float v = (bi >= j) ? xcol[(bi - j) * kSlot + b * kLd + a] : 0.f;
-        const int64_t off = (int64_t)row * r + j * kB + b;
-        if (p.linv_f32) p.linv_f32[off] = v;
-        if (p.linv_hi) {
-          const __nv_bfloat16 hi = __float2bfloat16(v);
-          p.linv_hi[off] = hi;
-          if (p.linv_lo) p.linv_lo[off] = __float2bfloat16(v - __bfloat162float(hi));
+      group_sync(2);
+      // block row k of the result: Linv[k*32 + a][j*32 + b] = Xt(k,j)[b][a]
+      for (int cidx = 0; cidx < n_cols; ++cidx) {
+        const int j = j0 + cidx;
+        if (j > k) continue;
+        const float* src = xt + ((cidx == 0 ? 0 : (nblk - j0)) + (k - j)) * kSlot;
+        const int ncol = min(kB, r - j * kB);
+        for (int e = gt; e < kB * kB; e += kGroup) {
+          const int a = e >> 5, b = e & 31;
+          const int row = k * kB + a;
+          if (row >= r || b >= ncol) continue;
+          const float v = src[b * kLd + a];
+          const int64_t off = (int64_t)row * r + j * kB + b;
+          if (p.linv_f32) p.linv_f32[off] = v;
+          if (p.linv_hi) {
+            const __nv_bfloat16 hi = __float2bfloat16(v);
+            p.linv_hi[off] = hi;
+            if (p.linv_lo) p.linv_lo[off] = __float2bfloat16(v - __bfloat162float(hi));
+          }
+        }
+      }
+      if (k + 1 >= nblk) break;
+      if (gt == 0) bar_wait(&panel_bar[k], &s_gave_up);
+      group_sync(2);
+      // Tt(i,j)[b][a] (+)= sum_q Xt(k,j)[b][q] L(i,k)[a][q] for the rows below
+      for (int cidx = 0; cidx < n_cols; ++cidx) {
+        const int j = j0 + cidx;
+        if (j > k) continue;
+        float* xcol = xt + (cidx == 0 ? 0 : (nblk - j0)) * kSlot;   // block (i, j) at xcol + (i - j) slots
+        const float* xk = xcol + (k - j) * kSlot + row0 * kLd;
+        for (int i = k + 1; i < nblk; ++i) {
+          float acc[4] = {0.f, 0.f, 0.f, 0.f};
+          mac_nt<4>(acc, xk, slots + tri(i, k) * kSlot + lane * kLd);
+          float* dst = xcol + (i - j) * kSlot + row0 * kLd + lane;
+          if (j == k) {
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr) dst[rr * kLd] = acc[rr];
+          } else {
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr) dst[rr * kLd] += acc[rr];
+          }
         }
       }
     }
@@ -490,7 +578,7 @@ cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t str
   p.linv_hi = a.linv_hi;
   p.linv_lo = a.linv_lo;
   p.dev_status = a.dev_status;
-  const size_t smem = (size_t)(kMaxTri + kXSlots + 2) * kSlot * sizeof(float) + (size_t)(kCThreads / 32) * 4 * kB * sizeof(float);
+  const size_t smem = (size_t)(kMaxTri + kXSlots) * kSlot * sizeof(float) + (size_t)((kCThreads / 32) * 4 * kB + kB * kLcolLd) * sizeof(float);
   static bool configured[64] = {};
   int dev = 0;
   LORACT_CUDA_TRY(cudaGetDevice(&dev));
