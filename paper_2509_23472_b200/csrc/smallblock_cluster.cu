@@ -125,20 +125,23 @@ __device__ __forceinline__ void cluster_sync_all() {
 }
 
 // acc[rr] += sum_q A[rr][q] * B[lane][q], q < 32: R rows of a block against all 32 rows of another.
+// The row of B is read once into registers; every row of A feeds four independent sums.
 template <int R>
 __device__ __forceinline__ void mac_nt(float (&acc)[R], const float* __restrict__ a_rows,
                                        const float* __restrict__ b_row) {
+  float4 b[kB / 4];
 #pragma unroll
-  for (int q4 = 0; q4 < kB / 4; ++q4) {
-    const float4 b = *reinterpret_cast<const float4*>(b_row + 4 * q4);
+  for (int q4 = 0; q4 < kB / 4; ++q4) b[q4] = *reinterpret_cast<const float4*>(b_row + 4 * q4);
 #pragma unroll
-    for (int rr = 0; rr < R; ++rr) {
+  for (int rr = 0; rr < R; ++rr) {
+    float2 s01 = make_float2(0.f, 0.f), s23 = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int q4 = 0; q4 < kB / 4; ++q4) {
       const float4 a = *reinterpret_cast<const float4*>(a_rows + rr * kLd + 4 * q4);
-      acc[rr] = fmaf(a.x, b.x, acc[rr]);
-      acc[rr] = fmaf(a.y, b.y, acc[rr]);
-      acc[rr] = fmaf(a.z, b.z, acc[rr]);
-      acc[rr] = fmaf(a.w, b.w, acc[rr]);
+      s01 = __ffma2_rn(make_float2(a.x, a.y), make_float2(b[q4].x, b[q4].y), s01);
+      s23 = __ffma2_rn(make_float2(a.z, a.w), make_float2(b[q4].z, b[q4].w), s23);
     }
+    acc[rr] += (s01.x + s01.y) + (s23.x + s23.y);
   }
 }
 
@@ -168,44 +171,74 @@ __device__ __forceinline__ void send_rows4(const float (&v)[4], float* stage /* 
 // 0 above), whose words start out as kUnset -- the consumer needs no flag and no fence, it waits for
 // each word to change.  Returns true if a pivot was clamped.
 constexpr uint32_t kUnset = 0xFFFFFFFFu;   // a NaN pattern arithmetic does not produce
-constexpr int kLcolLd = kB + 1;
+constexpr int kLcolLd = kLd;              // rows of `lcol` are read back as float4
+constexpr int kInvWarps = 4;
+constexpr int kInvCols = kB / kInvWarps;  // columns of the inverse one of those warps holds
 
+// Straight-line code like this runs at the rate instructions can be fetched, so what counts on the pivot
+// chain is the number of instructions per column: a published column is read back by every lane with
+// 16-byte broadcast loads (instead of one shuffle per element) and applied with packed fp32 FMAs.
 __device__ __forceinline__ bool factor_diag_block(const float* slot, float* lcol, float pivot_floor, int lane) {
-  float a[kB];
+  float2 a2[kB / 2];   // row `lane` of the block, columns (2p, 2p + 1)
 #pragma unroll
-  for (int j = 0; j < kB; ++j) a[j] = (j < lane) ? slot[lane * kLd + j] : 0.f;
+  for (int pp = 0; pp < kB / 2; ++pp)
+    a2[pp] = make_float2(2 * pp < lane ? slot[lane * kLd + 2 * pp] : 0.f,
+                         2 * pp + 1 < lane ? slot[lane * kLd + 2 * pp + 1] : 0.f);
   float diag = slot[lane * kLd + lane];
   bool clamped = false;
+  // a pivot that is not safely positive is replaced by the floor and its column is dropped (entries
+  // below such a pivot are rounding noise; dividing them by the tiny pivot would overflow later columns)
+  float akk = __shfl_sync(0xffffffffu, diag, 0);
+  bool bad = !(akk > pivot_floor);
+  if (bad) { akk = pivot_floor; clamped = true; }
+  float rinv = rsqrtf(akk);
 #pragma unroll
   for (int k = 0; k < kB; ++k) {
-    float akk = __shfl_sync(0xffffffffu, diag, k);
-    // a pivot that is not safely positive is replaced by the floor and its column is dropped (entries
-    // below such a pivot are rounding noise; dividing them by the tiny pivot would overflow later columns)
-    const bool bad = !(akk > pivot_floor);
-    if (bad) { akk = pivot_floor; clamped = true; }
-    const float rinv = rsqrtf(akk);
-    const float lik = (lane > k && !bad) ? a[k] * rinv : 0.f;   // L[lane][k]
+    const float ak = (k & 1) ? a2[k >> 1].y : a2[k >> 1].x;
+    const float lik = (lane > k && !bad) ? ak * rinv : 0.f;   // L[lane][k]
     float pub = (lane == k) ? rinv : lik;
     if (__float_as_uint(pub) == kUnset) pub = 0.f;
     lcol[k * kLcolLd + lane] = pub;
     diag = fmaf(-lik, lik, diag);
+    __syncwarp();
+    const float2 nl = make_float2(-lik, -lik);
+    const float4* col = reinterpret_cast<const float4*>(lcol + k * kLcolLd);
+    if (k + 1 < kB) {
+      // the quad that holds column k + 1 first, then the next pivot straight away: its square root is
+      // in flight while the rest of this column's updates are issued.  (Entries of the quad at or
+      // before column k only touch columns that are no longer read.)
+      const int q1 = (k + 1) >> 2;
+      const float4 l = col[q1];
+      a2[2 * q1] = __ffma2_rn(nl, make_float2(l.x, l.y), a2[2 * q1]);
+      a2[2 * q1 + 1] = __ffma2_rn(nl, make_float2(l.z, l.w), a2[2 * q1 + 1]);
+      float an = __shfl_sync(0xffffffffu, diag, k + 1);
+      bad = !(an > pivot_floor);
+      if (bad) { an = pivot_floor; clamped = true; }
+      rinv = rsqrtf(an);
 #pragma unroll
-    for (int j = k + 1; j < kB; ++j) {
-      const float ljk = __shfl_sync(0xffffffffu, lik, j);
-      a[j] = fmaf(-lik, ljk, a[j]);
+      for (int q = q1 + 1; q < kB / 4; ++q) {
+        const float4 l2 = col[q];
+        a2[2 * q] = __ffma2_rn(nl, make_float2(l2.x, l2.y), a2[2 * q]);
+        a2[2 * q + 1] = __ffma2_rn(nl, make_float2(l2.z, l2.w), a2[2 * q + 1]);
+      }
     }
   }
   return clamped;
 }
 
-// invert_diag_block (a second warp, lane i holds row i of the inverse): takes the columns of L as they
-// appear in `lcol` and forms X = L^{-1} right-looking: once column k is known, row k of X is final up to
-// its scale 1 / L[k][k], and every later row takes its multiple of it off -- no serial dot products.
-// Writes X (lower triangular, zeros above) into `slot`.  The wait for a column is bounded.
-__device__ __forceinline__ void invert_diag_block(float* slot, const float* lcol, volatile int* gave_up, int lane) {
-  float x[kB];
+// invert_diag_block (kInvWarps more warps, lane i holds row i of the inverse, warp `part` the columns
+// j = part, part + kInvWarps, ...): takes the columns of L as they appear in `lcol` and forms X = L^{-1}
+// right-looking: once column k is known, row k of X is final up to its scale 1 / L[k][k], and every later
+// row takes its multiple of it off -- no serial dot products.  Row k travels from lane k to the others
+// through `xrow` (2 x kInvCols floats, private to the warp, double-buffered).  Writes its columns of X
+// (lower triangular, zeros above) into `slot`.  The wait for a column is bounded.
+__device__ __forceinline__ void invert_diag_block(float* slot, const float* lcol, float* xrow,
+                                                  volatile int* gave_up, int part, int lane) {
+  float2 x2[kInvCols / 2];
 #pragma unroll
-  for (int j = 0; j < kB; ++j) x[j] = (j == lane) ? 1.f : 0.f;
+  for (int pp = 0; pp < kInvCols / 2; ++pp)
+    x2[pp] = make_float2((2 * pp) * kInvWarps + part == lane ? 1.f : 0.f,
+                         (2 * pp + 1) * kInvWarps + part == lane ? 1.f : 0.f);
   float my_rinv = 1.f;
 #pragma unroll
   for (int k = 0; k < kB; ++k) {
@@ -217,14 +250,27 @@ __device__ __forceinline__ void invert_diag_block(float* slot, const float* lcol
     }
     const float v = __uint_as_float(bits);
     const float rinv = __shfl_sync(0xffffffffu, v, k);
-    if (lane == k) my_rinv = rinv;
+    float4* buf = reinterpret_cast<float4*>(xrow + (k & 1) * kInvCols);
+    if (lane == k) {
+      my_rinv = rinv;
+      buf[0] = make_float4(x2[0].x, x2[0].y, x2[1].x, x2[1].y);
+      buf[1] = make_float4(x2[2].x, x2[2].y, x2[3].x, x2[3].y);
+    }
+    __syncwarp();
     // rows below take (L[i][k] / L[k][k]) times the unscaled row k off; rows up to k are left alone
     const float m = (lane > k) ? v * rinv : 0.f;
-#pragma unroll
-    for (int j = 0; j <= k; ++j) x[j] = fmaf(-m, __shfl_sync(0xffffffffu, x[j], k), x[j]);
+    const float2 nm = make_float2(-m, -m);
+    const float4 r0 = buf[0], r1 = buf[1];
+    x2[0] = __ffma2_rn(nm, make_float2(r0.x, r0.y), x2[0]);
+    x2[1] = __ffma2_rn(nm, make_float2(r0.z, r0.w), x2[1]);
+    x2[2] = __ffma2_rn(nm, make_float2(r1.x, r1.y), x2[2]);
+    x2[3] = __ffma2_rn(nm, make_float2(r1.z, r1.w), x2[3]);
   }
 #pragma unroll
-  for (int j = 0; j < kB; ++j) slot[lane * kLd + j] = x[j] * my_rinv;
+  for (int pp = 0; pp < kInvCols / 2; ++pp) {
+    slot[lane * kLd + (2 * pp) * kInvWarps + part] = x2[pp].x * my_rinv;
+    slot[lane * kLd + (2 * pp + 1) * kInvWarps + part] = x2[pp].y * my_rinv;
+  }
   __syncwarp();
 }
 
@@ -237,6 +283,8 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
   __shared__ float s_red[kCThreads / 32];
   __shared__ float s_shift, s_floor;
   __shared__ int s_gave_up;
+  __shared__ volatile int s_chain_step;                   // CTA 0: what the sender warps may send
+  __shared__ __align__(16) float s_xrow[kInvWarps][2 * kInvCols];
   __shared__ int s_clamped;
   // blocks (i, j) owned by this CTA, in column-major order
   __shared__ unsigned char s_mine_i[kMaxTri], s_mine_j[kMaxTri];
@@ -275,6 +323,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
   } else if (tid == 32) {
     s_gave_up = 0;
     s_clamped = 0;
+    s_chain_step = 0;
     int n = 0;
     for (int bj = 0; bj < nblk; ++bj)
       for (int bi = bj; bi < nblk; ++bi)
@@ -361,60 +410,74 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
 
   if (cta == 0) {
     // =========================================================== pivot chain
-    // Phase A: warp 0 factors the diagonal block, warp 1 inverts it alongside, one thread waits for the
-    // two blocks of the next step.  Phase B: warps 0..7 form L(k+1, k); warps 8..15 send D_k^{-1} out.
-    // Phase C: warps 0..7 update the next diagonal block; warps 8..15 send L(k+1, k) out.  Sending is
-    // kept off the warps the next pivot waits for.
+    // Warps 0..7 compute.  Phase A: warp 0 factors the diagonal block, warps 1..4 invert it alongside,
+    // one thread waits for the two blocks of the next step.  Phase B: L(k+1, k).  Phase C: the next
+    // diagonal block.  Warps 8..15 only send: D_k^{-1} after phase A, L(k+1, k) after phase B.  They
+    // follow a step counter in shared memory and never hold the computing warps up.
     const int row0 = (warp & 7) * 4;
-    for (int k = 0; k < nblk; ++k) {
-      float* dslot = slots + tri(k, k) * kSlot;
-      if (warp == 0) {
-        if (factor_diag_block(dslot, lcol, s_floor, lane) && lane == 0) s_clamped = 1;
-      } else if (warp == 1) {
-        invert_diag_block(dslot, lcol, &s_gave_up, lane);
-      } else if (tid == 64 && k + 1 < nblk && k >= 1) {
-        bar_wait(&chain_bar[k + 1], &s_gave_up);   // blocks (k+1, k) and (k+1, k+1)
-      }
-      __syncthreads();
-      float* sub = slots + tri(k + 1 < nblk ? k + 1 : k, k) * kSlot;
-      if (warp < 8) {
-        if (k + 1 < nblk) {
-          // L(k+1, k) = A(k+1, k) D_k^{-T}, in place (a warp reads only the rows it writes)
+    if (warp < 8) {
+      for (int k = 0; k < nblk; ++k) {
+        float* dslot = slots + tri(k, k) * kSlot;
+        if (warp == 0) {
+          if (factor_diag_block(dslot, lcol, s_floor, lane) && lane == 0) s_clamped = 1;
+        } else if (warp <= kInvWarps) {
+          invert_diag_block(dslot, lcol, s_xrow[warp - 1], &s_gave_up, warp - 1, lane);
+        } else if (tid == (kInvWarps + 1) * 32 && k + 1 < nblk && k >= 1) {
+          bar_wait(&chain_bar[k + 1], &s_gave_up);   // blocks (k+1, k) and (k+1, k+1)
+        }
+        group_sync(1);
+        if (tid == 0) { __threadfence_block(); s_chain_step = 2 * k + 1; }
+        if (k + 1 >= nblk) break;
+        // L(k+1, k) = A(k+1, k) D_k^{-T}, in place (a warp reads only the rows it writes)
+        float* sub = slots + tri(k + 1, k) * kSlot;
+        {
           float acc[4] = {0.f, 0.f, 0.f, 0.f};
           mac_nt<4>(acc, sub + row0 * kLd, dslot + lane * kLd);
           __syncwarp();
 #pragma unroll
           for (int rr = 0; rr < 4; ++rr) sub[(row0 + rr) * kLd + lane] = acc[rr];
         }
-      } else {
-        // D_k^{-1} to every worker
-        const int rr = lane >> 3, q4 = lane & 7;
-        const float* src = dslot + (row0 + rr) * kLd + 4 * q4;
-        const float4 val = *reinterpret_cast<const float4*>(src);
-        const uint32_t a0 = smem_addr(src), b0 = smem_addr(&dinv_bar[k]);
-        for (int c = 1; c < kCl; ++c) st_async_v4(map_to_cta(a0, c), val, map_to_cta(b0, c));
-      }
-      if (k + 1 >= nblk) break;
-      __syncthreads();
-      if (warp < 8) {
-        // next diagonal block: A(k+1, k+1) -= L(k+1, k) L(k+1, k)^T
-        float acc2[4] = {0.f, 0.f, 0.f, 0.f};
-        mac_nt<4>(acc2, sub + row0 * kLd, sub + lane * kLd);
-        float* dst = slots + tri(k + 1, k + 1) * kSlot + row0 * kLd + lane;
+        group_sync(1);
+        if (tid == 0) { __threadfence_block(); s_chain_step = 2 * k + 2; }
+        {
+          // next diagonal block: A(k+1, k+1) -= L(k+1, k) L(k+1, k)^T
+          float acc2[4] = {0.f, 0.f, 0.f, 0.f};
+          mac_nt<4>(acc2, sub + row0 * kLd, sub + lane * kLd);
+          float* dst = slots + tri(k + 1, k + 1) * kSlot + row0 * kLd + lane;
 #pragma unroll
-        for (int rr = 0; rr < 4; ++rr) dst[rr * kLd] -= acc2[rr];
-        for (int e = tid; e < kB * kLcolLd; e += kGroup) reinterpret_cast<uint32_t*>(lcol)[e] = kUnset;
-      } else {
-        // L(k+1, k) to every worker
-        const int rr = lane >> 3, q4 = lane & 7;
-        const float* src = sub + (row0 + rr) * kLd + 4 * q4;
+          for (int rr = 0; rr < 4; ++rr) dst[rr * kLd] -= acc2[rr];
+          for (int e = tid; e < kB * kLcolLd; e += kGroup) reinterpret_cast<uint32_t*>(lcol)[e] = kUnset;
+        }
+        group_sync(1);
+      }
+      if (tid == 0 && s_clamped && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_PIVOT_CLAMPED);
+    } else {
+      const int rr = lane >> 3, q4 = lane & 7;
+      for (int step = 1; step <= 2 * nblk - 1; ++step) {
+        // step 2k + 1: D_k^{-1} is ready;  step 2k + 2: L(k+1, k) is ready
+        if (lane == 0) {
+          uint64_t t0 = 0;
+          for (uint32_t spin = 1; s_chain_step < step; ++spin) {
+            __nanosleep(20);
+            if ((spin & 255u) == 0u) {
+              if (*(volatile int*)&s_gave_up) break;
+              const uint64_t now = timer_ns();
+              if (t0 == 0) t0 = now;
+              else if (now - t0 > kClusterWaitNs) { s_gave_up = 1; break; }
+            }
+          }
+          __threadfence_block();
+        }
+        __syncwarp();
+        const int k = (step - 1) >> 1;
+        const bool is_dinv = (step & 1) != 0;
+        const float* blk = slots + (is_dinv ? tri(k, k) : tri(k + 1, k)) * kSlot;
+        const float* src = blk + (row0 + rr) * kLd + 4 * q4;
         const float4 val = *reinterpret_cast<const float4*>(src);
-        const uint32_t a0 = smem_addr(src), b0 = smem_addr(&panel_bar[k]);
+        const uint32_t a0 = smem_addr(src), b0 = smem_addr(is_dinv ? &dinv_bar[k] : &panel_bar[k]);
         for (int c = 1; c < kCl; ++c) st_async_v4(map_to_cta(a0, c), val, map_to_cta(b0, c));
       }
-      __syncthreads();
     }
-    if (tid == 0 && s_clamped && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_PIVOT_CLAMPED);
   } else if (warp < 8) {
     // =========================================================== workers, factorisation half
     const int row0 = warp * 4;
