@@ -26,7 +26,7 @@ namespace {
 constexpr int kB = 32;                   // block edge
 constexpr int kLd = 36;                  // padded row stride of a block slot (floats): rows 16-byte aligned
 constexpr int kSlot = kB * kLd;          // floats per slot
-constexpr int kSlotTx = kB * kB * 4;     // bytes one pushed block adds to a barrier's transaction count
+constexpr int kSlotTx = kSlot * 4;        // bytes one sent block (padding included) adds to a barrier's transaction count
 constexpr int kMaxBlk = 8;               // r <= 256
 constexpr int kCl = 8;                   // CTAs per cluster
 constexpr int kWorkers = kCl - 1;
@@ -81,6 +81,9 @@ __device__ __forceinline__ void bar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void bar_expect(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
                : "memory");
+}
+__device__ __forceinline__ void bar_arrive_local(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
 __device__ __forceinline__ bool bar_try(uint64_t* bar) {
   uint32_t ok;
@@ -145,23 +148,29 @@ __device__ __forceinline__ void mac_nt(float (&acc)[R], const float* __restrict_
   }
 }
 
-// One warp holds rows [row0, row0 + 4) of a block (v[rr]: row row0 + rr, column = lane).  Writes them
-// into `slot_local` (if keep_local) and sends them to the same slot of the CTAs first_dst .. last_dst,
-// counting the bytes on each receiver's barrier `bar_local` (same address in every CTA).
-__device__ __forceinline__ void send_rows4(const float (&v)[4], float* stage /* 4 x 32 floats, warp-private */,
-                                           float* slot_local, int row0, const uint64_t* bar_local,
-                                           int first_dst, int last_dst, bool keep_local, int lane) {
-#pragma unroll
-  for (int rr = 0; rr < 4; ++rr) stage[rr * kB + lane] = v[rr];
+// Bulk copy of `bytes` (a multiple of 16, both addresses 16-byte aligned) from this CTA's shared memory
+// into a peer's; on arrival `bytes` is taken off the transaction count of the peer's barrier `bar`.
+__device__ __forceinline__ void bulk_to_peer(uint32_t dst_cluster_addr, uint32_t src_local_addr, uint32_t bytes,
+                                             uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(dst_cluster_addr), "r"(src_local_addr), "r"(bytes), "r"(bar_cluster_addr)
+      : "memory");
+}
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+constexpr uint32_t kStripBytes = 4 * kLd * 4;   // four padded rows of a slot
+
+// One warp has just written rows [row0, row0 + 4) of the block in `slot_local` (plain stores, every lane
+// has executed fence_async_proxy).  Lanes first_dst .. last_dst (except `skip`) each copy the strip into
+// the same slot of the CTA with their number, counting its bytes on that CTA's barrier `bar_local`.
+__device__ __forceinline__ void send_strip(const float* slot_local, int row0, const uint64_t* bar_local,
+                                           int first_dst, int last_dst, int skip, int lane) {
   __syncwarp();
-  // 4 rows x 8 float4: lane -> (row = lane / 8, quad = lane % 8)
-  const int rr = lane >> 3, q4 = lane & 7;
-  const float4 val = *reinterpret_cast<const float4*>(stage + rr * kB + 4 * q4);
-  float* dst_local = slot_local + (row0 + rr) * kLd + 4 * q4;
-  if (keep_local) *reinterpret_cast<float4*>(dst_local) = val;
-  const uint32_t dst_addr = smem_addr(dst_local), bar_addr = smem_addr(bar_local);
-  for (int c = first_dst; c <= last_dst; ++c) st_async_v4(map_to_cta(dst_addr, c), val, map_to_cta(bar_addr, c));
-  __syncwarp();
+  if (lane >= first_dst && lane <= last_dst && lane != skip) {
+    const uint32_t src = smem_addr(slot_local + row0 * kLd);
+    bulk_to_peer(map_to_cta(src, lane), src, kStripBytes, map_to_cta(smem_addr(bar_local), lane));
+  }
 }
 
 // The 32 x 32 diagonal block is handled by two warps that run side by side.
@@ -271,6 +280,7 @@ __device__ __forceinline__ void invert_diag_block(float* slot, const float* lcol
     slot[lane * kLd + (2 * pp) * kInvWarps + part] = x2[pp].x * my_rinv;
     slot[lane * kLd + (2 * pp + 1) * kInvWarps + part] = x2[pp].y * my_rinv;
   }
+  fence_async_proxy();   // the block is sent on with a bulk copy
   __syncwarp();
 }
 
@@ -292,8 +302,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
 
   float* slots = reinterpret_cast<float*>(sc_smem);        // kMaxTri slots: the matrix, then L / D^{-1}
   float* xt = slots + kMaxTri * kSlot;                      // kXSlots slots: transposed inverse blocks
-  float* stage = xt + kXSlots * kSlot;                            // 16 warps x 128 floats
-  float* lcol = stage + (kCThreads / 32) * 4 * kB;          // columns of the diagonal block's factor
+  float* lcol = xt + kXSlots * kSlot;                       // columns of the diagonal block's factor
 
   uint32_t rank;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
@@ -302,20 +311,23 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
   const int r = p.r;
   const int nblk = (r + kB - 1) / kB;
   const int ntri = nblk * (nblk + 1) / 2;
-  float* my_stage = stage + warp * 4 * kB;
 
   // ---- set-up, spread over threads: barriers (with the byte counts they will receive, known up front),
   // this CTA's block list, the sentinel words of the diagonal-block column buffer
   if (tid < kMaxBlk) {
     const int k = tid;
     bar_init(&dinv_bar[k], 1);
-    bar_init(&panel_bar[k], 1);
+    bar_init(&panel_bar[k], 2);   // the byte count (below) and the CTA's own blocks of the column
     bar_init(&chain_bar[k], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     if (k < nblk) {
       if (cta != 0) {
         bar_expect(&dinv_bar[k], kSlotTx);
-        if (k + 1 < nblk) bar_expect(&panel_bar[k], (uint32_t)(nblk - 1 - k) * kSlotTx);
+        if (k + 1 < nblk) {
+          int from_peers = 1;   // L(k+1, k) comes from CTA 0
+          for (int bi = k + 2; bi < nblk; ++bi) from_peers += owner_of(bi, k, nblk) != cta ? 1 : 0;
+          bar_expect(&panel_bar[k], (uint32_t)from_peers * kSlotTx);
+        }
       } else if (k >= 2) {
         bar_expect(&chain_bar[k], 2 * kSlotTx);
       }
@@ -436,6 +448,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
           __syncwarp();
 #pragma unroll
           for (int rr = 0; rr < 4; ++rr) sub[(row0 + rr) * kLd + lane] = acc[rr];
+          fence_async_proxy();   // the block is sent on with a bulk copy
         }
         group_sync(1);
         if (tid == 0) { __threadfence_block(); s_chain_step = 2 * k + 2; }
@@ -451,8 +464,8 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
         group_sync(1);
       }
       if (tid == 0 && s_clamped && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_PIVOT_CLAMPED);
-    } else {
-      const int rr = lane >> 3, q4 = lane & 7;
+    } else if (warp == 8) {
+      // the sender: lane c copies each finished block to CTA c
       for (int step = 1; step <= 2 * nblk - 1; ++step) {
         // step 2k + 1: D_k^{-1} is ready;  step 2k + 2: L(k+1, k) is ready
         if (lane == 0) {
@@ -472,10 +485,11 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
         const int k = (step - 1) >> 1;
         const bool is_dinv = (step & 1) != 0;
         const float* blk = slots + (is_dinv ? tri(k, k) : tri(k + 1, k)) * kSlot;
-        const float* src = blk + (row0 + rr) * kLd + 4 * q4;
-        const float4 val = *reinterpret_cast<const float4*>(src);
-        const uint32_t a0 = smem_addr(src), b0 = smem_addr(is_dinv ? &dinv_bar[k] : &panel_bar[k]);
-        for (int c = 1; c < kCl; ++c) st_async_v4(map_to_cta(a0, c), val, map_to_cta(b0, c));
+        if (lane >= 1 && lane < kCl) {
+          const uint32_t src = smem_addr(blk);
+          bulk_to_peer(map_to_cta(src, lane), src, kSlotTx,
+                       map_to_cta(smem_addr(is_dinv ? &dinv_bar[k] : &panel_bar[k]), lane));
+        }
       }
     }
   } else if (warp < 8) {
@@ -494,8 +508,14 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         mac_nt<4>(acc, blk + row0 * kLd, dk + lane * kLd);
         __syncwarp();
-        send_rows4(acc, my_stage, blk, row0, &panel_bar[k], 1, kCl - 1, false, lane);
+#pragma unroll
+        for (int rr = 0; rr < 4; ++rr) blk[(row0 + rr) * kLd + lane] = acc[rr];
+        fence_async_proxy();
+        send_strip(blk, row0, &panel_bar[k], 1, kCl - 1, cta, lane);
       }
+      // this CTA's own blocks of column k are in place: the second arrival on its own barrier
+      group_sync(1);
+      if (tid == 0 && k + 1 < nblk) bar_arrive_local(&panel_bar[k]);
       if (k + 1 >= nblk) break;
       if (tid == 0) bar_wait(&panel_bar[k], &s_gave_up);
       group_sync(1);
@@ -516,12 +536,11 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
           float v[4];
 #pragma unroll
           for (int rr = 0; rr < 4; ++rr) v[rr] = blk[(row0 + rr) * kLd + lane] - acc[rr];
-          if (urgent) {
-            __syncwarp();
-            send_rows4(v, my_stage, blk, row0, &chain_bar[k + 2], 0, 0, false, lane);
-          } else {
 #pragma unroll
-            for (int rr = 0; rr < 4; ++rr) blk[(row0 + rr) * kLd + lane] = v[rr];
+          for (int rr = 0; rr < 4; ++rr) blk[(row0 + rr) * kLd + lane] = v[rr];
+          if (urgent) {
+            fence_async_proxy();
+            send_strip(blk, row0, &chain_bar[k + 2], 0, 0, -1, lane);
           }
         }
       }
@@ -641,7 +660,7 @@ cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t str
   p.linv_hi = a.linv_hi;
   p.linv_lo = a.linv_lo;
   p.dev_status = a.dev_status;
-  const size_t smem = (size_t)(kMaxTri + kXSlots) * kSlot * sizeof(float) + (size_t)((kCThreads / 32) * 4 * kB + kB * kLcolLd) * sizeof(float);
+  const size_t smem = (size_t)(kMaxTri + kXSlots) * kSlot * sizeof(float) + (size_t)(kB * kLcolLd) * sizeof(float);
   static bool configured[64] = {};
   int dev = 0;
   LORACT_CUDA_TRY(cudaGetDevice(&dev));
