@@ -276,8 +276,10 @@ cudaError_t compress_core(const loract_desc_t* desc, const void* X, int64_t ldx,
 
 struct WgradWs {
   float* partials;
-  float* T;
+  float* T;                      // fp32 path
+  __nv_bfloat16 *Th, *Tm, *Tl;   // bf16 path: T as a bf16 triple, leading dimension g rounded up to 8
   int splits;
+  int g8;
 };
 size_t carve_wgrad(void* ws, const loract_desc_t* desc, int g, WgradWs* out) {
   Carver c(ws);
@@ -287,6 +289,10 @@ size_t carve_wgrad(void* ws, const loract_desc_t* desc, int g, WgradWs* out) {
                                         : (desc->n_tokens >= 4096 ? 16 : 1);
   w.partials = (float*)c.take((size_t)w.splits * desc->rank * g * 4);
   w.T = (float*)c.take((size_t)desc->rank * g * 4);
+  w.g8 = (g + 7) / 8 * 8;
+  w.Th = (__nv_bfloat16*)c.take((size_t)desc->rank * w.g8 * 2);
+  w.Tm = (__nv_bfloat16*)c.take((size_t)desc->rank * w.g8 * 2);
+  w.Tl = (__nv_bfloat16*)c.take((size_t)desc->rank * w.g8 * 2);
   if (out) *out = w;
   return c.off;
 }
@@ -399,6 +405,17 @@ loract_status_t loract_weight_grad(const loract_desc_t* desc, const void* U, con
   uint32_t* status = (uint32_t*)ws;
   cudaError_t e = cudaMemsetAsync(status, 0, 4, st);
   if (e == cudaSuccess) e = run_gemm(t, status, st);
+  if (e == cudaSuccess && el == ELEM_BF16) {
+    // dW = V^T T on the tensor cores: T (fp32) is carried as a bf16 triple, so that the three products
+    // together are as accurate as one fp32 product
+    e = reduce_split3_launch(w.partials, w.splits, t.split_stride, r, g, g, w.g8, w.Th, w.Tm, w.Tl, st);
+    GemmDesc q;
+    q.M = (int)desc->d; q.N = g; q.K = r; q.a_mn = true; q.b_mn = true; q.lda = desc->d; q.ldb = w.g8;
+    q.n_terms = 3;
+    q.terms[0] = {V, w.Th}; q.terms[1] = {V, w.Tm}; q.terms[2] = {V, w.Tl};
+    q.out = OUT_F32; q.C0 = dW; q.ldc = g; q.accumulate = accumulate != 0;
+    if (e == cudaSuccess && gemm_tc_supported(q)) return from_cuda(gemm_tc_launch(q, status, st));
+  }
   if (e == cudaSuccess)
     e = reduce_partials_launch(w.partials, w.splits, t.split_stride, t.split_stride, w.T, nullptr, st);
   if (e == cudaSuccess) {

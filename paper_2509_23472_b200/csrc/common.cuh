@@ -110,6 +110,10 @@ cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t str
 cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_t stride,
                                    int64_t count, float* out_f32, __nv_bfloat16* out_bf16,
                                    cudaStream_t stream);
+// out = sum_s partials[s] as a bf16 triple hi + mid + lo (rows x cols, leading dimensions ld_in / ld_out).
+cudaError_t reduce_split3_launch(const float* partials, int n_partials, int64_t stride, int rows, int cols,
+                                 int64_t ld_in, int64_t ld_out, __nv_bfloat16* hi, __nv_bfloat16* mid,
+                                 __nv_bfloat16* lo, cudaStream_t stream);
 // Section 3.3 forward: A = Norm(X); per-row rstd (and mean for LayerNorm).  One warp per row.
 cudaError_t norm_forward_launch(const void* X, int64_t n, int64_t d, int64_t ldx, int elem_type,
                                 const void* gamma, const void* beta, float eps, int kind, void* A,

@@ -48,6 +48,7 @@ struct TcParams {
   int64_t split_stride;
   uint32_t b_bytes;   // bytes of one B stage
   uint32_t tmem_cols;
+  int accumulate;     // OUT_F32, one split: C += result
   uint32_t* dev_status;
 };
 
@@ -250,7 +251,9 @@ gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
         if (valid <= 0) continue;
         if (p.out == OUT_F32) {
           float* dst = (float*)p.C0 + (int64_t)split * p.split_stride + (int64_t)m * p.ldc + n;
-          if (valid == 32 && ((((uintptr_t)dst) & 15) == 0)) {
+          if (p.accumulate) {
+            for (int q = 0; q < valid; ++q) dst[q] += __uint_as_float(v[q]);
+          } else if (valid == 32 && ((((uintptr_t)dst) & 15) == 0)) {
 #pragma unroll
             for (int q = 0; q < 8; ++q)
               reinterpret_cast<uint4*>(dst)[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
@@ -392,7 +395,8 @@ bool gemm_tc_supported(const GemmDesc& g) {
   if (g.M < 1 || g.N < 1 || g.K < 1 || g.n_terms < 1 || g.n_terms > 3) return false;
   if (g.lda % 8 || g.ldb % 8) return false;
   if (g.splits > 1 && g.out != OUT_F32) return false;
-  if (g.accumulate || g.alpha != 1.0f) return false;
+  if (g.alpha != 1.0f) return false;
+  if (g.accumulate && (g.out != OUT_F32 || g.splits > 1)) return false;
   for (int t = 0; t < g.n_terms; ++t)
     if (((uintptr_t)g.terms[t].A & 15) || ((uintptr_t)g.terms[t].B & 15)) return false;
   return true;
@@ -421,6 +425,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   p.b_bytes = g.b_mn ? (uint32_t)((p.bn + 63) / 64) * 8192u : (uint32_t)p.bn * 128u;
   p.tmem_cols = 32;
   while ((int)p.tmem_cols < p.bn) p.tmem_cols *= 2;
+  p.accumulate = g.accumulate ? 1 : 0;
   p.dev_status = dev_status;
 
   TmapPack maps;

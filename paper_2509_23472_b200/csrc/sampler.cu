@@ -27,17 +27,25 @@ constexpr int kSamplerMaxRounds = 4096;  // 4M candidates; a permutation of 512 
 constexpr int kMaxRank = 512;
 
 // One CTA.  Every round draws 1024 candidates in stream order; a candidate survives if no equal value
-// was accepted before and no equal value stands earlier in the same round; survivors are appended in
-// stream order until `rank` are found.  This is exactly "the first rank distinct values of the stream".
+// stands earlier in the stream (in this round or among those accepted before); survivors are appended
+// in stream order until `rank` are found.  This is exactly "the first rank distinct values of the
+// stream".  "Stands earlier" is decided with a hash table in shared memory that keeps, for every value
+// seen, the smallest stream position it occurred at (atomicMin), so the outcome does not depend on the
+// order in which threads run.  The table holds the accepted values (at most 512) and one round of
+// candidates (at most 1024), so 2048 slots never fill.
+constexpr int kTableSlots = 2048;
+
 __global__ void __launch_bounds__(kSamplerThreads)
 sample_indices_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_t call_lo, uint32_t call_hi,
                       uint32_t n_rows, int rank, int32_t* __restrict__ idx_out,
                       uint32_t* __restrict__ dev_status) {
   __shared__ uint32_t accepted[kMaxRank];
-  __shared__ uint32_t cand[kSamplerThreads];
+  __shared__ uint32_t tab_key[kTableSlots];   // value + 1, 0 = empty
+  __shared__ uint32_t tab_pos[kTableSlots];   // smallest stream position of that value
   __shared__ int warp_alive[kSamplerThreads / 32];
   __shared__ int s_count;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int e = tid; e < kTableSlots; e += kSamplerThreads) { tab_key[e] = 0u; tab_pos[e] = 0xFFFFFFFFu; }
   if (tid == 0) s_count = 0;
   __syncthreads();
   for (int round = 0; round < kSamplerMaxRounds; ++round) {
@@ -47,11 +55,16 @@ sample_indices_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_t call_lo, uint
     uint32_t w[4];
     philox4x32_10(i >> 2, 0u, call_lo, call_hi, seed_lo, seed_hi, w);
     const uint32_t c = __umulhi(w[i & 3u], n_rows);
-    cand[tid] = c;
+    uint32_t h = (c * 2654435761u) >> 21;   // 11 bits
+    bool placed = false;
+    for (int probe = 0; probe < kTableSlots; ++probe) {
+      const uint32_t prev = atomicCAS(&tab_key[h], 0u, c + 1u);
+      if (prev == 0u || prev == c + 1u) { placed = true; break; }
+      h = (h + 1u) & (kTableSlots - 1);
+    }
+    if (placed) atomicMin(&tab_pos[h], i);
     __syncthreads();
-    bool alive = true;
-    for (int j = 0; j < count; ++j) alive = alive && (accepted[j] != c);
-    for (int j = 0; j < tid; ++j) alive = alive && (cand[j] != c);
+    const bool alive = placed && tab_pos[h] == i;
     const uint32_t ballot = __ballot_sync(0xffffffffu, alive);
     if (lane == 0) warp_alive[warp] = __popc(ballot);
     __syncthreads();

@@ -122,6 +122,28 @@ __global__ void reduce_partials_kernel(const float* __restrict__ partials, int n
   }
 }
 
+// out = sum_s partials[s] (fixed order) written as three bf16 arrays hi + mid + lo (24 mantissa bits), so
+// that a tensor-core product with it is as accurate as an fp32 one.  Rows of `cols` elements; the
+// partials and the outputs may have different leading dimensions.
+__global__ void reduce_split3_kernel(const float* __restrict__ partials, int n_partials, int64_t stride,
+                                     int rows, int cols, int64_t ld_in, int64_t ld_out,
+                                     __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ mid,
+                                     __nv_bfloat16* __restrict__ lo) {
+  const int64_t count = (int64_t)rows * cols;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t row = i / cols, col = i - row * cols;
+    float s = 0.f;
+    for (int q = 0; q < n_partials; ++q) s += partials[(int64_t)q * stride + row * ld_in + col];
+    const __nv_bfloat16 h = __float2bfloat16(s);
+    const float r1 = s - __bfloat162float(h);
+    const __nv_bfloat16 m = __float2bfloat16(r1);
+    const float r2 = r1 - __bfloat162float(m);
+    const int64_t o = row * ld_out + col;
+    hi[o] = h; mid[o] = m; lo[o] = __float2bfloat16(r2);
+  }
+}
+
 // One warp per row.  RMS: rstd = 1/sqrt(mean x^2 + eps).  LayerNorm: mean first, then the centred
 // second moment (two passes over the row, which stays in L1/L2), A = (x - mean) rstd gamma + beta.
 template <typename T>
@@ -202,6 +224,17 @@ cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_
   if (grid < 1) grid = 1;
   reduce_partials_kernel<<<grid, 256, 0, stream>>>(partials, n_partials, stride, count, out_f32,
                                                    out_bf16);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t reduce_split3_launch(const float* partials, int n_partials, int64_t stride, int rows, int cols,
+                                 int64_t ld_in, int64_t ld_out, __nv_bfloat16* hi, __nv_bfloat16* mid,
+                                 __nv_bfloat16* lo, cudaStream_t stream) {
+  int grid = (int)(((int64_t)rows * cols + 255) / 256);
+  if (grid > 148 * 8) grid = 148 * 8;
+  if (grid < 1) grid = 1;
+  reduce_split3_kernel<<<grid, 256, 0, stream>>>(partials, n_partials, stride, rows, cols, ld_in, ld_out, hi, mid, lo);
   count_launch();
   return cudaGetLastError();
 }
