@@ -18,6 +18,31 @@ void count_launch(int n = 1);
     if (_e != cudaSuccess) return _e;                  \
   } while (0)
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// The kernels of one call run back to back on one stream.  Launched with programmatic stream
+// serialisation, a kernel may start (be scheduled, set up shared memory, barriers, tensor memory) while
+// its predecessor is still running; it must then execute pdl_wait() before its first access to global
+// memory, which returns once the predecessor has completed and its writes are visible.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename Kern, typename... Args>
+cudaError_t launch_pdl(Kern kernel, dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+#endif
+
 // ---------------------------------------------------------------- generic contraction
 // C (M x N) = sum over terms of  A_t (M x K) * B_t (K x N), fp32 (or fp64) accumulation.
 // Operands are row-major arrays; a_mn / b_mn say which index is contiguous in memory:

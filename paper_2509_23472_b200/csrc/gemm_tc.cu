@@ -179,6 +179,9 @@ gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_slot;
+  // everything above overlaps the tail of the previous kernel; global memory only from here on
+  pdl_wait();
+  pdl_launch_dependents();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -382,7 +385,7 @@ cudaError_t launch_variant(const TmapPack& maps, const TcParams& p, dim3 grid, s
                                          kStages * (kABytes + 32768) + 1024));
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
-  gemm_tc_kernel<A_MN, B_MN><<<grid, kThreads, smem, stream>>>(maps, p);
+  LORACT_CUDA_TRY(launch_pdl(gemm_tc_kernel<A_MN, B_MN>, grid, dim3(kThreads), smem, stream, maps, p));
   count_launch();
   return cudaGetLastError();
 }

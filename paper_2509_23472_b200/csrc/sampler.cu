@@ -45,6 +45,7 @@ sample_indices_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_t call_lo, uint
   __shared__ int warp_alive[kSamplerThreads / 32];
   __shared__ int s_count;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_launch_dependents();
   for (int e = tid; e < kTableSlots; e += kSamplerThreads) { tab_key[e] = 0u; tab_pos[e] = 0xFFFFFFFFu; }
   if (tid == 0) s_count = 0;
   __syncthreads();
@@ -81,6 +82,7 @@ sample_indices_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_t call_lo, uint
     __syncthreads();
   }
   const int found = s_count;
+  pdl_wait();   // the index array may still be read by the previous call's kernels
   for (int j = tid; j < rank; j += kSamplerThreads) idx_out[j] = (j < found) ? (int32_t)accepted[j] : 0;
   if (tid == 0 && found < rank && dev_status) atomicOr(dev_status, LORACT_DEV_SAMPLER_SHORT);
 }
@@ -90,6 +92,8 @@ __global__ void gather_rows_kernel(const uint4* __restrict__ src, int64_t ld_vec
                                    const int32_t* __restrict__ idx, int64_t d_vec,
                                    uint4* __restrict__ dst) {
   const int row = blockIdx.y;
+  pdl_wait();
+  pdl_launch_dependents();
   const int64_t srow = idx[row];
   for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < d_vec;
        v += (int64_t)gridDim.x * blockDim.x)
@@ -132,9 +136,9 @@ __global__ void gaussian_rows_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_
 
 cudaError_t sample_indices_launch(uint64_t seed, uint64_t call_id, uint32_t n_rows, int rank,
                                   int32_t* idx_dev, uint32_t* dev_status, cudaStream_t stream) {
-  sample_indices_kernel<<<1, kSamplerThreads, 0, stream>>>(
-      (uint32_t)seed, (uint32_t)(seed >> 32), (uint32_t)call_id, (uint32_t)(call_id >> 32), n_rows,
-      rank, idx_dev, dev_status);
+  LORACT_CUDA_TRY(launch_pdl(sample_indices_kernel, dim3(1), dim3(kSamplerThreads), 0, stream, (uint32_t)seed,
+                             (uint32_t)(seed >> 32), (uint32_t)call_id, (uint32_t)(call_id >> 32), n_rows, rank,
+                             idx_dev, dev_status));
   count_launch();
   return cudaGetLastError();
 }
@@ -146,8 +150,8 @@ cudaError_t gather_rows_launch(const void* src, int64_t ld, const int32_t* idx, 
   const int threads = 256;
   int gx = (int)((d_vec + threads - 1) / threads);
   if (gx > 64) gx = 64;
-  gather_rows_kernel<<<dim3(gx, rank), threads, 0, stream>>>((const uint4*)src, ld_vec, idx, d_vec,
-                                                             (uint4*)dst);
+  LORACT_CUDA_TRY(launch_pdl(gather_rows_kernel, dim3(gx, rank), dim3(threads), 0, stream, (const uint4*)src, ld_vec,
+                             idx, d_vec, (uint4*)dst));
   count_launch();
   return cudaGetLastError();
 }

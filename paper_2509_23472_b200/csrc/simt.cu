@@ -113,6 +113,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(SimtParams p) {
 __global__ void reduce_partials_kernel(const float* __restrict__ partials, int n_partials,
                                        int64_t stride, int64_t count, float* __restrict__ out_f32,
                                        __nv_bfloat16* __restrict__ out_bf16) {
+  pdl_wait();
+  pdl_launch_dependents();
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count;
        i += (int64_t)gridDim.x * blockDim.x) {
     float s = 0.f;
@@ -130,6 +132,8 @@ __global__ void reduce_split3_kernel(const float* __restrict__ partials, int n_p
                                      __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ mid,
                                      __nv_bfloat16* __restrict__ lo) {
   const int64_t count = (int64_t)rows * cols;
+  pdl_wait();
+  pdl_launch_dependents();
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count;
        i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t row = i / cols, col = i - row * cols;
@@ -222,8 +226,8 @@ cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_
   int grid = (int)((count + 255) / 256);
   if (grid > 148 * 16) grid = 148 * 16;
   if (grid < 1) grid = 1;
-  reduce_partials_kernel<<<grid, 256, 0, stream>>>(partials, n_partials, stride, count, out_f32,
-                                                   out_bf16);
+  LORACT_CUDA_TRY(launch_pdl(reduce_partials_kernel, dim3(grid), dim3(256), 0, stream, partials, n_partials, stride,
+                             count, out_f32, out_bf16));
   count_launch();
   return cudaGetLastError();
 }
@@ -234,7 +238,8 @@ cudaError_t reduce_split3_launch(const float* partials, int n_partials, int64_t 
   int grid = (int)(((int64_t)rows * cols + 255) / 256);
   if (grid > 148 * 8) grid = 148 * 8;
   if (grid < 1) grid = 1;
-  reduce_split3_kernel<<<grid, 256, 0, stream>>>(partials, n_partials, stride, rows, cols, ld_in, ld_out, hi, mid, lo);
+  LORACT_CUDA_TRY(launch_pdl(reduce_split3_kernel, dim3(grid), dim3(256), 0, stream, partials, n_partials, stride, rows,
+                             cols, ld_in, ld_out, hi, mid, lo));
   count_launch();
   return cudaGetLastError();
 }

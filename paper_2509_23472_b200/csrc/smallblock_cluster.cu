@@ -343,6 +343,9 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
     s_n_mine = n;
   }
   for (int e = tid; e < kB * kLcolLd; e += kCThreads) reinterpret_cast<uint32_t*>(lcol)[e] = kUnset;
+  // everything above overlaps the tail of the previous kernel; global memory only from here on
+  pdl_wait();
+  pdl_launch_dependents();
 
   // ---- load.  Block t is summed over the partials by CTA t mod 8 and written into the slot of the CTA
   // that works on it first (CTA 0 for block rows 0 and 1, the owner otherwise).  All global loads of a
@@ -674,13 +677,15 @@ cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t str
   cfg.blockDim = dim3(kCThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = kCl;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   LORACT_CUDA_TRY(cudaLaunchKernelEx(&cfg, small_block_cluster_kernel, p));
   count_launch();
   return cudaGetLastError();
