@@ -122,30 +122,59 @@ __device__ __forceinline__ bool bar_wait(uint64_t* bar, volatile int* gave_up) {
 __device__ __forceinline__ void group_sync(int id) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(kGroup) : "memory");
 }
+__device__ __forceinline__ void chain_sync() { asm volatile("bar.sync 3, 352;" ::: "memory"); }   // warps 0..10 of CTA 0
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-// acc[rr] += sum_q A[rr][q] * B[lane][q], q < 32: R rows of a block against all 32 rows of another.
-// The row of B is read once into registers; every row of A feeds four independent sums.
-template <int R>
-__device__ __forceinline__ void mac_nt(float (&acc)[R], const float* __restrict__ a_rows,
-                                       const float* __restrict__ b_row) {
-  float4 b[kB / 4];
+// 32 x 32 block product C += A B^T on (32 / TM) * (32 / TN) threads, thread t of them holding the TM x TN
+// outputs C[TM tm + i][tn + NT j], NT = 32 / TN, tm = t / NT, tn = t % NT.  Both operands are read along
+// the contraction index with 16-byte loads: TM + TN loads feed 4 TM TN FMAs, which is what keeps the
+// shared-memory pipe (the limit of these products) below the FMA pipe.  The eight lanes of a quarter
+// warp read one row of A (a broadcast) and eight different rows of B, whose stride of 36 words spreads
+// them over all banks.
+template <int TM, int TN>
+__device__ __forceinline__ void tile_mac(float (&acc)[TM][TN], const float* __restrict__ A,
+                                         const float* __restrict__ Bm, int tm, int tn) {
+  constexpr int NT = kB / TN;
 #pragma unroll
-  for (int q4 = 0; q4 < kB / 4; ++q4) b[q4] = *reinterpret_cast<const float4*>(b_row + 4 * q4);
+  for (int q4 = 0; q4 < kB / 4; ++q4) {
+    float4 a[TM], b[TN];
 #pragma unroll
-  for (int rr = 0; rr < R; ++rr) {
-    float2 s01 = make_float2(0.f, 0.f), s23 = make_float2(0.f, 0.f);
+    for (int i = 0; i < TM; ++i) a[i] = *reinterpret_cast<const float4*>(A + (TM * tm + i) * kLd + 4 * q4);
 #pragma unroll
-    for (int q4 = 0; q4 < kB / 4; ++q4) {
-      const float4 a = *reinterpret_cast<const float4*>(a_rows + rr * kLd + 4 * q4);
-      s01 = __ffma2_rn(make_float2(a.x, a.y), make_float2(b[q4].x, b[q4].y), s01);
-      s23 = __ffma2_rn(make_float2(a.z, a.w), make_float2(b[q4].z, b[q4].w), s23);
-    }
-    acc[rr] += (s01.x + s01.y) + (s23.x + s23.y);
+    for (int j = 0; j < TN; ++j) b[j] = *reinterpret_cast<const float4*>(Bm + (tn + NT * j) * kLd + 4 * q4);
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+      for (int j = 0; j < TN; ++j) {
+        acc[i][j] = fmaf(a[i].x, b[j].x, acc[i][j]);
+        acc[i][j] = fmaf(a[i].y, b[j].y, acc[i][j]);
+        acc[i][j] = fmaf(a[i].z, b[j].z, acc[i][j]);
+        acc[i][j] = fmaf(a[i].w, b[j].w, acc[i][j]);
+      }
   }
+}
+template <int TM, int TN>
+__device__ __forceinline__ void tile_zero(float (&acc)[TM][TN]) {
+#pragma unroll
+  for (int i = 0; i < TM; ++i)
+#pragma unroll
+    for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
+}
+// dst[TM tm + i][tn + NT j] = alpha * acc[i][j] + beta * dst[...]
+template <int TM, int TN>
+__device__ __forceinline__ void tile_store(float* dst, const float (&acc)[TM][TN], int tm, int tn, float alpha,
+                                           bool add) {
+  constexpr int NT = kB / TN;
+#pragma unroll
+  for (int i = 0; i < TM; ++i)
+#pragma unroll
+    for (int j = 0; j < TN; ++j) {
+      float* d = dst + (TM * tm + i) * kLd + tn + NT * j;
+      *d = add ? fmaf(alpha, acc[i][j], *d) : alpha * acc[i][j];
+    }
 }
 
 // Bulk copy of `bytes` (a multiple of 16, both addresses 16-byte aligned) from this CTA's shared memory
@@ -159,127 +188,177 @@ __device__ __forceinline__ void bulk_to_peer(uint32_t dst_cluster_addr, uint32_t
 }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-constexpr uint32_t kStripBytes = 4 * kLd * 4;   // four padded rows of a slot
-
-// One warp has just written rows [row0, row0 + 4) of the block in `slot_local` (plain stores, every lane
-// has executed fence_async_proxy).  Lanes first_dst .. last_dst (except `skip`) each copy the strip into
-// the same slot of the CTA with their number, counting its bytes on that CTA's barrier `bar_local`.
-__device__ __forceinline__ void send_strip(const float* slot_local, int row0, const uint64_t* bar_local,
-                                           int first_dst, int last_dst, int skip, int lane) {
+// One warp has just written rows [row0, row0 + n_rows) of the block in `slot_local` (plain stores, every
+// lane has executed fence_async_proxy).  Lanes first_dst .. last_dst (except `skip`) each copy those rows
+// into the same slot of the CTA with their number, counting the bytes on that CTA's barrier `bar_local`.
+__device__ __forceinline__ void send_rows(const float* slot_local, int row0, int n_rows, const uint64_t* bar_local,
+                                          int first_dst, int last_dst, int skip, int lane) {
   __syncwarp();
   if (lane >= first_dst && lane <= last_dst && lane != skip) {
     const uint32_t src = smem_addr(slot_local + row0 * kLd);
-    bulk_to_peer(map_to_cta(src, lane), src, kStripBytes, map_to_cta(smem_addr(bar_local), lane));
+    bulk_to_peer(map_to_cta(src, lane), src, (uint32_t)(n_rows * kLd * 4),
+                 map_to_cta(smem_addr(bar_local), lane));
   }
 }
 
-// The 32 x 32 diagonal block is handled by two warps that run side by side.
+// The 32 x 32 diagonal block is handled by ten warps that run side by side: two factor it (one the
+// columns 0..15, one the columns 16..31), eight invert the factor, four columns each.  Straight-line
+// code like this runs at the rate instructions can be fetched, so the work per column is spread thin;
+// what remains per column is the latency of the pivot (broadcast, reciprocal square root, one FMA).
 //
-// factor_diag_block (one warp, lane i holds row i): right-looking Cholesky in registers.  As soon as
-// column k of L is known it is published to `lcol` (lcol[k][i] = L[i][k] for i > k, 1 / L[k][k] for i = k,
-// 0 above), whose words start out as kUnset -- the consumer needs no flag and no fence, it waits for
-// each word to change.  Returns true if a pivot was clamped.
+// As soon as column k of L is known it is published twice, both arrays starting out as kUnset so that a
+// consumer needs no flag and no fence -- it waits for its word to change:
+//   lcol[k][i] = L[i][k] (i > k), 1 / L[k][k] (i = k), 0 (i < k)             for the other factor warp
+//   mcol[k][i] = L[i][k] / L[k][k] (i > k), 1 / L[k][k] (i = k), 0 (i < k)   for the inverting warps
 constexpr uint32_t kUnset = 0xFFFFFFFFu;   // a NaN pattern arithmetic does not produce
 constexpr int kLcolLd = kLd;              // rows of `lcol` are read back as float4
-constexpr int kInvWarps = 4;
+constexpr int kHalf = kB / 2;
+constexpr int kInvWarps = 8;
 constexpr int kInvCols = kB / kInvWarps;  // columns of the inverse one of those warps holds
 
-// Straight-line code like this runs at the rate instructions can be fetched, so what counts on the pivot
-// chain is the number of instructions per column: a published column is read back by every lane with
-// 16-byte broadcast loads (instead of one shuffle per element) and applied with packed fp32 FMAs.
-__device__ __forceinline__ bool factor_diag_block(const float* slot, float* lcol, float pivot_floor, int lane) {
-  float2 a2[kB / 2];   // row `lane` of the block, columns (2p, 2p + 1)
-#pragma unroll
-  for (int pp = 0; pp < kB / 2; ++pp)
-    a2[pp] = make_float2(2 * pp < lane ? slot[lane * kLd + 2 * pp] : 0.f,
-                         2 * pp + 1 < lane ? slot[lane * kLd + 2 * pp + 1] : 0.f);
-  float diag = slot[lane * kLd + lane];
-  bool clamped = false;
-  // a pivot that is not safely positive is replaced by the floor and its column is dropped (entries
-  // below such a pivot are rounding noise; dividing them by the tiny pivot would overflow later columns)
-  float akk = __shfl_sync(0xffffffffu, diag, 0);
-  bool bad = !(akk > pivot_floor);
-  if (bad) { akk = pivot_floor; clamped = true; }
-  float rinv = rsqrtf(akk);
-#pragma unroll
-  for (int k = 0; k < kB; ++k) {
-    const float ak = (k & 1) ? a2[k >> 1].y : a2[k >> 1].x;
-    const float lik = (lane > k && !bad) ? ak * rinv : 0.f;   // L[lane][k]
-    float pub = (lane == k) ? rinv : lik;
-    if (__float_as_uint(pub) == kUnset) pub = 0.f;
-    lcol[k * kLcolLd + lane] = pub;
-    diag = fmaf(-lik, lik, diag);
+// One MUFU instruction (2 ulp); the argument is a clamped, positive, normal pivot.
+__device__ __forceinline__ float fast_rsqrt(float x) {
+  float y;
+  asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float not_unset(float v) { return __float_as_uint(v) == kUnset ? 0.f : v; }
+
+// Bounded wait for one word of lcol / mcol.
+__device__ __forceinline__ float wait_word(const float* addr, volatile int* gave_up) {
+  const volatile uint32_t* src = reinterpret_cast<const volatile uint32_t*>(addr);
+  uint32_t bits = *src;
+  for (uint32_t spin = 0; bits == kUnset; ++spin) {
+    if (spin > (1u << 20) || *gave_up) { *gave_up = 1; bits = 0u; break; }
+    __nanosleep(32);   // a warp that spins would take issue slots from the factoring warp next to it
+    bits = *src;
+  }
+  return __uint_as_float(bits);
+}
+
+// One pivot column of the right-looking Cholesky inside a warp that holds the columns [c0, c0 + 16) of
+// every row (lane = row) as float2 pairs `a2`: takes the pivot's reciprocal square root `rinv`, forms and
+// publishes the column, updates the later columns of this warp with 16-byte broadcast loads and packed
+// FMAs, and starts the next pivot early.  K is the column inside the warp's range (compile time).
+template <int K>
+__device__ __forceinline__ void pivot_column(float2 (&a2)[kHalf / 2], float& diag, float& rinv, bool& bad,
+                                             bool& clamped, int c0, float* lcol, float* mcol, float pivot_floor,
+                                             int lane) {
+  const int k = c0 + K;
+  const float ak = (K & 1) ? a2[K >> 1].y : a2[K >> 1].x;
+  // a pivot that is not safely positive was replaced by the floor; its column is dropped (entries below
+  // such a pivot are rounding noise; dividing them by the tiny pivot would overflow later columns)
+  const float lik = (lane > k && !bad) ? ak * rinv : 0.f;   // L[lane][k]
+  lcol[k * kLcolLd + lane] = not_unset((lane == k) ? rinv : lik);
+  mcol[k * kLcolLd + lane] = not_unset((lane == k) ? rinv : lik * rinv);
+  diag = fmaf(-lik, lik, diag);
+  if (K + 1 < kHalf) {
+    // the next column first, through a shuffle (shorter than the round trip through shared memory), and
+    // the next pivot straight away: its square root is in flight while the rest of this column's
+    // updates are issued
+    const float l1 = __shfl_sync(0xffffffffu, lik, k + 1);
+    if ((K + 1) & 1) a2[(K + 1) >> 1].y = fmaf(-lik, l1, a2[(K + 1) >> 1].y);
+    else a2[(K + 1) >> 1].x = fmaf(-lik, l1, a2[(K + 1) >> 1].x);
+    float an = __shfl_sync(0xffffffffu, diag, k + 1);
+    bad = !(an > pivot_floor);
+    if (bad) { an = pivot_floor; clamped = true; }
+    rinv = fast_rsqrt(an);
     __syncwarp();
     const float2 nl = make_float2(-lik, -lik);
-    const float4* col = reinterpret_cast<const float4*>(lcol + k * kLcolLd);
-    if (k + 1 < kB) {
-      // the quad that holds column k + 1 first, then the next pivot straight away: its square root is
-      // in flight while the rest of this column's updates are issued.  (Entries of the quad at or
-      // before column k only touch columns that are no longer read.)
-      const int q1 = (k + 1) >> 2;
-      const float4 l = col[q1];
-      a2[2 * q1] = __ffma2_rn(nl, make_float2(l.x, l.y), a2[2 * q1]);
-      a2[2 * q1 + 1] = __ffma2_rn(nl, make_float2(l.z, l.w), a2[2 * q1 + 1]);
-      float an = __shfl_sync(0xffffffffu, diag, k + 1);
-      bad = !(an > pivot_floor);
-      if (bad) { an = pivot_floor; clamped = true; }
-      rinv = rsqrtf(an);
+    const float4* col = reinterpret_cast<const float4*>(lcol + k * kLcolLd + c0);
+    // columns K + 2 ..: 16-byte broadcast loads of the published column, packed FMAs.  In the quad that
+    // holds column K + 1 the entries up to it are masked out (K + 1 is done, earlier ones are not read).
+    constexpr int q1 = (K + 2) >> 2;
 #pragma unroll
-      for (int q = q1 + 1; q < kB / 4; ++q) {
-        const float4 l2 = col[q];
-        a2[2 * q] = __ffma2_rn(nl, make_float2(l2.x, l2.y), a2[2 * q]);
-        a2[2 * q + 1] = __ffma2_rn(nl, make_float2(l2.z, l2.w), a2[2 * q + 1]);
+    for (int q = q1; q < kHalf / 4; ++q) {
+      float4 l2 = col[q];
+      if (4 * q + 0 < K + 2) l2.x = 0.f;
+      if (4 * q + 1 < K + 2) l2.y = 0.f;
+      if (4 * q + 2 < K + 2) l2.z = 0.f;
+      if (4 * q + 3 < K + 2) l2.w = 0.f;
+      a2[2 * q] = __ffma2_rn(nl, make_float2(l2.x, l2.y), a2[2 * q]);
+      a2[2 * q + 1] = __ffma2_rn(nl, make_float2(l2.z, l2.w), a2[2 * q + 1]);
+    }
+  }
+}
+
+template <int K>
+__device__ __forceinline__ void pivot_columns_from(float2 (&a2)[kHalf / 2], float& diag, float& rinv, bool& bad,
+                                                   bool& clamped, int c0, float* lcol, float* mcol,
+                                                   float pivot_floor, int lane) {
+  if constexpr (K < kHalf) {
+    pivot_column<K>(a2, diag, rinv, bad, clamped, c0, lcol, mcol, pivot_floor, lane);
+    pivot_columns_from<K + 1>(a2, diag, rinv, bad, clamped, c0, lcol, mcol, pivot_floor, lane);
+  }
+}
+
+// Factor warp `half` (0: columns 0..15, 1: columns 16..31) of the diagonal block in `slot`.  The second
+// warp first follows the columns the first one publishes, taking them off its own columns, then carries
+// on with the pivots 16..31.  Returns true if a pivot was clamped.
+__device__ __forceinline__ bool factor_diag_half(const float* slot, float* lcol, float* mcol, float pivot_floor,
+                                                 volatile int* gave_up, int half, int lane) {
+  const int c0 = half * kHalf;
+  float2 a2[kHalf / 2];   // row `lane`, columns (c0 + 2p, c0 + 2p + 1), below the diagonal only
+#pragma unroll
+  for (int pp = 0; pp < kHalf / 2; ++pp)
+    a2[pp] = make_float2(c0 + 2 * pp < lane ? slot[lane * kLd + c0 + 2 * pp] : 0.f,
+                         c0 + 2 * pp + 1 < lane ? slot[lane * kLd + c0 + 2 * pp + 1] : 0.f);
+  float diag = slot[lane * kLd + lane];   // used by the lanes whose diagonal lies in this warp's columns
+  if (half == 1) {
+#pragma unroll
+    for (int k = 0; k < kHalf; ++k) {
+      const float v = wait_word(lcol + k * kLcolLd + lane, gave_up);
+      const float lik = (lane >= kHalf) ? v : 0.f;   // L[lane][k]
+      __syncwarp();
+      const float2 nl = make_float2(-lik, -lik);
+      const float4* col = reinterpret_cast<const float4*>(lcol + k * kLcolLd + kHalf);
+      diag = fmaf(-lik, lik, diag);
+#pragma unroll
+      for (int q = 0; q < kHalf / 4; ++q) {
+        const float4 l = col[q];
+        a2[2 * q] = __ffma2_rn(nl, make_float2(l.x, l.y), a2[2 * q]);
+        a2[2 * q + 1] = __ffma2_rn(nl, make_float2(l.z, l.w), a2[2 * q + 1]);
       }
     }
   }
+  bool clamped = false;
+  float akk = __shfl_sync(0xffffffffu, diag, c0);
+  bool bad = !(akk > pivot_floor);
+  if (bad) { akk = pivot_floor; clamped = true; }
+  float rinv = fast_rsqrt(akk);
+  pivot_columns_from<0>(a2, diag, rinv, bad, clamped, c0, lcol, mcol, pivot_floor, lane);
   return clamped;
 }
 
-// invert_diag_block (kInvWarps more warps, lane i holds row i of the inverse, warp `part` the columns
-// j = part, part + kInvWarps, ...): takes the columns of L as they appear in `lcol` and forms X = L^{-1}
-// right-looking: once column k is known, row k of X is final up to its scale 1 / L[k][k], and every later
-// row takes its multiple of it off -- no serial dot products.  Row k travels from lane k to the others
-// through `xrow` (2 x kInvCols floats, private to the warp, double-buffered).  Writes its columns of X
-// (lower triangular, zeros above) into `slot`.  The wait for a column is bounded.
-__device__ __forceinline__ void invert_diag_block(float* slot, const float* lcol, float* xrow,
-                                                  volatile int* gave_up, int part, int lane) {
-  float2 x2[kInvCols / 2];
-#pragma unroll
-  for (int pp = 0; pp < kInvCols / 2; ++pp)
-    x2[pp] = make_float2((2 * pp) * kInvWarps + part == lane ? 1.f : 0.f,
-                         (2 * pp + 1) * kInvWarps + part == lane ? 1.f : 0.f);
+// Inverting warp `part` (lane i holds row i of X = L^{-1}, columns 4 part .. 4 part + 3): takes the scaled
+// columns of L as they appear in `mcol` and works right-looking: once column k is known, row k of X is
+// final up to its scale 1 / L[k][k], and every later row takes L[i][k] / L[k][k] times the unscaled row k
+// (four shuffles from lane k) off -- no serial dot products.  Columns k < 4 part cannot touch this warp's
+// columns and are skipped.  Writes its columns of X (lower triangular, zeros above) into `slot`.
+__device__ __forceinline__ void invert_diag_part(float* slot, const float* mcol, volatile int* gave_up, int part,
+                                                 int lane) {
+  const int j0 = part * kInvCols;
+  float2 x01 = make_float2(j0 == lane ? 1.f : 0.f, j0 + 1 == lane ? 1.f : 0.f);
+  float2 x23 = make_float2(j0 + 2 == lane ? 1.f : 0.f, j0 + 3 == lane ? 1.f : 0.f);
   float my_rinv = 1.f;
-#pragma unroll
-  for (int k = 0; k < kB; ++k) {
-    const volatile uint32_t* src = reinterpret_cast<const volatile uint32_t*>(lcol + k * kLcolLd + lane);
-    uint32_t bits = *src;
-    for (uint32_t spin = 0; bits == kUnset; ++spin) {
-      if (spin > (1u << 22) || *gave_up) { *gave_up = 1; bits = 0u; break; }
-      bits = *src;
-    }
-    const float v = __uint_as_float(bits);
-    const float rinv = __shfl_sync(0xffffffffu, v, k);
-    float4* buf = reinterpret_cast<float4*>(xrow + (k & 1) * kInvCols);
-    if (lane == k) {
-      my_rinv = rinv;
-      buf[0] = make_float4(x2[0].x, x2[0].y, x2[1].x, x2[1].y);
-      buf[1] = make_float4(x2[2].x, x2[2].y, x2[3].x, x2[3].y);
-    }
-    __syncwarp();
-    // rows below take (L[i][k] / L[k][k]) times the unscaled row k off; rows up to k are left alone
-    const float m = (lane > k) ? v * rinv : 0.f;
+  // a real loop on purpose: straight-line code runs at the rate instructions can be fetched (several
+  // cycles each), a loop this small is served from the innermost instruction cache
+  // The word of the next column is read ahead (it may still be unset; then it is waited for at the top).
+  uint32_t ahead = *reinterpret_cast<const volatile uint32_t*>(mcol + j0 * kLcolLd + lane);
+#pragma unroll 1
+  for (int k = j0; k < kB; ++k) {
+    const float w = (ahead != kUnset) ? __uint_as_float(ahead) : wait_word(mcol + k * kLcolLd + lane, gave_up);
+    ahead = *reinterpret_cast<const volatile uint32_t*>(mcol + (k + 1 < kB ? k + 1 : k) * kLcolLd + lane);
+    my_rinv = (lane == k) ? w : my_rinv;
+    const float m = (lane > k) ? w : 0.f;
     const float2 nm = make_float2(-m, -m);
-    const float4 r0 = buf[0], r1 = buf[1];
-    x2[0] = __ffma2_rn(nm, make_float2(r0.x, r0.y), x2[0]);
-    x2[1] = __ffma2_rn(nm, make_float2(r0.z, r0.w), x2[1]);
-    x2[2] = __ffma2_rn(nm, make_float2(r1.x, r1.y), x2[2]);
-    x2[3] = __ffma2_rn(nm, make_float2(r1.z, r1.w), x2[3]);
+    const float2 r01 = make_float2(__shfl_sync(0xffffffffu, x01.x, k), __shfl_sync(0xffffffffu, x01.y, k));
+    const float2 r23 = make_float2(__shfl_sync(0xffffffffu, x23.x, k), __shfl_sync(0xffffffffu, x23.y, k));
+    x01 = __ffma2_rn(nm, r01, x01);
+    x23 = __ffma2_rn(nm, r23, x23);
   }
-#pragma unroll
-  for (int pp = 0; pp < kInvCols / 2; ++pp) {
-    slot[lane * kLd + (2 * pp) * kInvWarps + part] = x2[pp].x * my_rinv;
-    slot[lane * kLd + (2 * pp + 1) * kInvWarps + part] = x2[pp].y * my_rinv;
-  }
+  *reinterpret_cast<float4*>(slot + lane * kLd + j0) =
+      make_float4(x01.x * my_rinv, x01.y * my_rinv, x23.x * my_rinv, x23.y * my_rinv);
   fence_async_proxy();   // the block is sent on with a bulk copy
   __syncwarp();
 }
@@ -293,8 +372,8 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
   __shared__ float s_red[kCThreads / 32];
   __shared__ float s_shift, s_floor;
   __shared__ int s_gave_up;
+  __shared__ volatile int s_urgent;                       // workers: the factorisation half is on the chain's critical path
   __shared__ volatile int s_chain_step;                   // CTA 0: what the sender warps may send
-  __shared__ __align__(16) float s_xrow[kInvWarps][2 * kInvCols];
   __shared__ int s_clamped;
   // blocks (i, j) owned by this CTA, in column-major order
   __shared__ unsigned char s_mine_i[kMaxTri], s_mine_j[kMaxTri];
@@ -303,6 +382,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
   float* slots = reinterpret_cast<float*>(sc_smem);        // kMaxTri slots: the matrix, then L / D^{-1}
   float* xt = slots + kMaxTri * kSlot;                      // kXSlots slots: transposed inverse blocks
   float* lcol = xt + kXSlots * kSlot;                       // columns of the diagonal block's factor
+  float* mcol = lcol + kB * kLcolLd;                        // the same, scaled by the pivot
 
   uint32_t rank;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
@@ -336,13 +416,14 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
     s_gave_up = 0;
     s_clamped = 0;
     s_chain_step = 0;
+    s_urgent = 0;
     int n = 0;
     for (int bj = 0; bj < nblk; ++bj)
       for (int bi = bj; bi < nblk; ++bi)
         if (owner_of(bi, bj, nblk) == cta) { s_mine_i[n] = (unsigned char)bi; s_mine_j[n] = (unsigned char)bj; ++n; }
     s_n_mine = n;
   }
-  for (int e = tid; e < kB * kLcolLd; e += kCThreads) reinterpret_cast<uint32_t*>(lcol)[e] = kUnset;
+  for (int e = tid; e < 2 * kB * kLcolLd; e += kCThreads) reinterpret_cast<uint32_t*>(lcol)[e] = kUnset;
   // everything above overlaps the tail of the previous kernel; global memory only from here on
   pdl_wait();
   pdl_launch_dependents();
@@ -425,49 +506,50 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
 
   if (cta == 0) {
     // =========================================================== pivot chain
-    // Warps 0..7 compute.  Phase A: warp 0 factors the diagonal block, warps 1..4 invert it alongside,
-    // one thread waits for the two blocks of the next step.  Phase B: L(k+1, k).  Phase C: the next
-    // diagonal block.  Warps 8..15 only send: D_k^{-1} after phase A, L(k+1, k) after phase B.  They
-    // follow a step counter in shared memory and never hold the computing warps up.
-    const int row0 = (warp & 7) * 4;
-    if (warp < 8) {
+    // Phase A: warps 0, 1 factor the diagonal block, warps 2..9 invert it alongside, a thread of warp 10
+    // waits for the two blocks of the next step.  Phase B (warps 0..7): L(k+1, k).  Phase C (warps 0..7):
+    // the next diagonal block.  Warp 11 only sends: D_k^{-1} after phase A, L(k+1, k) after phase B; it
+    // follows a step counter in shared memory and never holds the others up.
+    constexpr int kChainWarps = 11;   // warps that take part in the phase barriers
+    if (warp < kChainWarps) {
       for (int k = 0; k < nblk; ++k) {
         float* dslot = slots + tri(k, k) * kSlot;
-        if (warp == 0) {
-          if (factor_diag_block(dslot, lcol, s_floor, lane) && lane == 0) s_clamped = 1;
-        } else if (warp <= kInvWarps) {
-          invert_diag_block(dslot, lcol, s_xrow[warp - 1], &s_gave_up, warp - 1, lane);
-        } else if (tid == (kInvWarps + 1) * 32 && k + 1 < nblk && k >= 1) {
+        if (warp < 2) {
+          if (factor_diag_half(dslot, lcol, mcol, s_floor, &s_gave_up, warp, lane) && lane == 0) s_clamped = 1;
+        } else if (warp < 2 + kInvWarps) {
+          invert_diag_part(dslot, mcol, &s_gave_up, warp - 2, lane);
+        } else if (lane == 0 && k + 1 < nblk && k >= 1) {
           bar_wait(&chain_bar[k + 1], &s_gave_up);   // blocks (k+1, k) and (k+1, k+1)
         }
-        group_sync(1);
+        chain_sync();
         if (tid == 0) { __threadfence_block(); s_chain_step = 2 * k + 1; }
         if (k + 1 >= nblk) break;
         // L(k+1, k) = A(k+1, k) D_k^{-T}, in place (a warp reads only the rows it writes)
         float* sub = slots + tri(k + 1, k) * kSlot;
-        {
-          float acc[4] = {0.f, 0.f, 0.f, 0.f};
-          mac_nt<4>(acc, sub + row0 * kLd, dslot + lane * kLd);
-          __syncwarp();
-#pragma unroll
-          for (int rr = 0; rr < 4; ++rr) sub[(row0 + rr) * kLd + lane] = acc[rr];
+        if (warp < 8) {
+          float acc[2][2];
+          tile_zero(acc);
+          tile_mac<2, 2>(acc, sub, dslot, tid >> 4, tid & 15);
+          group_sync(1);   // in place: everyone has read the block
+          tile_store<2, 2>(sub, acc, tid >> 4, tid & 15, 1.f, false);
           fence_async_proxy();   // the block is sent on with a bulk copy
         }
-        group_sync(1);
+        chain_sync();
         if (tid == 0) { __threadfence_block(); s_chain_step = 2 * k + 2; }
-        {
+        if (warp < 8) {
           // next diagonal block: A(k+1, k+1) -= L(k+1, k) L(k+1, k)^T
-          float acc2[4] = {0.f, 0.f, 0.f, 0.f};
-          mac_nt<4>(acc2, sub + row0 * kLd, sub + lane * kLd);
-          float* dst = slots + tri(k + 1, k + 1) * kSlot + row0 * kLd + lane;
-#pragma unroll
-          for (int rr = 0; rr < 4; ++rr) dst[rr * kLd] -= acc2[rr];
-          for (int e = tid; e < kB * kLcolLd; e += kGroup) reinterpret_cast<uint32_t*>(lcol)[e] = kUnset;
+          float acc2[2][2];
+          tile_zero(acc2);
+          tile_mac<2, 2>(acc2, sub, sub, tid >> 4, tid & 15);
+          tile_store<2, 2>(slots + tri(k + 1, k + 1) * kSlot, acc2, tid >> 4, tid & 15, -1.f, true);
+        } else {
+          for (int e = tid - 8 * 32; e < 2 * kB * kLcolLd; e += (kChainWarps - 8) * 32)
+            reinterpret_cast<uint32_t*>(lcol)[e] = kUnset;
         }
-        group_sync(1);
+        chain_sync();
       }
       if (tid == 0 && s_clamped && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_PIVOT_CLAMPED);
-    } else if (warp == 8) {
+    } else if (warp == kChainWarps) {
       // the sender: lane c copies each finished block to CTA c
       for (int step = 1; step <= 2 * nblk - 1; ++step) {
         // step 2k + 1: D_k^{-1} is ready;  step 2k + 2: L(k+1, k) is ready
@@ -497,65 +579,80 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
     }
   } else if (warp < 8) {
     // =========================================================== workers, factorisation half
-    const int row0 = warp * 4;
+    // Four pairs of warps; a pair does one 32 x 32 block product at a time (4 x 4 outputs per thread), the
+    // blocks of a phase are dealt out to the pairs in turn.  Warp h of a pair holds rows 16 h .. 16 h + 15.
+    const int pair = warp >> 1;
+    const int tp = tid & 63, tm = tp >> 3, tn = tp & 7;   // 4 x 4 outputs per thread on a pair of warps
+    const int t2m = tid >> 4, t2n = tid & 15;             // 2 x 2 outputs per thread on all eight warps
     const int n_mine = s_n_mine;
     for (int k = 0; k < nblk; ++k) {
-      if (tid == 0) bar_wait(&dinv_bar[k], &s_gave_up);
+      if (tid == 0) {
+        bar_wait(&dinv_bar[k], &s_gave_up);
+        s_urgent = 1;   // the other half of the CTA stands back until the chain has what it waits for
+      }
       group_sync(1);
       const float* dk = slots + tri(k, k) * kSlot;
-      // L(i, k) = A(i, k) D_k^{-T} for the blocks of column k this CTA owns (CTA 0 does block k + 1)
+      // L(i, k) = A(i, k) D_k^{-T} for the block of column k this CTA owns (CTA 0 does block k + 1): on the
+      // critical path, so all eight warps share the one product; in place
       for (int q = 0; q < n_mine; ++q) {
         const int bi = s_mine_i[q], bj = s_mine_j[q];
         if (bj != k || bi < k + 2) continue;
         float* blk = slots + tri(bi, k) * kSlot;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        mac_nt<4>(acc, blk + row0 * kLd, dk + lane * kLd);
-        __syncwarp();
-#pragma unroll
-        for (int rr = 0; rr < 4; ++rr) blk[(row0 + rr) * kLd + lane] = acc[rr];
+        float acc[2][2];
+        tile_zero(acc);
+        tile_mac<2, 2>(acc, blk, dk, t2m, t2n);
+        group_sync(1);   // everyone has read the block
+        tile_store<2, 2>(blk, acc, t2m, t2n, 1.f, false);
         fence_async_proxy();
-        send_strip(blk, row0, &panel_bar[k], 1, kCl - 1, cta, lane);
+        send_rows(blk, warp * 4, 4, &panel_bar[k], 1, kCl - 1, cta, lane);
       }
       // this CTA's own blocks of column k are in place: the second arrival on its own barrier
       group_sync(1);
       if (tid == 0 && k + 1 < nblk) bar_arrive_local(&panel_bar[k]);
-      if (k + 1 >= nblk) break;
+      if (k + 1 >= nblk) { if (tid == 0) s_urgent = 0; break; }
       if (tid == 0) bar_wait(&panel_bar[k], &s_gave_up);
       group_sync(1);
-      // trailing update with column k.  Pass 0: the two blocks CTA 0 needs next, sent on as soon as they
-      // are done.  Pass 1: the rest.  A diagonal block (j, j) takes columns k <= j - 2 here (CTA 0 applies
-      // column j - 1 itself), every other block (i, j) columns k <= j - 1.
-      for (int pass = 0; pass < 2; ++pass) {
-        for (int q = 0; q < n_mine; ++q) {
-          const int bi = s_mine_i[q], bj = s_mine_j[q];
-          if (bi < 2) continue;
-          const bool active = (bi == bj) ? (k <= bj - 2) : (k <= bj - 1);
-          if (!active) continue;
-          const bool urgent = (bi == k + 2) && (bj == k + 1 || bj == k + 2);
-          if (urgent != (pass == 0)) continue;
-          float acc[4] = {0.f, 0.f, 0.f, 0.f};
-          mac_nt<4>(acc, slots + tri(bi, k) * kSlot + row0 * kLd, slots + tri(bj, k) * kSlot + lane * kLd);
-          float* blk = slots + tri(bi, bj) * kSlot;
-          float v[4];
-#pragma unroll
-          for (int rr = 0; rr < 4; ++rr) v[rr] = blk[(row0 + rr) * kLd + lane] - acc[rr];
-#pragma unroll
-          for (int rr = 0; rr < 4; ++rr) blk[(row0 + rr) * kLd + lane] = v[rr];
-          if (urgent) {
-            fence_async_proxy();
-            send_strip(blk, row0, &chain_bar[k + 2], 0, 0, -1, lane);
-          }
-        }
+      // trailing update with column k.  A diagonal block (j, j) takes columns k <= j - 2 here (CTA 0
+      // applies column j - 1 itself), every other block (i, j) columns k <= j - 1.  First the two blocks
+      // CTA 0 needs next, each on all eight warps, sent on as soon as they are done ...
+      for (int q = 0; q < n_mine; ++q) {
+        const int bi = s_mine_i[q], bj = s_mine_j[q];
+        if (bi != k + 2 || (bj != k + 1 && bj != k + 2)) continue;
+        float acc[2][2];
+        tile_zero(acc);
+        tile_mac<2, 2>(acc, slots + tri(bi, k) * kSlot, slots + tri(bj, k) * kSlot, t2m, t2n);
+        float* blk = slots + tri(bi, bj) * kSlot;
+        tile_store<2, 2>(blk, acc, t2m, t2n, -1.f, true);
+        fence_async_proxy();
+        send_rows(blk, warp * 4, 4, &chain_bar[k + 2], 0, 0, -1, lane);
+      }
+      if (tid == 0) s_urgent = 0;
+      // ... then the rest, one block per pair of warps at a time
+      int turn = 0;
+      for (int q = 0; q < n_mine; ++q) {
+        const int bi = s_mine_i[q], bj = s_mine_j[q];
+        if (bi < 2) continue;
+        const bool active = (bi == bj) ? (k <= bj - 2) : (k <= bj - 1);
+        if (!active) continue;
+        if ((bi == k + 2) && (bj == k + 1 || bj == k + 2)) continue;
+        if ((turn++ & 3) != pair) continue;
+        float acc[4][4];
+        tile_zero(acc);
+        tile_mac<4, 4>(acc, slots + tri(bi, k) * kSlot, slots + tri(bj, k) * kSlot, tm, tn);
+        tile_store<4, 4>(slots + tri(bi, bj) * kSlot, acc, tm, tn, -1.f, true);
       }
     }
   } else {
     // =========================================================== workers, inverse half (warps 8..15)
     // Right-looking by block rows, in transposed storage Xt(i,j)[b][a] = X(i,j)[a][b]: at step k block row
     // k of the inverse becomes final, X(k,j) = -D_k^{-1} T(k,j) (X(k,k) = D_k^{-1}), is written out, and is
-    // added into the sums of all later rows, T(i,j) += L(i,k) X(k,j).  A warp only ever touches its own
-    // four rows b of every block (the columns of X are independent), except for the transposed copy.
+    // added into the sums of all later rows, T(i,j) += L(i,k) X(k,j).  Finishing a block is one product on
+    // all eight warps (2 x 2 outputs per thread); the products into the later rows are dealt out to four
+    // pairs of warps (4 x 4 outputs per thread).
     const int gt = tid - kGroup;
-    const int row0 = (warp - 8) * 4;
+    const int pair = (warp - 8) >> 1;
+    const int tp = gt & 63, tm = tp >> 3, tn = tp & 7;
+    const int t2m = gt >> 4, t2n = gt & 15;
     // block columns of the inverse this CTA computes: j0 = cta - 1, and 7 as well on the last worker
     const int j0 = cta - 1;
     const int n_cols = (j0 < nblk ? 1 : 0) + ((cta == kWorkers && kWorkers < nblk) ? 1 : 0);
@@ -587,11 +684,11 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
           }
         } else {
           // Xt(k,j)[b][a] = -sum_q Tt(k,j)[b][q] D_k^{-1}[a][q], in place
-          float acc[4] = {0.f, 0.f, 0.f, 0.f};
-          mac_nt<4>(acc, dst + row0 * kLd, dk + lane * kLd);
-          __syncwarp();
-#pragma unroll
-          for (int rr = 0; rr < 4; ++rr) dst[(row0 + rr) * kLd + lane] = -acc[rr];
+          float acc[2][2];
+          tile_zero(acc);
+          tile_mac<2, 2>(acc, dst, dk, t2m, t2n);
+          group_sync(2);   // everyone has read the sums
+          tile_store<2, 2>(dst, acc, t2m, t2n, -1.f, false);
         }
       }
       group_sync(2);
@@ -619,22 +716,19 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
       if (gt == 0) bar_wait(&panel_bar[k], &s_gave_up);
       group_sync(2);
       // Tt(i,j)[b][a] (+)= sum_q Xt(k,j)[b][q] L(i,k)[a][q] for the rows below
+      int turn = 0;
       for (int cidx = 0; cidx < n_cols; ++cidx) {
         const int j = j0 + cidx;
         if (j > k) continue;
         float* xcol = xt + (cidx == 0 ? 0 : (nblk - j0)) * kSlot;   // block (i, j) at xcol + (i - j) slots
-        const float* xk = xcol + (k - j) * kSlot + row0 * kLd;
+        const float* xk = xcol + (k - j) * kSlot;
         for (int i = k + 1; i < nblk; ++i) {
-          float acc[4] = {0.f, 0.f, 0.f, 0.f};
-          mac_nt<4>(acc, xk, slots + tri(i, k) * kSlot + lane * kLd);
-          float* dst = xcol + (i - j) * kSlot + row0 * kLd + lane;
-          if (j == k) {
-#pragma unroll
-            for (int rr = 0; rr < 4; ++rr) dst[rr * kLd] = acc[rr];
-          } else {
-#pragma unroll
-            for (int rr = 0; rr < 4; ++rr) dst[rr * kLd] += acc[rr];
-          }
+          if ((turn++ & 3) != pair) continue;
+          for (int spin = 0; s_urgent && spin < 256; ++spin) __nanosleep(64);   // a hint, not a lock
+          float acc[4][4];
+          tile_zero(acc);
+          tile_mac<4, 4>(acc, xk, slots + tri(i, k) * kSlot, tm, tn);
+          tile_store<4, 4>(xcol + (i - j) * kSlot, acc, tm, tn, 1.f, j != k);
         }
       }
     }
@@ -663,7 +757,7 @@ cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t str
   p.linv_hi = a.linv_hi;
   p.linv_lo = a.linv_lo;
   p.dev_status = a.dev_status;
-  const size_t smem = (size_t)(kMaxTri + kXSlots) * kSlot * sizeof(float) + (size_t)(kB * kLcolLd) * sizeof(float);
+  const size_t smem = (size_t)(kMaxTri + kXSlots) * kSlot * sizeof(float) + (size_t)(2 * kB * kLcolLd) * sizeof(float);
   static bool configured[64] = {};
   int dev = 0;
   LORACT_CUDA_TRY(cudaGetDevice(&dev));
