@@ -277,7 +277,8 @@ def _debug_lib():
 
 
 def debug_gemm(A_terms, B_terms, M: int, N: int, K: int, a_mn: bool, b_mn: bool, out_mode: int = OUT_F32,
-               engine: int = 1, splits: int = 1, acc64: bool = False, status: Optional[torch.Tensor] = None):
+               engine: int = 1, splits: int = 1, acc64: bool = False, status: Optional[torch.Tensor] = None,
+               out: Optional[Tuple[torch.Tensor, Optional[torch.Tensor]]] = None):
     """C = sum_t A_t B_t through one of the two contraction kernels.  Operands are 2-D row-major tensors
     stored [M][K] / [K][M] (a_mn) and [N][K] / [K][N] (b_mn).  Returns C (or (hi, lo), or the partials)."""
     l = _debug_lib()
@@ -286,7 +287,9 @@ def debug_gemm(A_terms, B_terms, M: int, N: int, K: int, a_mn: bool, b_mn: bool,
     PA = (ctypes.c_void_p * nt)(*[a.data_ptr() for a in A_terms])
     PB = (ctypes.c_void_p * nt)(*[b.data_ptr() for b in B_terms])
     tcode = lambda t: {torch.float32: 0, torch.bfloat16: 1}[t.dtype]
-    if out_mode == OUT_F32:
+    if out is not None:
+        C0, C1 = out          # caller-provided outputs (timing loops: nothing is allocated or cleared here)
+    elif out_mode == OUT_F32:
         C0 = torch.zeros(splits, M, N, dtype=torch.float32, device=dev); C1 = None
     elif out_mode == OUT_F64:
         C0 = torch.zeros(splits, M, N, dtype=torch.float64, device=dev); C1 = None

@@ -158,6 +158,7 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
     GemmDesc g;
     g.M = n; g.N = l; g.K = (int)p.d; g.lda = ldx; g.ldb = p.d; g.a_type = g.b_type = el;
     g.terms[0] = {X, Omega};
+    g.a_streams = true;
     g.ldc = l;
     if (p.bf16) { g.out = OUT_SPLIT; g.C0 = w.Yh; g.C1 = w.Yl; } else { g.out = OUT_F32; g.C0 = w.Y32; }
     LORACT_CUDA_TRY(run_gemm(g, status, stream));
@@ -206,6 +207,7 @@ cudaError_t project(const void* U, const void* X, int64_t ldx, const Plan& p, vo
   g.M = p.l; g.N = (int)p.d; g.K = (int)p.n; g.a_mn = true; g.b_mn = true; g.lda = p.l; g.ldb = ldx;
   g.a_type = g.b_type = p.bf16 ? ELEM_BF16 : ELEM_F32;
   g.terms[0] = {U, X};
+  g.b_streams = true;
   g.ldc = p.d;
   if (!p.bf16) { g.out = OUT_F32; g.C0 = V; return run_gemm(g, status, stream); }
   if (w.splits_v <= 1) { g.out = OUT_BF16; g.C0 = V; return run_gemm(g, status, stream); }

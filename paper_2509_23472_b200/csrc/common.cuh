@@ -81,6 +81,8 @@ struct GemmDesc {
   bool acc64 = false;      // SIMT path: accumulate in double
   bool accumulate = false; // SIMT path, OUT_F32, splits == 1: C += result
   float alpha = 1.0f;      // SIMT path: C = alpha * sum
+  // tensor-core path: the operand is large and read once from HBM (the activation matrix): prefetch it
+  bool a_streams = false, b_streams = false;
 };
 
 // tcgen05 engine: bf16 operands, fp32 accumulation in tensor memory.  Returns cudaErrorNotSupported
