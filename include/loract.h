@@ -58,7 +58,7 @@ typedef struct {
   int64_t d;             /* columns of X (the paper's n)                                     */
   int64_t ldx;           /* row stride of X in elements, >= d                                */
   int32_t rank;          /* r (the paper's k)                                                */
-  int32_t power_iters;   /* t of Algorithm 1; only 0 is implemented on the device            */
+  int32_t power_iters;   /* t of Algorithm 1 (lines 3 to 6), 0 <= t <= 8; the paper's runs use 0   */
   int32_t dtype;         /* loract_dtype_t of X, U, V, X_out, A_out, G, gamma, beta          */
   int32_t reserved;      /* must be 0                                                        */
   uint64_t seed;         /* Philox key                                                       */
@@ -76,7 +76,8 @@ size_t loract_workspace_bytes(const loract_desc_t* desc);
 loract_status_t loract_sample_indices(const loract_desc_t* desc, int32_t* idx_dev, void* ws,
                                       size_t ws_bytes, void* stream);
 
-/* Algorithm 1 with t = 0: sample rows, Y = X A_k^T, orthonormalise Y to Q, U = Q, V = Q^T X.
+/* Algorithm 1: sample rows, Y = X A_k^T, t = power_iters times { Y = QR, Y = X (X^T Q) }, Y = QR, U = Q,
+ * V = Q^T X.  (t = 0 is the setting of the paper's experiments.)
  * X: device, read only.  U (n_tokens x rank), V (rank x d): device, written.  idx_out: device, `rank`
  * int32, written if not NULL.  U has orthonormal columns; U V is the orthogonal projection of X onto
  * range(Y).  The entries of U are not unique (any orthonormal basis of range(Y) is a valid result). */

@@ -145,10 +145,11 @@ def sample_indices(desc: Desc, device, ws: Optional[torch.Tensor] = None) -> tor
 
 
 def compress(X: torch.Tensor, rank: int, seed: int = 0, call_id: int = 0, ws: Optional[torch.Tensor] = None,
-             out: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None, desc: Optional[Desc] = None):
-    """Algorithm 1 (t = 0).  Returns (U, V, idx)."""
+             out: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None, desc: Optional[Desc] = None,
+             power_iters: int = 0):
+    """Algorithm 1 with t = power_iters.  Returns (U, V, idx)."""
     _cuda(X, "X")
-    desc = desc or make_desc(X, rank, seed, call_id)
+    desc = desc or make_desc(X, rank, seed, call_id, power_iters)
     ws = ws if ws is not None else alloc_workspace(desc, X.device)
     if out is None:
         U = torch.empty(X.shape[0], rank, dtype=X.dtype, device=X.device)

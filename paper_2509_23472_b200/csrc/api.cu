@@ -17,6 +17,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // relative diagonal shifts of the three Cholesky factorisations (fp32 small blocks)
+constexpr int kMaxPowerIters = 8;      // t of Algorithm 1 accepted by loract_compress
 constexpr float kShiftSample = 1e-6f;  // Gram of the sampled rows
 constexpr float kShiftFirst = 3e-6f;   // first Gram of the sketch
 constexpr float kShiftSecond = 1e-7f;  // second Gram (already close to the identity)
@@ -41,7 +42,7 @@ loract_status_t check_desc(const loract_desc_t* d) {
   if (d->rank < 16 || d->rank > 512 || d->rank % 16) return LORACT_ERR_INVALID_ARG;
   if (d->rank > d->n_tokens || d->rank > d->d) return LORACT_ERR_INVALID_ARG;
   if (d->power_iters < 0) return LORACT_ERR_INVALID_ARG;
-  if (d->power_iters != 0) return LORACT_ERR_UNSUPPORTED;
+  if (d->power_iters > kMaxPowerIters) return LORACT_ERR_UNSUPPORTED;
   const int64_t mult = d->dtype == LORACT_BF16 ? 8 : 4;
   if (d->d % mult || d->ldx % mult) return LORACT_ERR_ALIGNMENT;
   return LORACT_OK;
@@ -254,25 +255,31 @@ cudaError_t compress_core(const loract_desc_t* desc, const void* X, int64_t ldx,
                                         w.status, stream));
   if (idx_out) LORACT_CUDA_TRY(cudaMemcpyAsync(idx_out, w.idx, (size_t)r * 4, cudaMemcpyDeviceToDevice, stream));
   LORACT_CUDA_TRY(gather_rows_launch(X, ldx, w.idx, r, desc->d, elem_bytes(desc), w.S, stream));
-  // small-block preconditioning: Omega = L_s^{-1} A_k with A_k A_k^T = L_s L_s^T.  Omega has the row
-  // space of A_k, so range(X Omega^T) = range(X A_k^T) (line 2), but its rows are close to orthonormal,
-  // which keeps the spectrum of the sketch from being squared.
-  LORACT_CUDA_TRY(gram_rows(w.S, r, desc->d, bf16, w.b, w.status, stream));
-  LORACT_CUDA_TRY(factor(r, bf16, w.b.splits_gram_sample, kShiftSample, w.b, w.status, stream));
-  {
-    GemmDesc g;
-    g.M = r; g.N = (int)desc->d; g.K = r; g.b_mn = true; g.lda = r; g.ldb = desc->d;
-    g.a_type = g.b_type = bf16 ? ELEM_BF16 : ELEM_F32;
-    g.ldc = desc->d; g.C0 = w.Omega;
-    if (bf16) {
-      g.n_terms = 2; g.terms[0] = {w.b.Lh, w.S}; g.terms[1] = {w.b.Ll, w.S}; g.out = OUT_BF16;
-    } else {
-      g.terms[0] = {w.b.Linv32, w.S}; g.out = OUT_F32;
+  // Lines 2 to 7.  The test matrix (the sampled rows A_k at first, Q^T X in the power iterations of lines
+  // 3 to 6) is preconditioned before every product with X: with T T^T = L L^T, Omega = L^{-1} T has the row
+  // space of T, so range(X Omega^T) = range(X T^T), but its rows are close to orthonormal, which keeps the
+  // spectrum of the sketch from being squared (and, in the iterations, raised to the fourth power).
+  for (int it = 0; it <= desc->power_iters; ++it) {
+    LORACT_CUDA_TRY(gram_rows(w.S, r, desc->d, bf16, w.b, w.status, stream));
+    LORACT_CUDA_TRY(factor(r, bf16, w.b.splits_gram_sample, kShiftSample, w.b, w.status, stream));
+    {
+      GemmDesc g;
+      g.M = r; g.N = (int)desc->d; g.K = r; g.b_mn = true; g.lda = r; g.ldb = desc->d;
+      g.a_type = g.b_type = bf16 ? ELEM_BF16 : ELEM_F32;
+      g.ldc = desc->d; g.C0 = w.Omega;
+      if (bf16) {
+        g.n_terms = 2; g.terms[0] = {w.b.Lh, w.S}; g.terms[1] = {w.b.Ll, w.S}; g.out = OUT_BF16;
+      } else {
+        g.terms[0] = {w.b.Linv32, w.S}; g.out = OUT_F32;
+      }
+      LORACT_CUDA_TRY(run_gemm(g, w.status, stream));
     }
-    LORACT_CUDA_TRY(run_gemm(g, w.status, stream));
+    // Y = X Omega^T, Y = QR (Q written to U)
+    LORACT_CUDA_TRY(range_basis(X, ldx, plan, w.Omega, U, w.b, w.status, stream));
+    // lines 4 and 5 of the loop: the next test matrix is (X^T Q)^T = Q^T X, kept where A_k was
+    if (it < desc->power_iters) LORACT_CUDA_TRY(project(U, X, ldx, plan, w.S, w.b, w.status, stream));
   }
-  // lines 2 and 7: Q, written to U;  line 8: V = U^T X
-  LORACT_CUDA_TRY(range_basis(X, ldx, plan, w.Omega, U, w.b, w.status, stream));
+  // line 8: V = U^T X
   return project(U, X, ldx, plan, V, w.b, w.status, stream);
 }
 

@@ -51,9 +51,10 @@ def _desc(**kw):
 def test_workspace_query_and_invalid_descriptors(lib):
     assert B.workspace_bytes(_desc()) > 0
     assert B.workspace_bytes(_desc(dtype=B.F32)) > 0
+    assert B.workspace_bytes(_desc(power_iters=2)) > 0
     bad = [dict(rank=0), dict(rank=24), dict(rank=528), dict(rank=2048, n_tokens=4096, d=4096),
            dict(n_tokens=32), dict(d=32, ldx=32), dict(ldx=256), dict(dtype=7), dict(reserved=1),
-           dict(d=516, ldx=516), dict(power_iters=-1), dict(power_iters=1)]
+           dict(d=516, ldx=516), dict(power_iters=-1), dict(power_iters=9)]
     for kw in bad:
         assert B.workspace_bytes(_desc(**kw)) == 0, kw
     # workspace grows with the problem
@@ -70,7 +71,7 @@ def test_bad_arguments_return_codes_and_launch_nothing(lib):
     assert lib.loract_compress(ctypes.byref(d), odd, one, one, null, one, 1 << 30, null) == 3
     assert lib.loract_compress(ctypes.byref(d), one, one, one, null, one, 16, null) == 4
     assert lib.loract_compress(ctypes.byref(_desc(rank=24)), one, one, one, null, one, 1 << 30, null) == 1
-    assert lib.loract_compress(ctypes.byref(_desc(power_iters=2)), one, one, one, null, one, 1 << 30, null) == 2
+    assert lib.loract_compress(ctypes.byref(_desc(power_iters=9)), one, one, one, null, one, 1 << 30, null) == 2
     assert lib.loract_compress(ctypes.byref(_desc(d=516, ldx=516)), one, one, one, null, one, 1 << 30, null) == 3
     assert lib.loract_reconstruct(ctypes.byref(d), one, null, one, null) == 1
     assert lib.loract_weight_grad(ctypes.byref(d), one, one, one, 0, 16, one, 0, one, 1 << 30, null) == 1

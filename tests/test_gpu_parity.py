@@ -199,3 +199,38 @@ def test_rsvd_comparator(dev):
     # a power iteration does not hurt
     Q0, B0 = B.rsvd(X, 64, oversample=16, power_iters=0, seed=3)
     assert e_gpu <= gpu_err(X64, Q0, B0) + 2e-3
+
+
+# ------------------------------------------------------------------ power iterations (Algorithm 1, lines 3 to 6)
+@pytest.mark.parametrize("t", [1, 2])
+def test_power_iterations_match_the_oracle_and_help_on_a_flat_spectrum(dev, t):
+    # a slowly decaying spectrum with strong noise: the regime in which the loop of Algorithm 1 pays
+    w = synth.scaled(synth.get_workload("llama13b_s1024_r64"), n_tokens=2048, d=1024, rank=64, signal_rank=256)
+    X = synth.make_inputs(w, device=dev)["X"]
+    X64 = X.double()
+    Xd = to64(X)
+    errs = {}
+    for tt in (0, t):
+        U, V, idx = B.compress(X, 64, seed=w.seed, power_iters=tt)
+        torch.cuda.synchronize()
+        Uo, Vo, io = orc.decompose(Xd, 64, t=tt, seed=w.seed)
+        assert np.array_equal(idx.cpu().numpy().astype(np.int64), io)
+        e_gpu, e_ref = gpu_err(X64, U, V), orc.rel_fro_error(Xd, Uo, Vo)
+        assert abs(e_gpu - e_ref) <= TOL_ERR["bf16"], (tt, e_gpu, e_ref)
+        assert orth_defect(U) <= orth_bound(U)
+        errs[tt] = (e_gpu, e_ref)
+    # the loop must not make things worse, on either side (it improves the oracle's error on this input)
+    assert errs[t][1] <= errs[0][1] + 1e-12
+    assert errs[t][0] <= errs[0][0] + 2e-3
+
+
+def test_power_iterations_fp32(dev):
+    w = synth.scaled(synth.WORKLOADS["small_f32"], n_tokens=384, d=256, rank=32, signal_rank=96)
+    X = synth.make_inputs(w, device=dev)["X"]
+    Xd = to64(X)
+    U, V, idx = B.compress(X, 32, seed=w.seed, power_iters=2)
+    torch.cuda.synchronize()
+    Uo, Vo, io = orc.decompose(Xd, 32, t=2, seed=w.seed)
+    assert np.array_equal(idx.cpu().numpy().astype(np.int64), io)
+    assert abs(gpu_err(X.double(), U, V) - orc.rel_fro_error(Xd, Uo, Vo)) <= TOL_ERR["f32"]
+    assert orth_defect(U) <= TOL_ORTH
