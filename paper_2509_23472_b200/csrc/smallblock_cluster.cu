@@ -3,20 +3,26 @@
 // matrices), as one thread-block-cluster kernel whose working set never leaves shared memory.
 //
 // The matrix is cut into 32 x 32 blocks.  Eight CTAs form a cluster:
-//   * CTA 0 is the pivot chain.  For block column k one warp factors the diagonal block in registers
-//     (shuffles) and inverts it; the CTA then forms L(k+1,k) = A(k+1,k) D_k^{-T} and applies it to the next
-//     diagonal block itself, so the chain waits for nothing but the two blocks it needs next.
+//   * CTA 0 is the pivot chain.  For block column k two warps factor the diagonal block in registers
+//     (one the columns 0..15, one the columns 16..31) while eight more invert the factor alongside; the
+//     CTA then forms L(k+1,k) = A(k+1,k) D_k^{-T} and applies it to the next diagonal block itself, so the
+//     chain waits for nothing but the two blocks it needs next.  One more warp only sends.
 //   * CTAs 1..7 own all blocks (dealt out column by column).  Half of their warps do the factorisation:
 //     for column k each forms its L(i,k), then updates its trailing blocks, A(i,j) -= L(i,k) L(j,k)^T; the
 //     two blocks the chain needs next, (k+2,k+1) and (k+2,k+2), are updated first and sent to CTA 0.
-//     The other half computes the inverse X = L^{-1} by block columns,
-//     X(i,j) = -D_i^{-1} sum_c L(i,c) X(c,j), one block row per step, behind the factorisation.
-//   * Every finished block (D_k^{-1}, L(i,k)) is written into the same slot of every worker's shared
-//     memory with asynchronous distributed-shared-memory stores that count bytes on an mbarrier of the
-//     receiving CTA (st.async ... mbarrier::complete_tx), so each worker ends up with a full copy of L
-//     without a global-memory round trip, a fence or a remote arrive.
-// Every wait is bounded by a wall-clock limit; on expiry the CTA records LORACT_DEV_WAIT_EXPIRED, stops
-// waiting and runs to its end (results are then invalid but every access stays in bounds).
+//     The other half computes the inverse X = L^{-1} by block columns, right-looking: block row k becomes
+//     final at step k, X(k,j) = -D_k^{-1} T(k,j), is written out and added into the sums of the later rows,
+//     T(i,j) += L(i,k) X(k,j).  It stands back while the first half is on the chain's critical path.
+//   * Every finished block (D_k^{-1}, L(i,k)) is copied into the same slot of every worker's shared memory
+//     with bulk distributed-shared-memory copies (cp.async.bulk shared::cta -> shared::cluster) that count
+//     bytes on an mbarrier of the receiving CTA, so each worker ends up with a full copy of L without a
+//     global-memory round trip, a fence or a remote arrive.  (16-byte st.async stores were tried first:
+//     one barrier update per 16 bytes made the sends the bottleneck.)
+//   * 32 x 32 block products run on CUDA cores with 4 x 4 (or 2 x 2) outputs per thread; they are bound by
+//     shared-memory bandwidth (a 16-byte load costs about four cycles of the pipe), hence the tiling.
+// Every wait is bounded (a wall-clock limit for barriers, an iteration limit for flag words); on expiry the
+// CTA records LORACT_DEV_WAIT_EXPIRED, stops waiting and runs to its end (results are then invalid but
+// every access stays in bounds).
 #include "common.cuh"
 
 namespace loract {
@@ -66,13 +72,6 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, int rank) {
 __device__ __forceinline__ void st_cluster_v4(uint32_t addr, float4 v) {
   asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z),
                "f"(v.w)
-               : "memory");
-}
-// 16 bytes into another CTA's shared memory; on arrival 16 is taken off the transaction count of `bar`
-// (an mbarrier of the same CTA).
-__device__ __forceinline__ void st_async_v4(uint32_t addr, float4 v, uint32_t bar) {
-  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
-               ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(bar)
                : "memory");
 }
 __device__ __forceinline__ void bar_init(uint64_t* bar, uint32_t count) {
