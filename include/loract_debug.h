@@ -27,6 +27,14 @@ loract_status_t loract_debug_gemm(int32_t M, int32_t N, int32_t K, int32_t a_mn,
                                   void* C0, void* C1, int64_t ldc, int32_t splits, int64_t split_stride,
                                   int32_t acc64, int32_t engine, uint32_t* status_word, void* stream);
 
+/* The tensor-core kernel exists in two forms: one CTA per 128-row tile, and a pair of CTAs (tcgen05
+ * cta_group::2) per 256-row tile, chosen by shape.  on = 0 keeps every contraction on the one-CTA form, so
+ * that a test can compare the two; on = 1 (the default) restores the choice by shape.  Process-wide. */
+void loract_debug_set_pair_mode(int32_t on);
+
+/* The cudaError_t behind the most recent LORACT_ERR_CUDA returned by any entry point (0 if none yet). */
+int32_t loract_debug_last_cuda_error(void);
+
 /* The small-block step of the orthonormalisation (Algorithm 1 line 7 done through Gram matrices):
  * W = sum of n_partials r x r matrices (fp32 if partial_f64 == 0, else fp64; `partial_stride` elements
  * apart); L L^T = W + shift_rel * mean(diag W) * I; writes L^{-1} (lower triangular, row-major) as fp32

@@ -34,7 +34,13 @@ class Desc(ctypes.Structure):
 
 class LoractError(RuntimeError):
     def __init__(self, code: int, what: str):
-        super().__init__(f"{what}: status {code} ({status_string(code)})")
+        extra = ""
+        if code == 5:
+            try:
+                extra = f", cudaError {int(lib().loract_debug_last_cuda_error())}"
+            except Exception:
+                pass
+        super().__init__(f"{what}: status {code} ({status_string(code)}{extra})")
         self.code = code
 
 
@@ -261,7 +267,8 @@ def read_device_status(ws: torch.Tensor) -> int:
 # Test hooks (include/loract_debug.h)
 # ---------------------------------------------------------------------------------------------
 OUT_F32, OUT_BF16, OUT_SPLIT, OUT_F64 = 0, 1, 2, 3
-DEBUG_EXPORTS = ("loract_debug_gemm", "loract_debug_small_block")
+DEBUG_EXPORTS = ("loract_debug_gemm", "loract_debug_small_block", "loract_debug_set_pair_mode",
+                 "loract_debug_last_cuda_error")
 
 
 def _debug_lib():
@@ -304,6 +311,14 @@ def debug_gemm(A_terms, B_terms, M: int, N: int, K: int, a_mn: bool, b_mn: bool,
     if out_mode in (OUT_F32, OUT_F64):
         return C0 if splits > 1 else C0[0]
     return C0 if C1 is None else (C0, C1)
+
+
+def debug_set_pair_mode(on: bool) -> None:
+    """Test hook: False keeps every contraction on the one-CTA tensor-core kernel."""
+    l = _debug_lib()
+    l.loract_debug_set_pair_mode.restype = None
+    l.loract_debug_set_pair_mode.argtypes = [ctypes.c_int32]
+    l.loract_debug_set_pair_mode(1 if on else 0)
 
 
 def debug_small_block(partials: torch.Tensor, use_f64: bool, shift_rel: float,

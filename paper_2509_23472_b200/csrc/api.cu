@@ -306,7 +306,12 @@ size_t carve_wgrad(void* ws, const loract_desc_t* desc, int g, WgradWs* out) {
   return c.off;
 }
 
-loract_status_t from_cuda(cudaError_t e) { return e == cudaSuccess ? LORACT_OK : LORACT_ERR_CUDA; }
+std::atomic<int> g_last_cuda_error{0};
+loract_status_t from_cuda(cudaError_t e) {
+  if (e == cudaSuccess) return LORACT_OK;
+  g_last_cuda_error.store((int)e, std::memory_order_relaxed);
+  return LORACT_ERR_CUDA;
+}
 
 }  // namespace
 }  // namespace loract
@@ -528,6 +533,10 @@ loract_status_t loract_debug_gemm(int32_t M, int32_t N, int32_t K, int32_t a_mn,
   }
   return from_cuda(gemm_simt_launch(g, (cudaStream_t)stream));
 }
+
+void loract_debug_set_pair_mode(int32_t on) { gemm_tc_set_pair_mode(on); }
+
+int32_t loract_debug_last_cuda_error(void) { return g_last_cuda_error.load(std::memory_order_relaxed); }
 
 loract_status_t loract_debug_small_block(int32_t r, const void* partials, int32_t partial_f64, int32_t n_partials,
                                          int64_t partial_stride, int32_t use_f64, float shift_rel, void* scratch,

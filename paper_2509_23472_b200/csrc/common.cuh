@@ -90,6 +90,7 @@ struct GemmDesc {
 bool gemm_tc_supported(const GemmDesc& g);
 cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t stream);
 int gemm_tc_pick_splits(int M, int N, int K, bool a_mn, bool b_mn);
+void gemm_tc_set_pair_mode(int on);   // test hook: 0 keeps every contraction on the one-CTA kernel
 
 // Plain CUDA-core kernel for any shape and type (fp32 path, small or odd shapes).
 cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t stream);

@@ -151,6 +151,74 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
+// Epilogue of one CTA (four warps): reads its 128 accumulator rows (tensor-memory lanes) and writes them.
+// Warp w may touch the lanes 32 * (w % 4) .. + 31.
+__device__ __forceinline__ void tc_epilogue(const TcParams& p, uint32_t tmem_base, uint64_t* accum_bar,
+                                          volatile int* abort_flag_ptr, int warp, int lane, int m0, int n0,
+                                          int split, int n_iter) {
+  const int quad = warp & 3;
+  const int row = quad * 32 + lane;
+  const int m = m0 + row;
+  bool ok = mbar_wait_bounded(accum_bar, 0, abort_flag_ptr);
+  ok = __all_sync(0xffffffffu, ok);
+  tc_fence_after();
+  if (ok && n_iter > 0) {
+    for (int c0 = 0; c0 < p.bn; c0 += 32) {
+      uint32_t v[32];
+      tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
+      tc_wait_ld();
+      const int n = n0 + c0;
+      if (m >= p.M) continue;
+      const int valid = min(32, min(p.bn - c0, p.N - n));
+      if (valid <= 0) continue;
+      if (p.out == OUT_F32) {
+        float* dst = (float*)p.C0 + (int64_t)split * p.split_stride + (int64_t)m * p.ldc + n;
+        if (p.accumulate) {
+          for (int q = 0; q < valid; ++q) dst[q] += __uint_as_float(v[q]);
+        } else if (valid == 32 && ((((uintptr_t)dst) & 15) == 0)) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            reinterpret_cast<uint4*>(dst)[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        } else {
+          for (int q = 0; q < valid; ++q) dst[q] = __uint_as_float(v[q]);
+        }
+      } else {
+        __nv_bfloat16* dst_hi = (__nv_bfloat16*)p.C0 + (int64_t)m * p.ldc + n;
+        __nv_bfloat16* dst_lo = (p.out == OUT_SPLIT) ? (__nv_bfloat16*)p.C1 + (int64_t)m * p.ldc + n : nullptr;
+        if (valid == 32 && ((((uintptr_t)dst_hi) & 15) == 0)) {
+          uint32_t hi[16], lo[16];
+#pragma unroll
+          for (int q = 0; q < 16; ++q) {
+            const float x0 = __uint_as_float(v[2 * q]), x1 = __uint_as_float(v[2 * q + 1]);
+            const __nv_bfloat16 h0 = __float2bfloat16(x0), h1 = __float2bfloat16(x1);
+            hi[q] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+            lo[q] = pack_bf16x2(x0 - __bfloat162float(h0), x1 - __bfloat162float(h1));
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            reinterpret_cast<uint4*>(dst_hi)[q] = make_uint4(hi[4 * q], hi[4 * q + 1], hi[4 * q + 2], hi[4 * q + 3]);
+          if (dst_lo) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              reinterpret_cast<uint4*>(dst_lo)[q] = make_uint4(lo[4 * q], lo[4 * q + 1], lo[4 * q + 2], lo[4 * q + 3]);
+          }
+        } else {
+          for (int q = 0; q < valid; ++q) {
+            const float x = __uint_as_float(v[q]);
+            const __nv_bfloat16 h = __float2bfloat16(x);
+            dst_hi[q] = h;
+            if (dst_lo) dst_lo[q] = __float2bfloat16(x - __bfloat162float(h));
+          }
+        }
+      }
+    }
+  } else if (ok && n_iter == 0 && m < p.M && p.out == OUT_F32) {
+    // an empty K range still owns its partial: write zeros
+    float* dst = (float*)p.C0 + (int64_t)split * p.split_stride + (int64_t)m * p.ldc + n0;
+    for (int q = 0; q < min(p.bn, p.N - n0); ++q) dst[q] = 0.f;
+  }
+  }
+
 template <bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
@@ -265,74 +333,170 @@ gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
       tc_commit(&accum_bar);       // accumulator complete (or nothing was issued)
     }
   } else {
-    // epilogue: warp w may touch tensor-memory lanes 32 * (w % 4) .. + 31
-    const int quad = warp & 3;
-    const int row = quad * 32 + lane;
-    const int m = m0 + row;
-    bool ok = mbar_wait_bounded(&accum_bar, 0, &abort_flag);
-    ok = __all_sync(0xffffffffu, ok);
-    tc_fence_after();
-    if (ok && n_iter > 0) {
-      for (int c0 = 0; c0 < p.bn; c0 += 32) {
-        uint32_t v[32];
-        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
-        tc_wait_ld();
-        const int n = n0 + c0;
-        if (m >= p.M) continue;
-        const int valid = min(32, min(p.bn - c0, p.N - n));
-        if (valid <= 0) continue;
-        if (p.out == OUT_F32) {
-          float* dst = (float*)p.C0 + (int64_t)split * p.split_stride + (int64_t)m * p.ldc + n;
-          if (p.accumulate) {
-            for (int q = 0; q < valid; ++q) dst[q] += __uint_as_float(v[q]);
-          } else if (valid == 32 && ((((uintptr_t)dst) & 15) == 0)) {
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-              reinterpret_cast<uint4*>(dst)[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-          } else {
-            for (int q = 0; q < valid; ++q) dst[q] = __uint_as_float(v[q]);
-          }
-        } else {
-          __nv_bfloat16* dst_hi = (__nv_bfloat16*)p.C0 + (int64_t)m * p.ldc + n;
-          __nv_bfloat16* dst_lo = (p.out == OUT_SPLIT) ? (__nv_bfloat16*)p.C1 + (int64_t)m * p.ldc + n : nullptr;
-          if (valid == 32 && ((((uintptr_t)dst_hi) & 15) == 0)) {
-            uint32_t hi[16], lo[16];
-#pragma unroll
-            for (int q = 0; q < 16; ++q) {
-              const float x0 = __uint_as_float(v[2 * q]), x1 = __uint_as_float(v[2 * q + 1]);
-              const __nv_bfloat16 h0 = __float2bfloat16(x0), h1 = __float2bfloat16(x1);
-              hi[q] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-              lo[q] = pack_bf16x2(x0 - __bfloat162float(h0), x1 - __bfloat162float(h1));
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-              reinterpret_cast<uint4*>(dst_hi)[q] = make_uint4(hi[4 * q], hi[4 * q + 1], hi[4 * q + 2], hi[4 * q + 3]);
-            if (dst_lo) {
-#pragma unroll
-              for (int q = 0; q < 4; ++q)
-                reinterpret_cast<uint4*>(dst_lo)[q] = make_uint4(lo[4 * q], lo[4 * q + 1], lo[4 * q + 2], lo[4 * q + 3]);
-            }
-          } else {
-            for (int q = 0; q < valid; ++q) {
-              const float x = __uint_as_float(v[q]);
-              const __nv_bfloat16 h = __float2bfloat16(x);
-              dst_hi[q] = h;
-              if (dst_lo) dst_lo[q] = __float2bfloat16(x - __bfloat162float(h));
-            }
-          }
-        }
-      }
-    } else if (ok && n_iter == 0 && m < p.M && p.out == OUT_F32) {
-      // an empty K range still owns its partial: write zeros
-      float* dst = (float*)p.C0 + (int64_t)split * p.split_stride + (int64_t)m * p.ldc + n0;
-      for (int q = 0; q < min(p.bn, p.N - n0); ++q) dst[q] = 0.f;
-    }
+    tc_epilogue(p, tmem_base, &accum_bar, &abort_flag, warp, lane, m0, n0, split, n_iter);
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols)
+                 : "memory");
+  }
+  if (threadIdx.x == 0 && abort_flag && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_WAIT_EXPIRED);
+}
+
+// ------------------------------------------------------------------ two CTAs on one tile
+// The same contraction with a pair of CTAs (a cluster of two along M) on one 256 x bn tile
+// (tcgen05 cta_group::2): each CTA loads its 128 rows of A and HALF of the B tile, the tensor cores of both
+// SMs read both halves, and each CTA ends up with its 128 rows of the accumulator in its own tensor
+// memory.  Per SM and K block this moves 16 KB + half a B tile instead of 16 KB + a whole one, which is
+// what limits the one-CTA kernel when B is re-read from L2 by every CTA; the ring gets six stages.
+//   * Both CTAs allocate tensor memory (cta_group::2) and run a TMA producer; the loads of both complete
+//     on the full barrier of the even CTA (the leader), which alone issues the MMAs.
+//   * tcgen05.commit (cta_group::2, multicast to both CTAs) frees a stage in both CTAs and, at the end,
+//     tells both epilogues that the accumulator is complete.
+//   * No load uses cluster multicast.
+constexpr int kPairStages = 6;
+
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+// TMA load whose bytes are counted on a barrier that may live in the peer CTA.
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* map, uint32_t bar_cluster_addr,
+                                                 int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(smem_u32(bar)), "h"((uint16_t)3)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+template <bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  __shared__ __align__(8) uint64_t full_bar[kPairStages];    // used in the leader: both CTAs' loads of a stage
+  __shared__ __align__(8) uint64_t empty_bar[kPairStages];   // in each CTA: the MMAs have read the stage
+  __shared__ __align__(8) uint64_t accum_bar;                // in each CTA: the accumulator is complete
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+
+  uint32_t cta_rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(cta_rank));
+  const bool leader = cta_rank == 0;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int half_n = p.bn / 2;                               // B rows (or columns) this CTA loads
+  // grid: x = 128-row tiles (the two CTAs of a pair are neighbours in x), y = column tiles, z = K splits
+  const int n0 = blockIdx.y * p.bn, m0 = blockIdx.x * kBM, split = blockIdx.z;
+  const int kb_begin = split * p.kb_per_split;
+  const int kb_count = max(0, min(p.kb_total, kb_begin + p.kb_per_split) - kb_begin);
+  const int n_iter = kb_count * p.n_terms;
+  const uint32_t stage_bytes = kABytes + p.b_bytes;          // per CTA (b_bytes: half a B tile)
+  unsigned char* tiles = (unsigned char*)(((uintptr_t)smem + 1023) & ~(uintptr_t)1023);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kPairStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    mbar_init(&accum_bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                 "r"(p.tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  // both CTAs' barriers exist before either CTA signals the other
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_slot;
+  pdl_wait();
+  pdl_launch_dependents();
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const int nb0 = n0 + (int)cta_rank * half_n;           // this CTA's half of the B tile
+      for (int it = 0; it < n_iter; ++it) {
+        const int s = it % kPairStages;
+        if (!mbar_wait_bounded(&empty_bar[s], ((it / kPairStages) & 1) ^ 1, &abort_flag)) break;
+        const int term = it / kb_count;
+        const int k0 = (kb_begin + (it - term * kb_count)) * kBK;
+        unsigned char* a_dst = tiles + (size_t)s * stage_bytes;
+        unsigned char* b_dst = a_dst + kABytes;
+        // the leader expects the bytes of both CTAs on its barrier
+        if (leader) mbar_arrive_expect_tx(&full_bar[s], 2u * stage_bytes);
+        const uint32_t bar = map_to_rank(smem_u32(&full_bar[s]), 0u);
+        if (A_MN) {
+          tma_load_2d_pair(a_dst, &maps.a[term], bar, m0, k0);
+          tma_load_2d_pair(a_dst + 8192, &maps.a[term], bar, m0 + 64, k0);
+        } else {
+          tma_load_2d_pair(a_dst, &maps.a[term], bar, k0, m0);
+        }
+        if (B_MN) {
+          for (uint32_t q = 0; q * 8192u < p.b_bytes; ++q)
+            tma_load_2d_pair(b_dst + q * 8192u, &maps.b[term], bar, nb0 + (int)q * 64, k0);
+        } else {
+          tma_load_2d_pair(b_dst, &maps.b[term], bar, k0, nb0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && leader) {
+      // instruction descriptor: fp32 accumulator, bf16 A and B, operand majors, N >> 3, M = 256 >> 4
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
+                             ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(p.bn >> 3) << 17) |
+                             ((uint32_t)((2 * kBM) >> 4) << 24);
+      bool ok = true;
+      for (int it = 0; it < n_iter && ok; ++it) {
+        const int s = it % kPairStages;
+        ok = mbar_wait_bounded(&full_bar[s], (it / kPairStages) & 1, &abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(tiles + (size_t)s * stage_bytes);
+        const uint32_t b_addr = a_addr + kABytes;
+        const uint64_t a_desc = make_smem_desc(a_addr, A_MN);
+        const uint64_t b_desc = make_smem_desc(b_addr, B_MN);
+#pragma unroll
+        for (int k = 0; k < kBK / 16; ++k) {
+          const uint64_t a_k = a_desc + (uint64_t)((A_MN ? 2048u : 32u) >> 4) * k;
+          const uint64_t b_k = b_desc + (uint64_t)((B_MN ? 2048u : 32u) >> 4) * k;
+          tc_mma_bf16_pair(tmem_base, a_k, b_k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+        }
+        tc_commit_pair(&empty_bar[s]);   // frees the stage in both CTAs once these MMAs have read it
+      }
+      tc_commit_pair(&accum_bar);        // accumulator complete in both CTAs (or nothing was issued)
+    }
+  } else {
+    tc_epilogue(p, tmem_base, &accum_bar, &abort_flag, warp, lane, m0, n0, split, n_iter);
+  }
+  tc_fence_before();
+  __syncthreads();
+  // neither CTA frees tensor memory or leaves while the other may still use its shared or tensor memory
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols)
                  : "memory");
   }
   if (threadIdx.x == 0 && abort_flag && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_WAIT_EXPIRED);
@@ -420,7 +584,40 @@ cudaError_t launch_variant(const TmapPack& maps, const TcParams& p, dim3 grid, s
   return cudaGetLastError();
 }
 
+template <bool A_MN, bool B_MN>
+cudaError_t launch_pair_variant(const TmapPack& maps, const TcParams& p, dim3 grid, size_t smem, cudaStream_t stream) {
+  static bool configured[64] = {};
+  int dev = 0;
+  LORACT_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    LORACT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_pair_kernel<A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kPairStages * (kABytes + 16384) + 1024));
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;   // the two CTAs of a pair are neighbours along M
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  LORACT_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel<A_MN, B_MN>, maps, p));
+  count_launch();
+  return cudaGetLastError();
+}
+
+int g_pair_mode = 1;   // 0: never use the two-CTA kernel (test hook)
+
 }  // namespace
+
+void gemm_tc_set_pair_mode(int on) { g_pair_mode = on; }
 
 bool gemm_tc_supported(const GemmDesc& g) {
   if (g.a_type != ELEM_BF16 || g.b_type != ELEM_BF16) return false;
@@ -455,7 +652,10 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   p.kb_per_split = (p.kb_total + splits - 1) / splits;
   p.n_terms = g.n_terms;
   p.out = g.out; p.C0 = g.C0; p.C1 = g.C1; p.ldc = g.ldc; p.split_stride = g.split_stride;
-  p.b_bytes = g.b_mn ? (uint32_t)((p.bn + 63) / 64) * 8192u : (uint32_t)p.bn * 128u;
+  // Two CTAs per 256-row tile when there are at least 256 rows and the B tile splits into two legal halves.
+  const bool pair = g_pair_mode != 0 && g.M >= 2 * kBM && (g.b_mn ? p.bn % 128 == 0 : p.bn % 32 == 0);
+  const int b_rows = pair ? p.bn / 2 : p.bn;   // rows (or columns) of B one CTA loads per K block
+  p.b_bytes = g.b_mn ? (uint32_t)((b_rows + 63) / 64) * 8192u : (uint32_t)b_rows * 128u;
   p.tmem_cols = 32;
   while ((int)p.tmem_cols < p.bn) p.tmem_cols *= 2;
   p.accumulate = g.accumulate ? 1 : 0;
@@ -471,7 +671,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
     if (g.a_mn) LORACT_CUDA_TRY(get_tmap(g.terms[t].A, g.M, g.K, g.lda, 64, 64, &maps.a[t]));
     else LORACT_CUDA_TRY(get_tmap(g.terms[t].A, g.K, g.M, g.lda, 64, kBM, &maps.a[t]));
     if (g.b_mn) LORACT_CUDA_TRY(get_tmap(g.terms[t].B, g.N, g.K, g.ldb, 64, 64, &maps.b[t]));
-    else LORACT_CUDA_TRY(get_tmap(g.terms[t].B, g.K, g.N, g.ldb, 64, (uint32_t)p.bn, &maps.b[t]));
+    else LORACT_CUDA_TRY(get_tmap(g.terms[t].B, g.K, g.N, g.ldb, 64, (uint32_t)b_rows, &maps.b[t]));
   }
   for (int t = g.n_terms; t < 3; ++t) { maps.a[t] = maps.a[0]; maps.b[t] = maps.b[0]; }
   maps.wide = maps.a[0];
@@ -481,6 +681,15 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
       LORACT_CUDA_TRY(get_tmap(g.terms[0].B, g.K, g.N, g.ldb, 256, (uint32_t)p.bn, &maps.wide));
   }
 
+  if (pair) {
+    dim3 pgrid(2 * ((g.M + 2 * kBM - 1) / (2 * kBM)), (g.N + p.bn - 1) / p.bn, splits);
+    const size_t psmem = (size_t)kPairStages * (kABytes + p.b_bytes) + 1024;
+    p.prefetch = 0;
+    if (g.a_mn && g.b_mn) return launch_pair_variant<true, true>(maps, p, pgrid, psmem, stream);
+    if (g.a_mn && !g.b_mn) return launch_pair_variant<true, false>(maps, p, pgrid, psmem, stream);
+    if (!g.a_mn && g.b_mn) return launch_pair_variant<false, true>(maps, p, pgrid, psmem, stream);
+    return launch_pair_variant<false, false>(maps, p, pgrid, psmem, stream);
+  }
   dim3 grid((g.N + p.bn - 1) / p.bn, (g.M + kBM - 1) / kBM, splits);
   const size_t smem = (size_t)kStages * (kABytes + p.b_bytes) + 1024;
   if (g.a_mn && g.b_mn) return launch_variant<true, true>(maps, p, grid, smem, stream);

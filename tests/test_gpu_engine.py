@@ -1,0 +1,88 @@
+"""GPU tests of the tensor-core contraction behind Algorithm 1 lines 2 and 8, the Gram products and
+Reconstruct: C = sum_t A_t B_t with bf16 operands and fp32 accumulation, for every operand major, with
+ragged shapes, split-K partials and the bf16 hi/lo output -- in both forms of the kernel (one CTA per
+128-row tile, and a pair of CTAs per 256-row tile).  The reference is the definition, evaluated in float64
+on the same bf16 inputs."""
+import pytest
+import torch
+
+import __graft_entry__ as entry
+from paper_2509_23472_b200 import binding as B
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dev():
+    entry.build()
+    B.lib()
+    yield torch.device("cuda:0")
+    B.debug_set_pair_mode(True)
+
+
+def operands(M, N, K, a_mn, b_mn, n_terms, dev, seed):
+    g = torch.Generator(device=dev)
+    g.manual_seed(seed)
+    As = [torch.randn((K, M) if a_mn else (M, K), generator=g, device=dev).bfloat16() for _ in range(n_terms)]
+    Bs = [torch.randn((K, N) if b_mn else (N, K), generator=g, device=dev).bfloat16() for _ in range(n_terms)]
+    ref = torch.zeros(M, N, dtype=torch.float64, device=dev)
+    for a, b in zip(As, Bs):
+        a64 = a.double().t() if a_mn else a.double()
+        b64 = b.double() if b_mn else b.double().t()
+        ref += a64 @ b64
+    return As, Bs, ref
+
+
+SHAPES = [(256, 256, 512), (384, 128, 200), (1000, 96, 264), (512, 256, 64), (300, 64, 1032), (128, 256, 256),
+          (2048, 512, 320)]
+
+
+@pytest.mark.parametrize("pair", [False, True])
+@pytest.mark.parametrize("a_mn,b_mn", [(False, False), (True, True), (False, True), (True, False)])
+@pytest.mark.parametrize("M,N,K", SHAPES)
+def test_contraction_matches_the_definition(dev, pair, a_mn, b_mn, M, N, K):
+    # leading dimensions must be multiples of 8 elements
+    if (a_mn and M % 8) or (b_mn and N % 8) or K % 8:
+        pytest.skip("stride rule")
+    B.debug_set_pair_mode(pair)
+    As, Bs, ref = operands(M, N, K, a_mn, b_mn, 1, dev, seed=M + N + K)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    C = B.debug_gemm(As, Bs, M, N, K, a_mn, b_mn, out_mode=B.OUT_F32, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    scale = float(ref.abs().max())
+    assert float((C.double() - ref).abs().max()) <= 2e-5 * scale * max(1.0, (K / 64) ** 0.5)
+
+
+@pytest.mark.parametrize("pair", [False, True])
+def test_three_terms_split_k_and_pair_output(dev, pair):
+    B.debug_set_pair_mode(pair)
+    M, N, K = 256, 256, 4096
+    As, Bs, ref = operands(M, N, K, True, True, 3, dev, seed=11)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    P = B.debug_gemm(As, Bs, M, N, K, True, True, out_mode=B.OUT_F32, splits=8, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and P.shape == (8, M, N)
+    scale = float(ref.abs().max())
+    assert float((P.double().sum(0) - ref).abs().max()) <= 1e-4 * scale
+    # bf16 hi/lo output: hi + lo carries 16 bits of the fp32 result
+    M2, N2, K2 = 1024, 256, 256
+    As, Bs, ref = operands(M2, N2, K2, False, False, 3, dev, seed=12)
+    hi, lo = B.debug_gemm(As, Bs, M2, N2, K2, False, False, out_mode=B.OUT_SPLIT, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got = hi.double() + lo.double()
+    assert float((got - ref).abs().max()) <= 2.0 ** -15 * float(ref.abs().max()) + 1e-4 * float(ref.abs().max())
+
+
+def test_both_forms_agree_bit_for_bit_on_a_gram_product(dev):
+    # same products, same order of accumulation along K inside a tile: the two forms must agree exactly
+    M = N = 256
+    K = 2048
+    As, Bs, _ = operands(M, N, K, True, True, 1, dev, seed=5)
+    B.debug_set_pair_mode(False)
+    C1 = B.debug_gemm(As, Bs, M, N, K, True, True, out_mode=B.OUT_F32)
+    B.debug_set_pair_mode(True)
+    C2 = B.debug_gemm(As, Bs, M, N, K, True, True, out_mode=B.OUT_F32)
+    torch.cuda.synchronize()
+    assert float((C1 - C2).abs().max()) <= 1e-5 * float(C1.abs().max())
