@@ -239,6 +239,11 @@ def main():
     total_ms = sum(times)
     status = B.read_device_status(ws)
 
+    # ---- where the time goes: one more step with an event behind every kernel (outside the timed region)
+    B.debug_trace_begin(dev)
+    step(Xs[1], Gs[1])
+    stages = B.debug_trace_end(dev)
+
     # ---- end to end: inputs start in pinned host memory, the gradient is read back to the host
     Xh, Gh = X.cpu().pin_memory(), G.cpu().pin_memory()
     Xd2, Gd2 = torch.empty_like(X), torch.empty_like(G)
@@ -335,6 +340,7 @@ def main():
         "step_roofline_frac": step_floor_ms / ms_per_step,
         "ms_min": min(times), "ms_median": statistics.median(times),
         "ms_per_step_l2_flushed": sum(flushed) / len(flushed),
+        "stages_us": [[name, round(us, 1)] for name, us in stages],
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": X.numel() * es + G.numel() * es,
                 "d2h_bytes_per_step": dW.numel() * 4, "ms_per_step": e2e_ms / e2e_steps},
         "gpu_launches": int(launches), "device_status": status, "clocks": clocks,

@@ -32,6 +32,15 @@ loract_status_t loract_debug_gemm(int32_t M, int32_t N, int32_t K, int32_t a_mn,
  * that a test can compare the two; on = 1 (the default) restores the choice by shape.  Process-wide. */
 void loract_debug_set_pair_mode(int32_t on);
 
+/* Stage trace.  Between trace_begin and trace_end every kernel the library launches on `stream` is followed by
+ * a CUDA event; trace_end synchronises the stream and writes, per kernel in launch order, a label (64 bytes
+ * each, zero-terminated: the step of the path and the kernel's launch function) and the time from the
+ * previous event to this kernel's event in microseconds.  Returns the number of entries (at most max_entries),
+ * or -1.  The events keep neighbouring kernels from overlapping, so the sum is a little above the untraced
+ * time.  One trace at a time, from one host thread. */
+void loract_debug_trace_begin(void* stream);
+int32_t loract_debug_trace_end(void* stream, char* names, float* micros, int32_t max_entries);
+
 /* The cudaError_t behind the most recent LORACT_ERR_CUDA returned by any entry point (0 if none yet). */
 int32_t loract_debug_last_cuda_error(void);
 

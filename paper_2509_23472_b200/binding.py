@@ -268,7 +268,7 @@ def read_device_status(ws: torch.Tensor) -> int:
 # ---------------------------------------------------------------------------------------------
 OUT_F32, OUT_BF16, OUT_SPLIT, OUT_F64 = 0, 1, 2, 3
 DEBUG_EXPORTS = ("loract_debug_gemm", "loract_debug_small_block", "loract_debug_set_pair_mode",
-                 "loract_debug_last_cuda_error")
+                 "loract_debug_last_cuda_error", "loract_debug_trace_begin", "loract_debug_trace_end")
 
 
 def _debug_lib():
@@ -319,6 +319,26 @@ def debug_set_pair_mode(on: bool) -> None:
     l.loract_debug_set_pair_mode.restype = None
     l.loract_debug_set_pair_mode.argtypes = [ctypes.c_int32]
     l.loract_debug_set_pair_mode(1 if on else 0)
+
+
+def debug_trace_begin(device) -> None:
+    l = _debug_lib()
+    l.loract_debug_trace_begin.restype = None
+    l.loract_debug_trace_begin.argtypes = [ctypes.c_void_p]
+    l.loract_debug_trace_begin(_stream(device))
+
+
+def debug_trace_end(device, max_entries: int = 256):
+    """Returns [(label, microseconds), ...] for the kernels launched since debug_trace_begin."""
+    l = _debug_lib()
+    l.loract_debug_trace_end.restype = ctypes.c_int32
+    l.loract_debug_trace_end.argtypes = [ctypes.c_void_p, ctypes.c_char_p, ctypes.POINTER(ctypes.c_float), ctypes.c_int32]
+    names = ctypes.create_string_buffer(64 * max_entries)
+    us = (ctypes.c_float * max_entries)()
+    n = l.loract_debug_trace_end(_stream(device), names, us, max_entries)
+    if n < 0:
+        raise LoractError(5, "loract_debug_trace_end")
+    return [(names.raw[64 * i:64 * (i + 1)].split(b"\0", 1)[0].decode(), float(us[i])) for i in range(n)]
 
 
 def debug_small_block(partials: torch.Tensor, use_f64: bool, shift_rel: float,

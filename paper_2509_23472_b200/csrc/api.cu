@@ -2,6 +2,8 @@
 // of each entry point.  All arithmetic happens in the kernels of the other translation units.
 #include <atomic>
 #include <cstring>
+#include <string>
+#include <vector>
 
 #include "common.cuh"
 #include "../../include/loract_debug.h"
@@ -9,7 +11,32 @@
 namespace loract {
 
 static std::atomic<uint64_t> g_launches{0};
-void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+// ---- stage trace (test hook, one thread at a time): an event behind every launch while it is open
+static bool g_trace_open = false;
+static std::vector<cudaEvent_t> g_trace_events;
+static std::vector<std::string> g_trace_names;
+static size_t g_trace_used = 0;
+static const char* g_trace_label = "";
+
+static cudaEvent_t trace_event() {
+  if (g_trace_used == g_trace_events.size()) {
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+    g_trace_events.push_back(e);
+  }
+  return g_trace_events[g_trace_used++];
+}
+
+void trace_label(const char* label) { g_trace_label = label; }
+
+void count_launch(const char* kernel, cudaStream_t stream) {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (!g_trace_open) return;
+  cudaEvent_t e = trace_event();
+  if (!e) return;
+  cudaEventRecord(e, stream);
+  g_trace_names.push_back(std::string(g_trace_label) + " [" + kernel + "]");
+}
 
 namespace {
 
@@ -162,6 +189,7 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
     g.a_streams = true;
     g.ldc = l;
     if (p.bf16) { g.out = OUT_SPLIT; g.C0 = w.Yh; g.C1 = w.Yl; } else { g.out = OUT_F32; g.C0 = w.Y32; }
+    trace_label("pass 1: Y = X Omega^T");
     LORACT_CUDA_TRY(run_gemm(g, status, stream));
   }
   for (int round = 0; round < 2; ++round) {
@@ -180,8 +208,10 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
         g.terms[0] = {Yh, Yh};
         g.out = OUT_F64; g.C0 = w.gram64; g.acc64 = true;
       }
+      trace_label(round ? "Gram 2" : "Gram 1");
       LORACT_CUDA_TRY(run_gemm(g, status, stream));
     }
+    trace_label(round ? "small block 3" : "small block 2");
     LORACT_CUDA_TRY(factor(l, p.bf16, w.splits_gram, round ? kShiftSecond : kShiftFirst, w, status, stream));
     {  // Y <- Y L^{-T}:  C[m][j] = sum_k Y[m][k] Linv[j][k]
       GemmDesc g;
@@ -195,6 +225,7 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
         g.terms[0] = {Yh, w.Linv32};
         g.out = OUT_F32; g.C0 = round == 0 ? (void*)w.Q32 : U;
       }
+      trace_label(round ? "apply L^-T 2" : "apply L^-T 1");
       LORACT_CUDA_TRY(run_gemm(g, status, stream));
     }
   }
@@ -210,6 +241,7 @@ cudaError_t project(const void* U, const void* X, int64_t ldx, const Plan& p, vo
   g.terms[0] = {U, X};
   g.b_streams = true;
   g.ldc = p.d;
+  trace_label("pass 2: V = U^T X");
   if (!p.bf16) { g.out = OUT_F32; g.C0 = V; return run_gemm(g, status, stream); }
   if (w.splits_v <= 1) { g.out = OUT_BF16; g.C0 = V; return run_gemm(g, status, stream); }
   g.out = OUT_F32; g.C0 = w.v_partials; g.splits = w.splits_v; g.split_stride = (int64_t)p.l * p.d;
@@ -251,16 +283,20 @@ cudaError_t compress_core(const loract_desc_t* desc, const void* X, int64_t ldx,
   const int r = desc->rank;
   LORACT_CUDA_TRY(cudaMemsetAsync(w.status, 0, 4, stream));
   // line 1: sample rows, gather them
+  trace_label("sample");
   LORACT_CUDA_TRY(sample_indices_launch(desc->seed, desc->call_id, (uint32_t)desc->n_tokens, r, w.idx,
                                         w.status, stream));
   if (idx_out) LORACT_CUDA_TRY(cudaMemcpyAsync(idx_out, w.idx, (size_t)r * 4, cudaMemcpyDeviceToDevice, stream));
+  trace_label("gather");
   LORACT_CUDA_TRY(gather_rows_launch(X, ldx, w.idx, r, desc->d, elem_bytes(desc), w.S, stream));
   // Lines 2 to 7.  The test matrix (the sampled rows A_k at first, Q^T X in the power iterations of lines
   // 3 to 6) is preconditioned before every product with X: with T T^T = L L^T, Omega = L^{-1} T has the row
   // space of T, so range(X Omega^T) = range(X T^T), but its rows are close to orthonormal, which keeps the
   // spectrum of the sketch from being squared (and, in the iterations, raised to the fourth power).
   for (int it = 0; it <= desc->power_iters; ++it) {
+    trace_label("Gram of the test rows");
     LORACT_CUDA_TRY(gram_rows(w.S, r, desc->d, bf16, w.b, w.status, stream));
+    trace_label("small block 1");
     LORACT_CUDA_TRY(factor(r, bf16, w.b.splits_gram_sample, kShiftSample, w.b, w.status, stream));
     {
       GemmDesc g;
@@ -272,6 +308,7 @@ cudaError_t compress_core(const loract_desc_t* desc, const void* X, int64_t ldx,
       } else {
         g.terms[0] = {w.b.Linv32, w.S}; g.out = OUT_F32;
       }
+      trace_label("Omega = L^-1 T");
       LORACT_CUDA_TRY(run_gemm(g, w.status, stream));
     }
     // Y = X Omega^T, Y = QR (Q written to U)
@@ -417,6 +454,7 @@ loract_status_t loract_weight_grad(const loract_desc_t* desc, const void* U, con
   t.terms[0] = {U, G};
   t.out = OUT_F32; t.C0 = w.partials; t.ldc = g; t.splits = w.splits; t.split_stride = (int64_t)r * g;
   uint32_t* status = (uint32_t*)ws;
+  trace_label("weight grad");
   cudaError_t e = cudaMemsetAsync(status, 0, 4, st);
   if (e == cudaSuccess) e = run_gemm(t, status, st);
   if (e == cudaSuccess && el == ELEM_BF16) {
@@ -532,6 +570,29 @@ loract_status_t loract_debug_gemm(int32_t M, int32_t N, int32_t K, int32_t a_mn,
     return from_cuda(gemm_tc_launch(g, status_word, (cudaStream_t)stream));
   }
   return from_cuda(gemm_simt_launch(g, (cudaStream_t)stream));
+}
+
+void loract_debug_trace_begin(void* stream) {
+  g_trace_used = 0;
+  g_trace_names.clear();
+  g_trace_open = true;
+  trace_label("");
+  cudaEvent_t e = trace_event();
+  if (e) cudaEventRecord(e, (cudaStream_t)stream);
+}
+
+int32_t loract_debug_trace_end(void* stream, char* names, float* micros, int32_t max_entries) {
+  g_trace_open = false;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return -1;
+  int32_t n = 0;
+  for (size_t i = 0; i + 1 < g_trace_used && n < max_entries; ++i, ++n) {
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, g_trace_events[i], g_trace_events[i + 1]);
+    micros[n] = ms * 1000.f;
+    std::strncpy(names + (size_t)n * 64, g_trace_names[i].c_str(), 63);
+    names[(size_t)n * 64 + 63] = 0;
+  }
+  return n;
 }
 
 void loract_debug_set_pair_mode(int32_t on) { gemm_tc_set_pair_mode(on); }

@@ -10,7 +10,10 @@
 namespace loract {
 
 // ---------------------------------------------------------------- launch accounting
-void count_launch(int n = 1);
+// Called after every kernel launch: counts it and, while a trace is open (test hook), records an event
+// behind it on `stream` under the label set with trace_label().
+void count_launch(const char* kernel = "", cudaStream_t stream = nullptr);
+void trace_label(const char* label);
 
 #define LORACT_CUDA_TRY(expr)                          \
   do {                                                 \

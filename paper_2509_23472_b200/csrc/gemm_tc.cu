@@ -580,7 +580,7 @@ cudaError_t launch_variant(const TmapPack& maps, const TcParams& p, dim3 grid, s
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   LORACT_CUDA_TRY(launch_pdl(gemm_tc_kernel<A_MN, B_MN>, grid, dim3(kThreads), smem, stream, maps, p));
-  count_launch();
+  count_launch(__func__, stream);
   return cudaGetLastError();
 }
 
@@ -609,7 +609,7 @@ cudaError_t launch_pair_variant(const TmapPack& maps, const TcParams& p, dim3 gr
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   LORACT_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel<A_MN, B_MN>, maps, p));
-  count_launch();
+  count_launch(__func__, stream);
   return cudaGetLastError();
 }
 

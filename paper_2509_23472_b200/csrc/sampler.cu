@@ -139,7 +139,7 @@ cudaError_t sample_indices_launch(uint64_t seed, uint64_t call_id, uint32_t n_ro
   LORACT_CUDA_TRY(launch_pdl(sample_indices_kernel, dim3(1), dim3(kSamplerThreads), 0, stream, (uint32_t)seed,
                              (uint32_t)(seed >> 32), (uint32_t)call_id, (uint32_t)(call_id >> 32), n_rows, rank,
                              idx_dev, dev_status));
-  count_launch();
+  count_launch(__func__, stream);
   return cudaGetLastError();
 }
 
@@ -152,7 +152,7 @@ cudaError_t gather_rows_launch(const void* src, int64_t ld, const int32_t* idx, 
   if (gx > 64) gx = 64;
   LORACT_CUDA_TRY(launch_pdl(gather_rows_kernel, dim3(gx, rank), dim3(threads), 0, stream, (const uint4*)src, ld_vec,
                              idx, d_vec, (uint4*)dst));
-  count_launch();
+  count_launch(__func__, stream);
   return cudaGetLastError();
 }
 
@@ -164,7 +164,7 @@ cudaError_t gaussian_rows_launch(uint64_t seed, uint64_t call_id, int l, int64_t
   gaussian_rows_kernel<<<grid, 256, 0, stream>>>((uint32_t)seed, (uint32_t)(seed >> 32),
                                                  (uint32_t)call_id, (uint32_t)(call_id >> 32), l, d,
                                                  dst);
-  count_launch();
+  count_launch(__func__, stream);
   return cudaGetLastError();
 }
 

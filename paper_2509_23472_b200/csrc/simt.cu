@@ -194,7 +194,7 @@ cudaError_t launch_simt_typed(const SimtParams& p, bool acc64, cudaStream_t stre
   dim3 grid((p.N + kTile - 1) / kTile, (p.M + kTile - 1) / kTile, p.splits);
   if (acc64) gemm_simt_kernel<TA, TB, double><<<grid, 256, 0, stream>>>(p);
   else gemm_simt_kernel<TA, TB, float><<<grid, 256, 0, stream>>>(p);
-  count_launch();
+  count_launch(__func__, stream);
   return cudaGetLastError();
 }
 
@@ -228,7 +228,7 @@ cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_
   if (grid < 1) grid = 1;
   LORACT_CUDA_TRY(launch_pdl(reduce_partials_kernel, dim3(grid), dim3(256), 0, stream, partials, n_partials, stride,
                              count, out_f32, out_bf16));
-  count_launch();
+  count_launch(__func__, stream);
   return cudaGetLastError();
 }
 
@@ -240,7 +240,7 @@ cudaError_t reduce_split3_launch(const float* partials, int n_partials, int64_t 
   if (grid < 1) grid = 1;
   LORACT_CUDA_TRY(launch_pdl(reduce_split3_kernel, dim3(grid), dim3(256), 0, stream, partials, n_partials, stride, rows,
                              cols, ld_in, ld_out, hi, mid, lo));
-  count_launch();
+  count_launch(__func__, stream);
   return cudaGetLastError();
 }
 
@@ -257,7 +257,7 @@ cudaError_t norm_forward_launch(const void* X, int64_t n, int64_t d, int64_t ldx
     norm_forward_kernel<float><<<grid, warps * 32, 0, stream>>>(
         (const float*)X, n, d, ldx, (const float*)gamma, (const float*)beta, eps, kind, (float*)A, lda,
         rstd, mean);
-  count_launch();
+  count_launch(__func__, stream);
   return cudaGetLastError();
 }
 

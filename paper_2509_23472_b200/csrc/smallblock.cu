@@ -266,7 +266,7 @@ cudaError_t launch_typed(const SBParams& p, cudaStream_t stream) {
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   small_block_kernel<T><<<kCluster, kSBThreads, smem, stream>>>(p);
-  count_launch();
+  count_launch(__func__, stream);
   return cudaGetLastError();
 }
 
