@@ -110,6 +110,20 @@ loract_status_t loract_compress_prenorm(const loract_desc_t* desc, const void* X
                                         float* rstd, float* mean, void* U, void* V, int32_t* idx_out,
                                         void* ws, size_t ws_bytes, void* stream);
 
+/* Section 3.3, the backward pass of the pre-norm unit (RMS form) from the compressed normalised activation:
+ *   Xbar = A~ / gamma,  grad_Xbar = grad_A * gamma,
+ *   grad_X = rstd * (grad_Xbar - Xbar * (1/d) sum_j [grad_Xbar * Xbar]_j),        A~ = U V.
+ * (U, V) and rstd are those of loract_compress_prenorm (LORACT_NORM_RMS).  grad_A: device, n_tokens x d, row
+ * stride ldx, the gradient with respect to the sub-layer input A (all consumers already summed).  grad_X:
+ * device, n_tokens x d, row stride ldx, written.  A~ is never stored: the row means come from the factors
+ * ((1/d) U_i . (grad_A V^T)_i, since gamma cancels in the product) and the reconstructed tiles exist only
+ * inside the kernel that writes grad_X.  bf16 only (LORACT_ERR_UNSUPPORTED for fp32).  ws: at least
+ * loract_prenorm_backward_workspace_bytes(desc) bytes. */
+size_t loract_prenorm_backward_workspace_bytes(const loract_desc_t* desc);
+loract_status_t loract_prenorm_backward(const loract_desc_t* desc, const void* U, const void* V,
+                                        const void* gamma, const float* rstd, const void* grad_A,
+                                        void* grad_X, void* ws, size_t ws_bytes, void* stream);
+
 /* The same result as loract_weight_grad, for callers that cannot allocate device memory and so cannot
  * provide `ws`.  (The paper has no counterpart: this is a property of the library, not of the method.)
  * Typical callers: a backward hook running while the framework's caching allocator is locked or out of

@@ -21,7 +21,8 @@ DEV_PIVOT_CLAMPED, DEV_WAIT_EXPIRED, DEV_SAMPLER_SHORT, DEV_NONFINITE = 1, 2, 4,
 
 EXPORTS = (
     "loract_workspace_bytes", "loract_sample_indices", "loract_compress", "loract_reconstruct",
-    "loract_weight_grad", "loract_weight_grad_static", "loract_compress_prenorm", "loract_rsvd_workspace_bytes", "loract_rsvd",
+    "loract_weight_grad", "loract_weight_grad_static", "loract_compress_prenorm",
+    "loract_prenorm_backward_workspace_bytes", "loract_prenorm_backward", "loract_rsvd_workspace_bytes", "loract_rsvd",
     "loract_read_device_status", "loract_status_string", "loract_kernel_launch_count",
 )
 
@@ -71,6 +72,10 @@ def lib() -> ctypes.CDLL:
         l.loract_compress_prenorm.restype = ctypes.c_int
         l.loract_compress_prenorm.argtypes = [dp, vp, vp, vp, ctypes.c_float, i32, vp, vp, vp, vp, vp, vp,
                                               vp, sz, vp]
+        l.loract_prenorm_backward_workspace_bytes.restype = sz
+        l.loract_prenorm_backward_workspace_bytes.argtypes = [dp]
+        l.loract_prenorm_backward.restype = ctypes.c_int
+        l.loract_prenorm_backward.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         l.loract_rsvd_workspace_bytes.restype = sz
         l.loract_rsvd_workspace_bytes.argtypes = [dp, i32]
         l.loract_rsvd.restype = ctypes.c_int
@@ -236,6 +241,27 @@ def compress_prenorm(X: torch.Tensor, gamma: torch.Tensor, beta: Optional[torch.
                                          _ptr(rstd), _ptr(mean), _ptr(U), _ptr(V), _ptr(idx), _ptr(ws),
                                          ws.numel(), _stream(X.device)), "loract_compress_prenorm")
     return A, rstd, mean, U, V, idx
+
+
+def prenorm_backward(U: torch.Tensor, V: torch.Tensor, gamma: torch.Tensor, rstd: torch.Tensor,
+                     grad_A: torch.Tensor, ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """grad_X of the RMS pre-norm unit from the compressed normalised activation (Section 3.3)."""
+    for t, what in ((U, "U"), (V, "V"), (gamma, "gamma"), (rstd, "rstd"), (grad_A, "grad_A")):
+        _cuda(t, what)
+    n, r = U.shape
+    d = V.shape[1]
+    if grad_A.shape != (n, d) or grad_A.stride(1) != 1:
+        raise ValueError("grad_A must be a row-major (n_tokens x d) tensor")
+    desc = Desc(n, d, grad_A.stride(0), r, 0, _dtype_code(U), 0, 0, 0)
+    need = int(lib().loract_prenorm_backward_workspace_bytes(ctypes.byref(desc)))
+    if need == 0:
+        raise LoractError(1, "loract_prenorm_backward_workspace_bytes")
+    ws = ws if ws is not None else torch.empty(need, dtype=torch.uint8, device=U.device)
+    grad_X = torch.empty_like(grad_A)
+    _check(lib().loract_prenorm_backward(ctypes.byref(desc), _ptr(U), _ptr(V), _ptr(gamma), _ptr(rstd), _ptr(grad_A),
+                                         _ptr(grad_X), _ptr(ws), ws.numel(), _stream(U.device)),
+           "loract_prenorm_backward")
+    return grad_X
 
 
 def rsvd(X: torch.Tensor, rank: int, oversample: int = 8, power_iters: int = 1, seed: int = 0, call_id: int = 0,

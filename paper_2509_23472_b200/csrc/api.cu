@@ -481,6 +481,63 @@ loract_status_t loract_weight_grad(const loract_desc_t* desc, const void* U, con
   return from_cuda(e);
 }
 
+size_t loract_prenorm_backward_workspace_bytes(const loract_desc_t* desc) {
+  if (check_desc(desc) != LORACT_OK) return 0;
+  Carver c(nullptr);
+  c.take(256);
+  c.take((size_t)desc->n_tokens * desc->rank * 4);   // P = grad_A V^T
+  c.take((size_t)desc->n_tokens * 4);                // row_a
+  c.take((size_t)desc->n_tokens * 4);                // row_b
+  return c.off;
+}
+
+loract_status_t loract_prenorm_backward(const loract_desc_t* desc, const void* U, const void* V, const void* gamma,
+                                        const float* rstd, const void* grad_A, void* grad_X, void* ws,
+                                        size_t ws_bytes, void* stream) {
+  loract_status_t s = check_desc(desc);
+  if (s != LORACT_OK) return s;
+  if (desc->dtype != LORACT_BF16) return LORACT_ERR_UNSUPPORTED;
+  if (!U || !V || !gamma || !rstd || !grad_A || !grad_X || !ws) return LORACT_ERR_INVALID_ARG;
+  if (misaligned(U) || misaligned(V) || misaligned(gamma) || misaligned(grad_A) || misaligned(grad_X) ||
+      ((uintptr_t)ws & 255))
+    return LORACT_ERR_ALIGNMENT;
+  if (ws_bytes < loract_prenorm_backward_workspace_bytes(desc)) return LORACT_ERR_WORKSPACE_TOO_SMALL;
+  const int n = (int)desc->n_tokens, d = (int)desc->d, r = desc->rank;
+  Carver c(ws);
+  uint32_t* status = (uint32_t*)c.take(256);
+  float* P = (float*)c.take((size_t)n * r * 4);
+  float* row_a = (float*)c.take((size_t)n * 4);
+  float* row_b = (float*)c.take((size_t)n * 4);
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMemsetAsync(status, 0, 4, st);
+  // With A~ = U V: (grad_Xbar . Xbar)_ij = grad_A_ij A~_ij (gamma cancels), so the row mean of Section 3.3 is
+  // (1 / d) U_i . (grad_A V^T)_i -- a tall-skinny product instead of a pass over a reconstructed matrix.
+  if (e == cudaSuccess) {
+    GemmDesc g;
+    g.M = n; g.N = r; g.K = d; g.lda = desc->ldx; g.ldb = d;
+    g.terms[0] = {grad_A, V};
+    g.a_streams = true;
+    g.out = OUT_F32; g.C0 = P; g.ldc = r;
+    trace_label("pre-norm backward: P = grad_A V^T");
+    e = gemm_tc_supported(g) ? gemm_tc_launch(g, status, st) : cudaErrorNotSupported;
+  }
+  if (e == cudaSuccess) {
+    trace_label("pre-norm backward: row coefficients");
+    e = rms_backward_rows_launch((const __nv_bfloat16*)U, P, rstd, n, r, d, row_a, row_b, st);
+  }
+  if (e == cudaSuccess) {
+    // grad_X = rstd * (grad_A * gamma - (A~ / gamma) * inner), A~ tile by tile in tensor memory only
+    GemmDesc g;
+    g.M = n; g.N = d; g.K = r; g.b_mn = true; g.lda = r; g.ldb = d;
+    g.terms[0] = {U, V};
+    g.out = OUT_RMS_BWD; g.C0 = grad_X; g.ldc = desc->ldx;
+    g.ep_E = grad_A; g.ep_ld = desc->ldx; g.ep_row_a = row_a; g.ep_row_b = row_b; g.ep_col = gamma;
+    trace_label("pre-norm backward: grad_X");
+    e = gemm_tc_supported(g) ? gemm_tc_launch(g, status, st) : cudaErrorNotSupported;
+  }
+  return from_cuda(e);
+}
+
 size_t loract_rsvd_workspace_bytes(const loract_desc_t* desc, int32_t oversample) {
   if (check_desc(desc) != LORACT_OK || desc->dtype != LORACT_BF16) return 0;
   const int l = desc->rank + oversample;

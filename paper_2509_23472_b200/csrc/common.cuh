@@ -57,7 +57,10 @@ enum OutMode : int {
   OUT_F32 = 0,    // C0: float
   OUT_BF16 = 1,   // C0: bf16
   OUT_SPLIT = 2,  // C0: bf16 hi, C1: bf16 lo  (hi = bf16(x), lo = bf16(x - hi))
-  OUT_F64 = 3     // C0: double (SIMT path only)
+  OUT_F64 = 3,    // C0: double (SIMT path only)
+  // C0: bf16, C0[m][n] = row_a[m] * col[n] * E[m][n] - row_b[m] / col[n] * acc[m][n]  (tensor-core path only):
+  // the input gradient of the RMS pre-norm unit from a reconstructed tile that is never stored
+  OUT_RMS_BWD = 4
 };
 
 enum ElemType : int { ELEM_F32 = 0, ELEM_BF16 = 1, ELEM_F64 = 2 };
@@ -84,6 +87,12 @@ struct GemmDesc {
   bool acc64 = false;      // SIMT path: accumulate in double
   bool accumulate = false; // SIMT path, OUT_F32, splits == 1: C += result
   float alpha = 1.0f;      // SIMT path: C = alpha * sum
+  // OUT_RMS_BWD: E (bf16, M x N, leading dimension ep_ld), per-row and per-column coefficients
+  const void* ep_E = nullptr;
+  int64_t ep_ld = 0;
+  const float* ep_row_a = nullptr;
+  const float* ep_row_b = nullptr;
+  const void* ep_col = nullptr;
   // tensor-core path: the operand is large and read once from HBM (the activation matrix): prefetch it
   bool a_streams = false, b_streams = false;
 };
@@ -145,6 +154,10 @@ cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_
 cudaError_t reduce_split3_launch(const float* partials, int n_partials, int64_t stride, int rows, int cols,
                                  int64_t ld_in, int64_t ld_out, __nv_bfloat16* hi, __nv_bfloat16* mid,
                                  __nv_bfloat16* lo, cudaStream_t stream);
+// Section 3.3 backward, row coefficients: inner_i = (1 / d) sum_k U[i][k] P[i][k] (P = grad_A V^T, fp32, n x r),
+// row_a[i] = rstd[i], row_b[i] = rstd[i] * inner_i.  One warp per row.
+cudaError_t rms_backward_rows_launch(const __nv_bfloat16* U, const float* P, const float* rstd, int64_t n, int r,
+                                     int64_t d, float* row_a, float* row_b, cudaStream_t stream);
 // Section 3.3 forward: A = Norm(X); per-row rstd (and mean for LayerNorm).  One warp per row.
 cudaError_t norm_forward_launch(const void* X, int64_t n, int64_t d, int64_t ldx, int elem_type,
                                 const void* gamma, const void* beta, float eps, int kind, void* A,

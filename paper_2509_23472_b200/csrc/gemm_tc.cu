@@ -51,6 +51,11 @@ struct TcParams {
   uint32_t b_bytes;   // bytes of one B stage
   uint32_t tmem_cols;
   int accumulate;     // OUT_F32, one split: C += result
+  const void* ep_E;   // OUT_RMS_BWD epilogue operands
+  int64_t ep_ld;
+  const float* ep_row_a;
+  const float* ep_row_b;
+  const void* ep_col;
   int prefetch;       // bit 0: operand A streams from HBM, bit 1: operand B does -- prefetch it into L2 ahead
   uint32_t* dev_status;
 };
@@ -181,6 +186,36 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, uint32_t tmem_bas
             reinterpret_cast<uint4*>(dst)[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
         } else {
           for (int q = 0; q < valid; ++q) dst[q] = __uint_as_float(v[q]);
+        }
+      } else if (p.out == OUT_RMS_BWD) {
+        // grad_X = rstd * (grad_A * gamma - (reconstructed A / gamma) * inner): the tile of the reconstructed
+        // activation exists only in tensor memory and in these registers
+        __nv_bfloat16* dst = (__nv_bfloat16*)p.C0 + (int64_t)m * p.ldc + n;
+        const __nv_bfloat16* e = (const __nv_bfloat16*)p.ep_E + (int64_t)m * p.ep_ld + n;
+        const __nv_bfloat16* col = (const __nv_bfloat16*)p.ep_col + n;
+        const float ra = p.ep_row_a[m], rb = p.ep_row_b[m];
+        if (valid == 32 && ((((uintptr_t)dst) & 15) == 0) && ((((uintptr_t)e) & 15) == 0) &&
+            ((((uintptr_t)col) & 15) == 0)) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint4 ev = reinterpret_cast<const uint4*>(e)[q];
+            const uint4 cv = __ldg(reinterpret_cast<const uint4*>(col) + q);
+            const uint32_t ew[4] = {ev.x, ev.y, ev.z, ev.w}, cw[4] = {cv.x, cv.y, cv.z, cv.w};
+            uint32_t ow[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              const float e0 = __uint_as_float(ew[h] << 16), e1 = __uint_as_float(ew[h] & 0xffff0000u);
+              const float c0f = __uint_as_float(cw[h] << 16), c1f = __uint_as_float(cw[h] & 0xffff0000u);
+              const float a0 = __uint_as_float(v[8 * q + 2 * h]), a1 = __uint_as_float(v[8 * q + 2 * h + 1]);
+              ow[h] = pack_bf16x2(ra * c0f * e0 - rb * a0 / c0f, ra * c1f * e1 - rb * a1 / c1f);
+            }
+            reinterpret_cast<uint4*>(dst)[q] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+          }
+        } else {
+          for (int q = 0; q < valid; ++q) {
+            const float c = __bfloat162float(col[q]);
+            dst[q] = __float2bfloat16(ra * c * __bfloat162float(e[q]) - rb * __uint_as_float(v[q]) / c);
+          }
         }
       } else {
         __nv_bfloat16* dst_hi = (__nv_bfloat16*)p.C0 + (int64_t)m * p.ldc + n;
@@ -621,7 +656,8 @@ void gemm_tc_set_pair_mode(int on) { g_pair_mode = on; }
 
 bool gemm_tc_supported(const GemmDesc& g) {
   if (g.a_type != ELEM_BF16 || g.b_type != ELEM_BF16) return false;
-  if (!(g.out == OUT_F32 || g.out == OUT_BF16 || g.out == OUT_SPLIT)) return false;
+  if (!(g.out == OUT_F32 || g.out == OUT_BF16 || g.out == OUT_SPLIT || g.out == OUT_RMS_BWD)) return false;
+  if (g.out == OUT_RMS_BWD && (!g.ep_E || !g.ep_row_a || !g.ep_row_b || !g.ep_col || g.splits > 1)) return false;
   if (g.M < 1 || g.N < 1 || g.K < 1 || g.n_terms < 1 || g.n_terms > 3) return false;
   if (g.lda % 8 || g.ldb % 8) return false;
   if (g.splits > 1 && g.out != OUT_F32) return false;
@@ -659,6 +695,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   p.tmem_cols = 32;
   while ((int)p.tmem_cols < p.bn) p.tmem_cols *= 2;
   p.accumulate = g.accumulate ? 1 : 0;
+  p.ep_E = g.ep_E; p.ep_ld = g.ep_ld; p.ep_row_a = g.ep_row_a; p.ep_row_b = g.ep_row_b; p.ep_col = g.ep_col;
   // an operand too large to have stayed in L2 (tens of MB) streams from HBM even if the caller did not say so
   const size_t stream_bytes = (size_t)32 << 20;
   const bool a_big = (size_t)g.M * g.K * 2 >= stream_bytes, b_big = (size_t)g.N * g.K * 2 >= stream_bytes;

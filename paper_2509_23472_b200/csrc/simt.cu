@@ -148,6 +148,28 @@ __global__ void reduce_split3_kernel(const float* __restrict__ partials, int n_p
   }
 }
 
+// One warp per row: inner = (1 / d) sum_k U[i][k] P[i][k];  row_a = rstd, row_b = rstd * inner.
+__global__ void __launch_bounds__(256) rms_backward_rows_kernel(const __nv_bfloat16* __restrict__ U,
+                                                                const float* __restrict__ P,
+                                                                const float* __restrict__ rstd, int64_t n, int r,
+                                                                float inv_d, float* __restrict__ row_a,
+                                                                float* __restrict__ row_b) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= n) return;
+  float s = 0.f;
+  for (int k = lane; k < r; k += 32) s += __bfloat162float(U[row * r + k]) * P[row * r + k];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if (lane == 0) {
+    const float rs = rstd[row];
+    row_a[row] = rs;
+    row_b[row] = rs * s * inv_d;
+  }
+}
+
 // One warp per row.  RMS: rstd = 1/sqrt(mean x^2 + eps).  LayerNorm: mean first, then the centred
 // second moment (two passes over the row, which stays in L1/L2), A = (x - mean) rstd gamma + beta.
 template <typename T>
@@ -240,6 +262,16 @@ cudaError_t reduce_split3_launch(const float* partials, int n_partials, int64_t 
   if (grid < 1) grid = 1;
   LORACT_CUDA_TRY(launch_pdl(reduce_split3_kernel, dim3(grid), dim3(256), 0, stream, partials, n_partials, stride, rows,
                              cols, ld_in, ld_out, hi, mid, lo));
+  count_launch(__func__, stream);
+  return cudaGetLastError();
+}
+
+cudaError_t rms_backward_rows_launch(const __nv_bfloat16* U, const float* P, const float* rstd, int64_t n, int r,
+                                     int64_t d, float* row_a, float* row_b, cudaStream_t stream) {
+  const int warps = 8;
+  const int grid = (int)((n + warps - 1) / warps);
+  LORACT_CUDA_TRY(launch_pdl(rms_backward_rows_kernel, dim3(grid), dim3(warps * 32), 0, stream, U, P, rstd, n, r,
+                             1.0f / (float)d, row_a, row_b));
   count_launch(__func__, stream);
   return cudaGetLastError();
 }

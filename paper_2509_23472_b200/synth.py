@@ -153,3 +153,20 @@ def exact_low_rank(n: int, d: int, inner: int, seed: int, device="cpu") -> torch
     B = torch.randn(n, inner, generator=gen, device=device, dtype=torch.float64)
     C = torch.randn(inner, d, generator=gen, device=device, dtype=torch.float64)
     return B @ C / math.sqrt(inner)
+
+
+def plant_private_outliers(X: torch.Tensor, n_out: int, scale: float, seed: int) -> torch.Tensor:
+    """A coherent variant of an input: `n_out` feature columns are cleared everywhere and each is given one
+    entry of size scale * (RMS of X) in a token row of its own.  These rank-one components live on single
+    rows, so a uniform row sample that misses those rows cannot see them (the regime where the paper's
+    coherence term bites); the rest of X is unchanged.  Rows and columns are drawn from `seed`."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed)
+    n, d = X.shape
+    rows = torch.randperm(n, generator=gen)[:n_out].to(X.device)
+    cols = torch.randperm(d, generator=gen)[:n_out].to(X.device)
+    rms = float(X.float().pow(2).mean().sqrt())
+    Y = X.clone()
+    Y[:, cols] = 0
+    Y[rows, cols] = torch.tensor(scale * rms, dtype=X.dtype, device=X.device)
+    return Y

@@ -234,3 +234,48 @@ def test_power_iterations_fp32(dev):
     assert np.array_equal(idx.cpu().numpy().astype(np.int64), io)
     assert abs(gpu_err(X.double(), U, V) - orc.rel_fro_error(Xd, Uo, Vo)) <= TOL_ERR["f32"]
     assert orth_defect(U) <= TOL_ORTH
+
+
+# ------------------------------------------------------------------ coherent inputs
+def test_private_outlier_tokens_need_one_power_iteration(dev):
+    """A few token rows carry large components nobody else has (high coherence).  Uniform row sampling at
+    t = 0 misses them on both sides; one pass of the loop of Algorithm 1 (t = 1) recovers them, on both sides."""
+    w = synth.scaled(synth.get_workload("llama13b_s1024_r64"), n_tokens=2048, d=1024, rank=64, signal_rank=48)
+    X = synth.plant_private_outliers(synth.make_inputs(w, device=dev)["X"], n_out=8, scale=400.0, seed=123)
+    X64, Xd = X.double(), to64(X)
+    got = {}
+    for t in (0, 1):
+        U, V, idx = B.compress(X, 64, seed=w.seed, power_iters=t)
+        torch.cuda.synchronize()
+        Uo, Vo, io = orc.decompose(Xd, 64, t=t, seed=w.seed)
+        assert np.array_equal(idx.cpu().numpy().astype(np.int64), io)
+        got[t] = (gpu_err(X64, U, V), orc.rel_fro_error(Xd, Uo, Vo))
+        assert abs(got[t][0] - got[t][1]) <= TOL_ERR["bf16"], (t, got[t])
+        assert orth_defect(U) <= orth_bound(U, spiky=True)   # t = 1: basis vectors sit on single rows
+    assert got[0][1] > 0.5 and got[0][0] > 0.5          # the sample cannot see the private components
+    assert got[1][1] < 0.1 and got[1][0] < 0.1 + TOL_ERR["bf16"]   # one iteration finds them
+
+
+# ------------------------------------------------------------------ pre-norm unit, backward (Section 3.3)
+@pytest.mark.parametrize("n,d,r", [(1024, 512, 64), (1000, 768, 96), (4096, 1024, 256)])
+def test_prenorm_backward_matches_the_three_gradient_equations(dev, n, d, r):
+    w = synth.scaled(synth.WORKLOADS["llama7b_block"], n_tokens=n, d=d, rank=r, signal_rank=min(2 * r, d // 2))
+    w = synth.Workload(**{**w.__dict__, "prenorm": "rms"})
+    inp = synth.make_inputs(w, device=dev)
+    X, gamma = inp["X"], inp["gamma"]
+    A, rstd, _, U, V, idx = B.compress_prenorm(X, gamma, None, 1e-6, B.NORM_RMS, r, seed=w.seed)
+    g = torch.Generator(device=dev)
+    g.manual_seed(77)
+    gA = torch.randn(n, d, generator=g, device=dev).to(X.dtype)
+    gX = B.prenorm_backward(U, V, gamma, rstd, gA)
+    torch.cuda.synchronize()
+    # the oracle's equations on the same stored factors: this isolates the backward step
+    A_tilde = to64(U) @ to64(V)
+    want = orc.prenorm_backward_rms(A_tilde, to64(gamma), to64(rstd), to64(gA))
+    rel = np.linalg.norm(to64(gX) - want) / np.linalg.norm(want)
+    assert rel <= 1e-2, rel                     # bf16 output: 2^-9 per entry
+    # and against the exact (uncompressed) gradient the difference is the compression error, not more
+    exact = orc.prenorm_backward_rms(to64(A), to64(gamma), to64(rstd), to64(gA))
+    err_A = np.linalg.norm(A_tilde - to64(A)) / np.linalg.norm(to64(A))
+    rel_exact = np.linalg.norm(to64(gX) - exact) / np.linalg.norm(exact)
+    assert rel_exact <= 2.0 * err_A + 1e-2, (rel_exact, err_A)
