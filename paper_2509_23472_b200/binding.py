@@ -373,7 +373,8 @@ def debug_small_block(partials: torch.Tensor, use_f64: bool, shift_rel: float,
     l = _debug_lib()
     dev = partials.device
     n_p, r, _ = partials.shape
-    scratch = torch.empty(2 * (r * r + 32 * r), dtype=torch.float64 if use_f64 else torch.float32, device=dev)
+    scratch = torch.empty(2 * r * r + 2 * 256 * 256 + 64 * r, dtype=torch.float64 if use_f64 else torch.float32,
+                          device=dev)
     L32 = torch.zeros(r, r, dtype=torch.float32, device=dev)
     Lh = torch.zeros(r, r, dtype=torch.bfloat16, device=dev)
     Ll = torch.zeros(r, r, dtype=torch.bfloat16, device=dev)

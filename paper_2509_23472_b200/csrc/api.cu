@@ -117,7 +117,9 @@ void carve_basis(Carver& c, const Plan& p, BasisWs* w) {
   if (p.bf16) {
     w->Lh = (__nv_bfloat16*)c.take(l * l * 2);
     w->Ll = (__nv_bfloat16*)c.take(l * l * 2);
-    w->sb_scratch = c.take((l * l + (l + 31) / 32 * 1024) * sizeof(float));
+    // r <= 256 needs none (shared-memory kernel); above that the two-level scheme keeps W, X and two 256 x 256
+    // temporaries here
+    w->sb_scratch = c.take((2 * l * l + 2 * 256 * 256) * sizeof(float));
     const size_t gs = (size_t)(p.splits_gs > p.splits_w ? p.splits_gs : p.splits_w);
     w->gram_partials = (float*)c.take(gs * l * l * 4);
     w->Yh = (__nv_bfloat16*)c.take(n * l * 2);

@@ -138,6 +138,9 @@ struct SmallBlockArgs {
   __nv_bfloat16* linv_hi = nullptr;
   __nv_bfloat16* linv_lo = nullptr;
   uint32_t* dev_status = nullptr;
+  // row strides (elements) of the partial matrices and of the outputs; 0 means r.  The matrix may be a
+  // diagonal sub-block of a larger one (the r > 256 path factors a 512 x 512 matrix through its 256 x 256 blocks)
+  int64_t in_ld = 0, out_ld = 0;
 };
 cudaError_t small_block_launch(const SmallBlockArgs& a, cudaStream_t stream);
 // The same computation for r <= 256 in fp32 from fp32 partials, entirely in the shared memory of a
@@ -147,6 +150,10 @@ cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t str
 
 // ---------------------------------------------------------------- elementwise helpers
 // out = sum_s partials[s] (fixed order), written as fp32 and/or bf16.
+// X21 of a 2 x 2 block lower-triangular inverse as bf16 hi/lo (and optionally fp32), plus zeros in the block
+// above the diagonal: src (rows x cols fp32, leading dimension ld) -> hi/lo at the same place.
+cudaError_t split_block_launch(const float* src, int rows, int cols, int64_t ld, __nv_bfloat16* hi,
+                               __nv_bfloat16* lo, cudaStream_t stream);
 cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_t stride,
                                    int64_t count, float* out_f32, __nv_bfloat16* out_bf16,
                                    cudaStream_t stream);

@@ -148,6 +148,19 @@ __global__ void reduce_split3_kernel(const float* __restrict__ partials, int n_p
   }
 }
 
+// hi/lo split of a block of an fp32 matrix, in place of the same block of two bf16 matrices.
+__global__ void split_block_kernel(const float* __restrict__ src, int rows, int cols, int64_t ld,
+                                   __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < (int64_t)rows * cols;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t row = i / cols, col = i - row * cols;
+    const float v = src[row * ld + col];
+    const __nv_bfloat16 h = __float2bfloat16(v);
+    hi[row * ld + col] = h;
+    if (lo) lo[row * ld + col] = __float2bfloat16(v - __bfloat162float(h));
+  }
+}
+
 // One warp per row: inner = (1 / d) sum_k U[i][k] P[i][k];  row_a = rstd, row_b = rstd * inner.
 __global__ void __launch_bounds__(256) rms_backward_rows_kernel(const __nv_bfloat16* __restrict__ U,
                                                                 const float* __restrict__ P,
@@ -262,6 +275,15 @@ cudaError_t reduce_split3_launch(const float* partials, int n_partials, int64_t 
   if (grid < 1) grid = 1;
   LORACT_CUDA_TRY(launch_pdl(reduce_split3_kernel, dim3(grid), dim3(256), 0, stream, partials, n_partials, stride, rows,
                              cols, ld_in, ld_out, hi, mid, lo));
+  count_launch(__func__, stream);
+  return cudaGetLastError();
+}
+
+cudaError_t split_block_launch(const float* src, int rows, int cols, int64_t ld, __nv_bfloat16* hi,
+                               __nv_bfloat16* lo, cudaStream_t stream) {
+  int grid = (int)(((int64_t)rows * cols + 255) / 256);
+  if (grid > 148 * 4) grid = 148 * 4;
+  split_block_kernel<<<grid, 256, 0, stream>>>(src, rows, cols, ld, hi, lo);
   count_launch(__func__, stream);
   return cudaGetLastError();
 }

@@ -272,8 +272,61 @@ cudaError_t launch_typed(const SBParams& p, cudaStream_t stream) {
 
 }  // namespace
 
+// 256 < r <= 512 in fp32: the matrix as 2 x 2 blocks, W = [W11 . ; W21 W22], the leading block 256 wide.
+//   L11 = chol(W11), X11 = L11^-1            (shared-memory cluster kernel)
+//   L21 = W21 X11^T,  S = W22 - L21 L21^T    (fp32 CUDA-core products)
+//   L22 = chol(S), X22 = L22^-1              (shared-memory cluster kernel)
+//   X21 = -X22 (L21 X11)                     (fp32 CUDA-core products)
+// scratch: W (r x r) + X (r x r) + two 256 x 256 temporaries, fp32.
+cudaError_t small_block_two_level(const SmallBlockArgs& a, cudaStream_t stream) {
+  const int r = a.r, r1 = 256, r2 = r - r1;
+  float* W = (float*)a.scratch;
+  float* X = a.linv_f32 ? a.linv_f32 : W + (size_t)r * r;
+  float* T1 = W + 2 * (size_t)r * r;
+  float* T2 = T1 + (size_t)r1 * r1;
+  LORACT_CUDA_TRY(reduce_partials_launch((const float*)a.partials, a.n_partials, a.partial_stride, (int64_t)r * r, W,
+                                         nullptr, stream));
+  if (a.linv_f32) LORACT_CUDA_TRY(cudaMemsetAsync(X, 0, (size_t)r * r * 4, stream));
+  LORACT_CUDA_TRY(cudaMemsetAsync(a.linv_hi, 0, (size_t)r * r * 2, stream));   // the block above the diagonal
+  if (a.linv_lo) LORACT_CUDA_TRY(cudaMemsetAsync(a.linv_lo, 0, (size_t)r * r * 2, stream));
+  SmallBlockArgs s1 = a;
+  s1.r = r1; s1.partials = W; s1.n_partials = 1; s1.partial_stride = 0; s1.in_ld = r; s1.out_ld = r;
+  s1.linv_f32 = X; s1.scratch = nullptr;
+  LORACT_CUDA_TRY(small_block_cluster_launch(s1, stream));
+  auto simt = [&](int M, int N, int K, const float* A, int64_t lda, const float* B, int64_t ldb, bool b_mn, float* C,
+                  int64_t ldc, float alpha, bool accumulate) {
+    GemmDesc g;
+    g.M = M; g.N = N; g.K = K; g.lda = lda; g.ldb = ldb; g.b_mn = b_mn;
+    g.a_type = g.b_type = ELEM_F32;
+    g.terms[0] = {A, B};
+    g.out = OUT_F32; g.C0 = C; g.ldc = ldc; g.alpha = alpha; g.accumulate = accumulate;
+    return gemm_simt_launch(g, stream);
+  };
+  const float* W21 = W + (size_t)r1 * r;
+  float* W22 = W + (size_t)r1 * r + r1;
+  // L21 = W21 X11^T : C[m][n] = sum_k W21[m][k] X11[n][k]
+  LORACT_CUDA_TRY(simt(r2, r1, r1, W21, r, X, r, false, T1, r1, 1.f, false));
+  // S = W22 - L21 L21^T, in place
+  LORACT_CUDA_TRY(simt(r2, r2, r1, T1, r1, T1, r1, false, W22, r, -1.f, true));
+  SmallBlockArgs s2 = s1;
+  s2.r = r2; s2.partials = W22; s2.linv_f32 = X + (size_t)r1 * r + r1;
+  s2.linv_hi = a.linv_hi + (size_t)r1 * r + r1;
+  s2.linv_lo = a.linv_lo ? a.linv_lo + (size_t)r1 * r + r1 : nullptr;
+  LORACT_CUDA_TRY(small_block_cluster_launch(s2, stream));
+  // X21 = -X22 (L21 X11): T2[m][n] = sum_k L21[m][k] X11[k][n];  X21[m][n] = -sum_k X22[m][k] T2[k][n]
+  LORACT_CUDA_TRY(simt(r2, r1, r1, T1, r1, X, r, true, T2, r1, 1.f, false));
+  float* X21 = X + (size_t)r1 * r;
+  LORACT_CUDA_TRY(simt(r2, r1, r2, X + (size_t)r1 * r + r1, r, T2, r1, true, X21, r, -1.f, false));
+  return split_block_launch(X21, r2, r1, r, a.linv_hi + (size_t)r1 * r, a.linv_lo ? a.linv_lo + (size_t)r1 * r : nullptr,
+                            stream);
+}
+
 cudaError_t small_block_launch(const SmallBlockArgs& a, cudaStream_t stream) {
   if (small_block_cluster_supported(a)) return small_block_cluster_launch(a, stream);
+  if (!a.use_f64 && a.partial_type == ELEM_F32 && a.r > 256 && a.r <= 512 && a.r % 16 == 0 && !a.linv_full &&
+      a.linv_hi && a.in_ld == 0 && a.out_ld == 0 && (((uintptr_t)a.partials & 15) == 0) &&
+      (a.partial_stride % 4 == 0))
+    return small_block_two_level(a, stream);
   SBParams p;
   p.r = a.r;
   p.partials = a.partials;

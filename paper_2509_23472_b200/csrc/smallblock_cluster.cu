@@ -52,6 +52,7 @@ struct SCParams {
   __nv_bfloat16* linv_hi;
   __nv_bfloat16* linv_lo;
   uint32_t* dev_status;
+  int64_t in_ld, out_ld;   // row strides of the partial matrices and of the outputs
 };
 
 __device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }
@@ -435,7 +436,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
     float t = 0.f;
     for (int i = tid; i < r; i += kCThreads) {
       float d = 0.f;
-      for (int q = 0; q < p.n_partials; ++q) d += __ldg(p.partials + (int64_t)q * p.partial_stride + (int64_t)i * r + i);
+      for (int q = 0; q < p.n_partials; ++q) d += __ldg(p.partials + (int64_t)q * p.partial_stride + (int64_t)i * p.in_ld + i);
       t += d;
     }
     constexpr int kMaxMine = (kMaxTri + kCl - 1) / kCl;          // blocks one CTA loads
@@ -455,7 +456,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
       const int a = (e & 255) >> 3, q4 = e & 7;
       const int row = bi * kB + a, col = bj * kB + 4 * q4;
       if (row < r && col < r) {
-        const float* src = p.partials + (int64_t)row * r + col;
+        const float* src = p.partials + (int64_t)row * p.in_ld + col;
         for (int q = 0; q < p.n_partials; ++q) {
           const float4 v = __ldg(reinterpret_cast<const float4*>(src + (int64_t)q * p.partial_stride));
           acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
@@ -662,7 +663,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
       for (int e = gt; e < j * kB * kB; e += kGroup) {
         const int row = e >> 5, b = e & 31;
         if (b >= ncol) continue;
-        const int64_t off = (int64_t)row * r + j * kB + b;
+        const int64_t off = (int64_t)row * p.out_ld + j * kB + b;
         if (p.linv_f32) p.linv_f32[off] = 0.f;
         if (p.linv_hi) p.linv_hi[off] = __float2bfloat16(0.f);
         if (p.linv_lo) p.linv_lo[off] = __float2bfloat16(0.f);
@@ -702,7 +703,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
           const int row = k * kB + a;
           if (row >= r || b >= ncol) continue;
           const float v = src[b * kLd + a];
-          const int64_t off = (int64_t)row * r + j * kB + b;
+          const int64_t off = (int64_t)row * p.out_ld + j * kB + b;
           if (p.linv_f32) p.linv_f32[off] = v;
           if (p.linv_hi) {
             const __nv_bfloat16 hi = __float2bfloat16(v);
@@ -742,13 +743,15 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
 
 bool small_block_cluster_supported(const SmallBlockArgs& a) {
   return !a.use_f64 && a.partial_type == ELEM_F32 && a.r <= kMaxBlk * kB && a.r % 4 == 0 &&
-         a.linv_full == nullptr && (((uintptr_t)a.partials & 15) == 0) && (a.partial_stride % 4 == 0);
+         a.linv_full == nullptr && (((uintptr_t)a.partials & 15) == 0) && (a.partial_stride % 4 == 0) && (a.in_ld % 4 == 0);
 }
 
 cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t stream) {
   SCParams p;
   p.r = a.r;
   p.partials = (const float*)a.partials;
+  p.in_ld = a.in_ld ? a.in_ld : a.r;
+  p.out_ld = a.out_ld ? a.out_ld : a.r;
   p.n_partials = a.n_partials;
   p.partial_stride = a.partial_stride;
   p.shift_rel = a.shift_rel;

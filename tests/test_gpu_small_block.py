@@ -32,7 +32,8 @@ def spd(r: int, cond: float, seed: int) -> np.ndarray:
 @pytest.mark.parametrize("r,n_partials,cond", [(16, 1, 1e2), (32, 3, 1e3), (48, 2, 1e3), (64, 4, 1e4),
                                               (96, 1, 1e4), (128, 5, 1e5), (160, 2, 1e3), (192, 1, 1e3),
                                               (208, 3, 1e4), (224, 1, 1e2), (240, 2, 1e5), (256, 16, 1e5),
-                                              (256, 1, 1.5), (272, 2, 1e3), (512, 4, 1e4)])
+                                              (256, 1, 1.5), (272, 2, 1e3), (320, 1, 1e4), (384, 3, 1e5),
+                                              (496, 2, 1e3), (512, 4, 1e4)])
 def test_inverse_cholesky_factor(dev, r, n_partials, cond):
     W = spd(r, cond, seed=r + n_partials)
     rng = np.random.default_rng(7)
