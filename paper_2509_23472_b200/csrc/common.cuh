@@ -106,6 +106,8 @@ void gemm_tc_set_pair_mode(int on);   // test hook: 0 keeps every contraction on
 
 // Plain CUDA-core kernel for any shape and type (fp32 path, small or odd shapes).
 cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t stream);
+// fp32 x fp32 -> fp32 for matrices of a few hundred rows and columns (32 x 32 tiles, one per CTA).
+cudaError_t gemm_f32_small_launch(const GemmDesc& g, cudaStream_t stream);
 
 // ---------------------------------------------------------------- sampler and gather
 cudaError_t sample_indices_launch(uint64_t seed, uint64_t call_id, uint32_t n_rows, int rank,

@@ -148,6 +148,92 @@ __global__ void reduce_split3_kernel(const float* __restrict__ partials, int n_p
   }
 }
 
+// fp32 product for the r x r blocks of the two-level small-block scheme: C = alpha * A B (+ C), all of a few
+// hundred rows and columns.  32 x 32 output tiles on 64 threads (4 x 4 outputs each, operands read from
+// shared memory along the contraction index with 16-byte loads), so that a 256 x 256 product spreads over
+// 64 SMs; the K loop is double-buffered through registers.
+constexpr int kT32 = 32, kT32Ld = 36;
+
+__global__ void __launch_bounds__(64) gemm_f32_tile32_kernel(SimtParams p) {
+  __shared__ __align__(16) float As[kT32 * kT32Ld];   // [m][k]
+  __shared__ __align__(16) float Bs[kT32 * kT32Ld];   // [n][k]
+  const int tid = threadIdx.x;
+  const int m0 = blockIdx.y * kT32, n0 = blockIdx.x * kT32;
+  const int tm = tid >> 3, tn = tid & 7;               // outputs (4 tm + i, tn + 8 j)
+  const float* A = (const float*)p.A[0];
+  const float* B = (const float*)p.B[0];
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+  // each thread stages 16 elements of either tile per K chunk; the faster-varying index follows memory
+  float ra[16], rb[16];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int u = 0; u < 16; ++u) {
+      const int e = tid + 64 * u;
+      int mm, kk;
+      if (p.sak == 1) { kk = e & 31; mm = e >> 5; } else { mm = e & 31; kk = e >> 5; }
+      const int m = m0 + mm, k = k0 + kk;
+      ra[u] = (m < p.M && k < p.K) ? A[m * p.sam + k * p.sak] : 0.f;
+      int nn, kb;
+      if (p.sbk == 1) { kb = e & 31; nn = e >> 5; } else { nn = e & 31; kb = e >> 5; }
+      const int n = n0 + nn, k2 = k0 + kb;
+      rb[u] = (n < p.N && k2 < p.K) ? B[k2 * p.sbk + n * p.sbn] : 0.f;
+    }
+  };
+  auto stash = [&]() {
+#pragma unroll
+    for (int u = 0; u < 16; ++u) {
+      const int e = tid + 64 * u;
+      int mm, kk;
+      if (p.sak == 1) { kk = e & 31; mm = e >> 5; } else { mm = e & 31; kk = e >> 5; }
+      As[mm * kT32Ld + kk] = ra[u];
+      int nn, kb;
+      if (p.sbk == 1) { kb = e & 31; nn = e >> 5; } else { nn = e & 31; kb = e >> 5; }
+      Bs[nn * kT32Ld + kb] = rb[u];
+    }
+  };
+  fetch(0);
+  for (int k0 = 0; k0 < p.K; k0 += kT32) {
+    __syncthreads();
+    stash();
+    __syncthreads();
+    if (k0 + kT32 < p.K) fetch(k0 + kT32);
+#pragma unroll
+    for (int q4 = 0; q4 < kT32 / 4; ++q4) {
+      float4 a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = *reinterpret_cast<const float4*>(As + (4 * tm + i) * kT32Ld + 4 * q4);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = *reinterpret_cast<const float4*>(Bs + (tn + 8 * j) * kT32Ld + 4 * q4);
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          acc[i][j] = fmaf(a[i].x, b[j].x, acc[i][j]);
+          acc[i][j] = fmaf(a[i].y, b[j].y, acc[i][j]);
+          acc[i][j] = fmaf(a[i].z, b[j].z, acc[i][j]);
+          acc[i][j] = fmaf(a[i].w, b[j].w, acc[i][j]);
+        }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + 4 * tm + i;
+    if (m >= p.M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tn + 8 * j;
+      if (n >= p.N) continue;
+      float* c = (float*)p.C0 + (int64_t)m * p.ldc + n;
+      const float v = acc[i][j] * p.alpha;
+      *c = p.accumulate ? (*c + v) : v;
+    }
+  }
+}
+
 // hi/lo split of a block of an fp32 matrix, in place of the same block of two bf16 matrices.
 __global__ void split_block_kernel(const float* __restrict__ src, int rows, int cols, int64_t ld,
                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
@@ -275,6 +361,24 @@ cudaError_t reduce_split3_launch(const float* partials, int n_partials, int64_t 
   if (grid < 1) grid = 1;
   LORACT_CUDA_TRY(launch_pdl(reduce_split3_kernel, dim3(grid), dim3(256), 0, stream, partials, n_partials, stride, rows,
                              cols, ld_in, ld_out, hi, mid, lo));
+  count_launch(__func__, stream);
+  return cudaGetLastError();
+}
+
+cudaError_t gemm_f32_small_launch(const GemmDesc& g, cudaStream_t stream) {
+  if (g.a_type != ELEM_F32 || g.b_type != ELEM_F32 || g.out != OUT_F32 || g.n_terms != 1 || g.splits > 1)
+    return cudaErrorNotSupported;
+  SimtParams p = {};
+  p.M = g.M; p.N = g.N; p.K = g.K;
+  if (g.a_mn) { p.sam = 1; p.sak = g.lda; } else { p.sam = g.lda; p.sak = 1; }
+  if (g.b_mn) { p.sbn = 1; p.sbk = g.ldb; } else { p.sbn = g.ldb; p.sbk = 1; }
+  p.n_terms = 1;
+  p.A[0] = g.terms[0].A; p.B[0] = g.terms[0].B;
+  p.out = g.out; p.C0 = g.C0; p.ldc = g.ldc; p.splits = 1;
+  p.accumulate = g.accumulate ? 1 : 0;
+  p.alpha = g.alpha;
+  dim3 grid((g.N + kT32 - 1) / kT32, (g.M + kT32 - 1) / kT32);
+  gemm_f32_tile32_kernel<<<grid, 64, 0, stream>>>(p);
   count_launch(__func__, stream);
   return cudaGetLastError();
 }

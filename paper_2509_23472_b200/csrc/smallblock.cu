@@ -300,7 +300,7 @@ cudaError_t small_block_two_level(const SmallBlockArgs& a, cudaStream_t stream) 
     g.a_type = g.b_type = ELEM_F32;
     g.terms[0] = {A, B};
     g.out = OUT_F32; g.C0 = C; g.ldc = ldc; g.alpha = alpha; g.accumulate = accumulate;
-    return gemm_simt_launch(g, stream);
+    return gemm_f32_small_launch(g, stream);
   };
   const float* W21 = W + (size_t)r1 * r;
   float* W22 = W + (size_t)r1 * r + r1;
