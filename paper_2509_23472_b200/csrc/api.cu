@@ -188,7 +188,6 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
     GemmDesc g;
     g.M = n; g.N = l; g.K = (int)p.d; g.lda = ldx; g.ldb = p.d; g.a_type = g.b_type = el;
     g.terms[0] = {X, Omega};
-    g.a_streams = true;
     g.ldc = l;
     if (p.bf16) { g.out = OUT_SPLIT; g.C0 = w.Yh; g.C1 = w.Yl; } else { g.out = OUT_F32; g.C0 = w.Y32; }
     trace_label("pass 1: Y = X Omega^T");
@@ -241,7 +240,6 @@ cudaError_t project(const void* U, const void* X, int64_t ldx, const Plan& p, vo
   g.M = p.l; g.N = (int)p.d; g.K = (int)p.n; g.a_mn = true; g.b_mn = true; g.lda = p.l; g.ldb = ldx;
   g.a_type = g.b_type = p.bf16 ? ELEM_BF16 : ELEM_F32;
   g.terms[0] = {U, X};
-  g.b_streams = true;
   g.ldc = p.d;
   trace_label("pass 2: V = U^T X");
   if (!p.bf16) { g.out = OUT_F32; g.C0 = V; return run_gemm(g, status, stream); }
@@ -518,7 +516,6 @@ loract_status_t loract_prenorm_backward(const loract_desc_t* desc, const void* U
     GemmDesc g;
     g.M = n; g.N = r; g.K = d; g.lda = desc->ldx; g.ldb = d;
     g.terms[0] = {grad_A, V};
-    g.a_streams = true;
     g.out = OUT_F32; g.C0 = P; g.ldc = r;
     trace_label("pre-norm backward: P = grad_A V^T");
     e = gemm_tc_supported(g) ? gemm_tc_launch(g, status, st) : cudaErrorNotSupported;

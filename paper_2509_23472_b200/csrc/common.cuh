@@ -93,8 +93,6 @@ struct GemmDesc {
   const float* ep_row_a = nullptr;
   const float* ep_row_b = nullptr;
   const void* ep_col = nullptr;
-  // tensor-core path: the operand is large and read once from HBM (the activation matrix): prefetch it
-  bool a_streams = false, b_streams = false;
 };
 
 // tcgen05 engine: bf16 operands, fp32 accumulation in tensor memory.  Returns cudaErrorNotSupported

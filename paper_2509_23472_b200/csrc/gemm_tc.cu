@@ -26,7 +26,6 @@ namespace {
 constexpr int kBM = 128;
 constexpr int kBK = 64;          // bf16 elements = one 128-byte swizzle row
 constexpr int kStages = 4;
-constexpr int kPrefetchAhead = 8;  // K blocks asked for in L2 beyond the shared-memory ring
 constexpr int kThreads = 192;    // warp 0: TMA, warp 1: MMA + tensor memory, warps 2..5: epilogue
 constexpr uint32_t kABytes = kBM * kBK * 2;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
@@ -34,7 +33,6 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
 struct alignas(64) TmapPack {
   CUtensorMap a[3];
   CUtensorMap b[3];
-  CUtensorMap wide;   // K-major streaming operand, boxes of 256 elements along K: L2 prefetch only
 };
 
 struct TcParams {
@@ -56,7 +54,6 @@ struct TcParams {
   const float* ep_row_a;
   const float* ep_row_b;
   const void* ep_col;
-  int prefetch;       // bit 0: operand A streams from HBM, bit 1: operand B does -- prefetch it into L2 ahead
   uint32_t* dev_status;
 };
 
@@ -105,11 +102,6 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y)
       : "memory");
-}
-// Asks for a tile to be brought into L2; nothing is written to shared memory and nothing is waited for.
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"((uint64_t)map), "r"(x), "r"(y)
-               : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -297,29 +289,8 @@ gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   if (warp == 0) {
     if (lane == 0) {
       const uint32_t tx_bytes = stage_bytes;
-      // An operand that streams from HBM is asked for kPrefetchAhead K blocks early: the shared-memory
-      // ring (4 stages) then only has to cover the latency of L2, not that of HBM under load.
-      auto prefetch_block = [&](int it2) {
-        const int term2 = it2 / kb_count;
-        const int kb2 = kb_begin + (it2 - term2 * kb_count);
-        const int k2 = kb2 * kBK;
-        if (p.prefetch & 1) {
-          if (A_MN) { tma_prefetch_2d(&maps.a[term2], m0, k2); tma_prefetch_2d(&maps.a[term2], m0 + 64, k2); }
-          else if ((kb2 & 3) == 0) tma_prefetch_2d(&maps.wide, k2, m0);   // 512 contiguous bytes per row
-        }
-        if (p.prefetch & 2) {
-          if (B_MN) {
-            for (uint32_t q = 0; q * 8192u < p.b_bytes; ++q) tma_prefetch_2d(&maps.b[term2], n0 + (int)q * 64, k2);
-          } else if ((kb2 & 3) == 0) {
-            tma_prefetch_2d(&maps.wide, k2, n0);
-          }
-        }
-      };
-      if (p.prefetch)
-        for (int it2 = 0; it2 < min(n_iter, kStages + kPrefetchAhead); ++it2) prefetch_block(it2);
       for (int it = 0; it < n_iter; ++it) {
         const int s = it % kStages;
-        if (p.prefetch && it + kStages + kPrefetchAhead < n_iter) prefetch_block(it + kStages + kPrefetchAhead);
         if (!mbar_wait_bounded(&empty_bar[s], ((it / kStages) & 1) ^ 1, &abort_flag)) break;
         const int term = it / kb_count;
         const int k0 = (kb_begin + (it - term * kb_count)) * kBK;
@@ -580,7 +551,7 @@ cudaError_t get_tmap(const void* ptr, uint64_t inner, uint64_t outer, uint64_t l
   CUtensorMap m;
   const CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box,
                         elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        box_inner > 64 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
   {
@@ -696,11 +667,6 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   while ((int)p.tmem_cols < p.bn) p.tmem_cols *= 2;
   p.accumulate = g.accumulate ? 1 : 0;
   p.ep_E = g.ep_E; p.ep_ld = g.ep_ld; p.ep_row_a = g.ep_row_a; p.ep_row_b = g.ep_row_b; p.ep_col = g.ep_col;
-  // an operand too large to have stayed in L2 (tens of MB) streams from HBM even if the caller did not say so
-  const size_t stream_bytes = (size_t)32 << 20;
-  const bool a_big = (size_t)g.M * g.K * 2 >= stream_bytes, b_big = (size_t)g.N * g.K * 2 >= stream_bytes;
-  p.prefetch = g.n_terms == 1 ? (((g.a_streams || a_big) ? 1 : 0) | ((g.b_streams || b_big) ? 2 : 0)) : 0;
-  if (p.prefetch == 3 && !g.a_mn && !g.b_mn) p.prefetch = 1;   // one wide map: the larger role wins
   p.dev_status = dev_status;
 
   TmapPack maps;
@@ -711,17 +677,10 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
     else LORACT_CUDA_TRY(get_tmap(g.terms[t].B, g.K, g.N, g.ldb, 64, (uint32_t)b_rows, &maps.b[t]));
   }
   for (int t = g.n_terms; t < 3; ++t) { maps.a[t] = maps.a[0]; maps.b[t] = maps.b[0]; }
-  maps.wide = maps.a[0];
-  if (g.n_terms == 1) {
-    if ((p.prefetch & 1) && !g.a_mn) LORACT_CUDA_TRY(get_tmap(g.terms[0].A, g.K, g.M, g.lda, 256, kBM, &maps.wide));
-    else if ((p.prefetch & 2) && !g.b_mn)
-      LORACT_CUDA_TRY(get_tmap(g.terms[0].B, g.K, g.N, g.ldb, 256, (uint32_t)p.bn, &maps.wide));
-  }
 
   if (pair) {
     dim3 pgrid(2 * ((g.M + 2 * kBM - 1) / (2 * kBM)), (g.N + p.bn - 1) / p.bn, splits);
     const size_t psmem = (size_t)kPairStages * (kABytes + p.b_bytes) + 1024;
-    p.prefetch = 0;
     if (g.a_mn && g.b_mn) return launch_pair_variant<true, true>(maps, p, pgrid, psmem, stream);
     if (g.a_mn && !g.b_mn) return launch_pair_variant<true, false>(maps, p, pgrid, psmem, stream);
     if (!g.a_mn && g.b_mn) return launch_pair_variant<false, true>(maps, p, pgrid, psmem, stream);
