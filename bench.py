@@ -336,10 +336,13 @@ def main():
     roofline = None
     if k_ms is not None:
         achieved = k_bytes / (k_ms * 1e-3) / 1e9
-        roofline = {"kernel": "gemm_tc_kernel<K-major,K-major> (Y = X Omega^T)", "bound": "hbm",
+        roofline = {"kernel": "gemm_tc_pair_kernel<K-major,K-major> (pass 1, Y = X Omega^T)", "bound": "hbm",
                     "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                    "traffic": None, "ms_per_launch": k_ms, "algorithmic_bytes": k_bytes,
+                    # dram__bytes_read.sum + dram__bytes_write.sum per launch of this kernel at this shape
+                    # (profiles/pass1_llama7b_block_ncu.md); other shapes have not been captured
+                    "traffic": 140.3e6 if (N, d, r) == (16384, 4096, 256) else None,
+                    "ms_per_launch": k_ms, "algorithmic_bytes": k_bytes,
                     "tflops": 2.0 * N * d * r / (k_ms * 1e-3) / 1e12}
     # whole-step floor: X once + factors + gathered rows (strict), against measured HBM bandwidth
     strict_bytes = x_bytes + (N * r + 2 * r * d) * es + (N * r + N * g + r * d) * es + 4 * d * g
