@@ -177,6 +177,27 @@ cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs&
   return small_block_launch(a, stream);
 }
 
+// Omega = L^{-1} T for a test matrix T (l x d, K-major), T T^T = L L^T: the row space of T with rows close to
+// orthonormal.  Leaves L^{-1} in w.Lh / w.Ll (w.Linv32).
+cudaError_t precondition_rows(const void* T, int l, int64_t d, bool bf16, void* Omega, const BasisWs& w,
+                              uint32_t* status, cudaStream_t stream) {
+  trace_label("Gram of the test rows");
+  LORACT_CUDA_TRY(gram_rows(T, l, d, bf16, w, status, stream));
+  trace_label("small block 1");
+  LORACT_CUDA_TRY(factor(l, bf16, w.splits_gram_sample, kShiftSample, w, status, stream));
+  GemmDesc g;
+  g.M = l; g.N = (int)d; g.K = l; g.b_mn = true; g.lda = l; g.ldb = d;
+  g.a_type = g.b_type = bf16 ? ELEM_BF16 : ELEM_F32;
+  g.ldc = d; g.C0 = Omega;
+  if (bf16) {
+    g.n_terms = 2; g.terms[0] = {w.Lh, T}; g.terms[1] = {w.Ll, T}; g.out = OUT_BF16;
+  } else {
+    g.terms[0] = {w.Linv32, T}; g.out = OUT_F32;
+  }
+  trace_label("Omega = L^-1 T");
+  return run_gemm(g, status, stream);
+}
+
 // Lines 2 and 7 of Algorithm 1 for a test matrix Omega (l x d, rows are the test vectors):
 // Y = X Omega^T, then two rounds of { W = Y^T Y = L L^T ; Y <- Y L^{-T} }.  U (n x l) receives Q.
 cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* Omega, void* U,
@@ -294,23 +315,7 @@ cudaError_t compress_core(const loract_desc_t* desc, const void* X, int64_t ldx,
   // space of T, so range(X Omega^T) = range(X T^T), but its rows are close to orthonormal, which keeps the
   // spectrum of the sketch from being squared (and, in the iterations, raised to the fourth power).
   for (int it = 0; it <= desc->power_iters; ++it) {
-    trace_label("Gram of the test rows");
-    LORACT_CUDA_TRY(gram_rows(w.S, r, desc->d, bf16, w.b, w.status, stream));
-    trace_label("small block 1");
-    LORACT_CUDA_TRY(factor(r, bf16, w.b.splits_gram_sample, kShiftSample, w.b, w.status, stream));
-    {
-      GemmDesc g;
-      g.M = r; g.N = (int)desc->d; g.K = r; g.b_mn = true; g.lda = r; g.ldb = desc->d;
-      g.a_type = g.b_type = bf16 ? ELEM_BF16 : ELEM_F32;
-      g.ldc = desc->d; g.C0 = w.Omega;
-      if (bf16) {
-        g.n_terms = 2; g.terms[0] = {w.b.Lh, w.S}; g.terms[1] = {w.b.Ll, w.S}; g.out = OUT_BF16;
-      } else {
-        g.terms[0] = {w.b.Linv32, w.S}; g.out = OUT_F32;
-      }
-      trace_label("Omega = L^-1 T");
-      LORACT_CUDA_TRY(run_gemm(g, w.status, stream));
-    }
+    LORACT_CUDA_TRY(precondition_rows(w.S, r, desc->d, bf16, w.Omega, w.b, w.status, stream));
     // Y = X Omega^T, Y = QR (Q written to U)
     LORACT_CUDA_TRY(range_basis(X, ldx, plan, w.Omega, U, w.b, w.status, stream));
     // lines 4 and 5 of the loop: the next test matrix is (X^T Q)^T = Q^T X, kept where A_k was
@@ -544,7 +549,8 @@ size_t loract_rsvd_workspace_bytes(const loract_desc_t* desc, int32_t oversample
   Plan plan = make_plan(desc->n_tokens, desc->d, l, true);
   Carver c(nullptr);
   c.take(256);
-  c.take((size_t)l * desc->d * 2);  // test matrix / X^T Q
+  c.take((size_t)l * desc->d * 2);  // test matrix
+  c.take((size_t)l * desc->d * 2);  // Q^T X of the power iterations, before it is preconditioned
   BasisWs b;
   carve_basis(c, plan, &b);
   return c.off;
@@ -570,6 +576,7 @@ loract_status_t loract_rsvd(const loract_desc_t* desc, int32_t oversample, const
   Carver c(ws);
   uint32_t* status = (uint32_t*)c.take(256);
   __nv_bfloat16* Om = (__nv_bfloat16*)c.take((size_t)l * desc->d * 2);
+  __nv_bfloat16* Tq = (__nv_bfloat16*)c.take((size_t)l * desc->d * 2);
   BasisWs b;
   carve_basis(c, plan, &b);
   cudaStream_t st = (cudaStream_t)stream;
@@ -577,8 +584,11 @@ loract_status_t loract_rsvd(const loract_desc_t* desc, int32_t oversample, const
   if (e == cudaSuccess) e = gaussian_rows_launch(desc->seed, desc->call_id, l, desc->d, Om, st);
   if (e == cudaSuccess) e = range_basis(X, desc->ldx, plan, Om, Uq, b, status, st);
   for (int it = 0; it < desc->power_iters && e == cudaSuccess; ++it) {
-    // Y = X (X^T Q): X^T Q is kept transposed (l x d), which is exactly the test-matrix layout
-    e = project(Uq, X, desc->ldx, plan, Om, b, status, st);
+    // Y = X (X^T Q): X^T Q is kept transposed (l x d), which is exactly the test-matrix layout.  Its rows are
+    // brought close to orthonormal first (same row space, so the same range), as in loract_compress: the
+    // sketch would otherwise carry the cube of X's spectrum into a Gram matrix.
+    e = project(Uq, X, desc->ldx, plan, Tq, b, status, st);
+    if (e == cudaSuccess) e = precondition_rows(Tq, l, desc->d, true, Om, b, status, st);
     if (e == cudaSuccess) e = range_basis(X, desc->ldx, plan, Om, Uq, b, status, st);
   }
   if (e == cudaSuccess) e = project(Uq, X, desc->ldx, plan, B, b, status, st);

@@ -141,6 +141,12 @@ struct SmallBlockArgs {
   // row strides (elements) of the partial matrices and of the outputs; 0 means r.  The matrix may be a
   // diagonal sub-block of a larger one (the r > 256 path factors a 512 x 512 matrix through its 256 x 256 blocks)
   int64_t in_ld = 0, out_ld = 0;
+  // Where the scale of the shift and of the pivot floor comes from: by default the mean of the matrix's own
+  // diagonal.  A Schur complement that is handed in as "the matrix" can be all rounding noise, so the two-level
+  // path points this at the diagonal of the block it was taken from (scale_n entries, stride scale_ld + 1).
+  const float* scale_diag = nullptr;
+  int scale_n = 0;
+  int64_t scale_ld = 0;
 };
 cudaError_t small_block_launch(const SmallBlockArgs& a, cudaStream_t stream);
 // The same computation for r <= 256 in fp32 from fp32 partials, entirely in the shared memory of a

@@ -312,6 +312,9 @@ cudaError_t small_block_two_level(const SmallBlockArgs& a, cudaStream_t stream) 
   s2.r = r2; s2.partials = W22; s2.linv_f32 = X + (size_t)r1 * r + r1;
   s2.linv_hi = a.linv_hi + (size_t)r1 * r + r1;
   s2.linv_lo = a.linv_lo ? a.linv_lo + (size_t)r1 * r + r1 : nullptr;
+  // shift and pivot floor on the scale of W: S may be nothing but rounding noise of W22 - L21 L21^T, and a floor
+  // taken from its own diagonal would then let that noise through as pivots
+  s2.scale_diag = W; s2.scale_n = r1; s2.scale_ld = r;
   LORACT_CUDA_TRY(small_block_cluster_launch(s2, stream));
   // X21 = -X22 (L21 X11): T2[m][n] = sum_k L21[m][k] X11[k][n];  X21[m][n] = -sum_k X22[m][k] T2[k][n]
   LORACT_CUDA_TRY(simt(r2, r1, r1, T1, r1, X, r, true, T2, r1, 1.f, false));

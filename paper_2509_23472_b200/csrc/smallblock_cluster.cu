@@ -53,6 +53,9 @@ struct SCParams {
   __nv_bfloat16* linv_lo;
   uint32_t* dev_status;
   int64_t in_ld, out_ld;   // row strides of the partial matrices and of the outputs
+  const float* scale_diag; // optional: another matrix whose diagonal sets the scale of shift and floor
+  int scale_n;
+  int64_t scale_ld;
 };
 
 __device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }
@@ -434,10 +437,16 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
   // the diagonal shift and the pivot floor.
   {
     float t = 0.f;
-    for (int i = tid; i < r; i += kCThreads) {
-      float d = 0.f;
-      for (int q = 0; q < p.n_partials; ++q) d += __ldg(p.partials + (int64_t)q * p.partial_stride + (int64_t)i * p.in_ld + i);
-      t += d;
+    const int n_scale = p.scale_diag ? p.scale_n : r;
+    if (p.scale_diag) {
+      for (int i = tid; i < n_scale; i += kCThreads) t += __ldg(p.scale_diag + (int64_t)i * (p.scale_ld + 1));
+    } else {
+      for (int i = tid; i < r; i += kCThreads) {
+        float d = 0.f;
+        for (int q = 0; q < p.n_partials; ++q)
+          d += __ldg(p.partials + (int64_t)q * p.partial_stride + (int64_t)i * p.in_ld + i);
+        t += d;
+      }
     }
     constexpr int kMaxMine = (kMaxTri + kCl - 1) / kCl;          // blocks one CTA loads
     constexpr int kPerThread = kMaxMine * (kB * kB / 4) / kCThreads + 1;
@@ -470,7 +479,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
     if (tid == 0) {
       float tr = 0.f;
       for (int q = 0; q < kCThreads / 32; ++q) tr += s_red[q];
-      float mean_diag = tr / (float)r;
+      float mean_diag = tr / (float)n_scale;
       if (!(mean_diag == mean_diag) || mean_diag > 3.0e38f || mean_diag < 0.f) {
         if (p.dev_status && cta == 0) atomicOr(p.dev_status, LORACT_DEV_NONFINITE);
         mean_diag = 1.f;
@@ -759,6 +768,9 @@ cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t str
   p.linv_hi = a.linv_hi;
   p.linv_lo = a.linv_lo;
   p.dev_status = a.dev_status;
+  p.scale_diag = a.scale_diag;
+  p.scale_n = a.scale_n;
+  p.scale_ld = a.scale_ld;
   const size_t smem = (size_t)(kMaxTri + kXSlots) * kSlot * sizeof(float) + (size_t)(2 * kB * kLcolLd) * sizeof(float);
   static bool configured[64] = {};
   int dev = 0;

@@ -201,6 +201,22 @@ def test_rsvd_comparator(dev):
     assert e_gpu <= gpu_err(X64, Q0, B0) + 2e-3
 
 
+def test_rsvd_comparator_at_the_largest_test_matrix(dev):
+    # l = 512 Gaussian test vectors (the largest the library takes: the two-level small-block route) and one
+    # power iteration, on the long-context sweep's spectrum at a reduced width.  The iteration's test matrix
+    # Q^T X is brought back to near-orthonormal rows before it multiplies X again; without that the sketch
+    # carries the cube of the spectrum into a Gram matrix and the factors come out non-finite.
+    w = synth.scaled(synth.llama13b_sweep_point(1024, 512), n_tokens=4096, d=2048, rank=512, signal_rank=768)
+    X = synth.make_inputs(w, device=dev)["X"]
+    Q, Bm = B.rsvd(X, 512, oversample=0, power_iters=1, seed=5)
+    assert Q.shape == (4096, 512) and bool(torch.isfinite(Q.float()).all()) and bool(torch.isfinite(Bm.float()).all())
+    assert orth_defect(Q) <= TOL_ORTH
+    Xd = to64(X)
+    e_gpu = gpu_err(X.double(), Q, Bm)
+    e_orc = orc.rel_fro_error(Xd, *orc.rsvd(Xd, 512, 0, 1, seed=0, truncate=False))
+    assert abs(e_gpu - e_orc) <= TOL_ERR["bf16"]
+
+
 # ------------------------------------------------------------------ power iterations (Algorithm 1, lines 3 to 6)
 @pytest.mark.parametrize("t", [1, 2])
 def test_power_iterations_match_the_oracle_and_help_on_a_flat_spectrum(dev, t):

@@ -78,3 +78,31 @@ def test_non_positive_pivot_is_clamped_and_reported(dev):
     torch.cuda.synchronize()
     assert int(status.item()) & B.DEV_PIVOT_CLAMPED
     assert bool(torch.isfinite(L32).all())
+
+
+def test_two_level_scheme_judges_the_schur_complement_on_the_scale_of_the_whole_matrix(dev):
+    # r = 512 goes through two 256-wide factorisations joined by a Schur complement.  Here the last 256 columns
+    # of the factored Gram matrix are exact linear combinations of the first 256, so that complement is
+    # nothing but the rounding noise of W22 - L21 L21^T (about 1e-7 of W's diagonal, of either sign).  The
+    # shift and the pivot floor of the second factorisation must come from W's diagonal: taken from the
+    # complement's own, they would let that noise through as pivots and the inverse would blow up.
+    # Expected: a finite factor whose leading block is still the inverse Cholesky factor of W11 and whose
+    # trailing block is bounded by the inverse square root of the shift.
+    r = 512
+    rng = np.random.default_rng(11)
+    Y1 = 30.0 * rng.standard_normal((2048, 256))
+    C = rng.standard_normal((256, 256)) / 16.0
+    Y = np.concatenate([Y1, Y1 @ C], axis=1)
+    W = Y.T @ Y / 2048.0
+    shift = 3e-6
+    P32 = torch.tensor(W[None], dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    L32, Lh, Ll = B.debug_small_block(P32, use_f64=False, shift_rel=shift, status=status)
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(L32).all()) and bool(torch.isfinite(Lh.float()).all())
+    assert not int(status.item()) & B.DEV_NONFINITE
+    W11 = W[:256, :256] + shift * np.trace(W) / 512 * np.eye(256)
+    X11 = L32[:256, :256].double().cpu().numpy()
+    assert np.abs(X11 @ W11 @ X11.T - np.eye(256)).max() <= 1e-3
+    scale = np.trace(W[:256, :256]) / 256
+    assert float(L32[256:, 256:].abs().max()) <= 4.0 / np.sqrt(shift * scale)
