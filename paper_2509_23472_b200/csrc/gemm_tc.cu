@@ -55,6 +55,8 @@ struct TcParams {
   const float* ep_row_b;
   const void* ep_col;
   uint32_t* dev_status;
+  int st_m_tiles;     // streaming kernel: 256-row tiles along M
+  int st_units;       // streaming kernel: tiles in all (column tile major, then M)
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -148,18 +150,14 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
-// Epilogue of one CTA (four warps): reads its 128 accumulator rows (tensor-memory lanes) and writes them.
-// Warp w may touch the lanes 32 * (w % 4) .. + 31.
-__device__ __forceinline__ void tc_epilogue(const TcParams& p, uint32_t tmem_base, uint64_t* accum_bar,
-                                          volatile int* abort_flag_ptr, int warp, int lane, int m0, int n0,
-                                          int split, int n_iter) {
+// Writes one finished accumulator tile (128 rows of this CTA x bn columns, starting at tensor-memory column
+// tmem_base) in the output mode of p.  Warp w may touch the lanes 32 * (w % 4) .. + 31.
+__device__ __forceinline__ void tc_store_tile(const TcParams& p, uint32_t tmem_base, int warp, int lane, int m0,
+                                              int n0, int split) {
   const int quad = warp & 3;
   const int row = quad * 32 + lane;
   const int m = m0 + row;
-  bool ok = mbar_wait_bounded(accum_bar, 0, abort_flag_ptr);
-  ok = __all_sync(0xffffffffu, ok);
-  tc_fence_after();
-  if (ok && n_iter > 0) {
+  {
     for (int c0 = 0; c0 < p.bn; c0 += 32) {
       uint32_t v[32];
       tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
@@ -239,12 +237,25 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, uint32_t tmem_bas
         }
       }
     }
+  }
+}
+
+// Epilogue of one CTA (four warps) of the one-tile kernels: waits for the accumulator, then writes it.
+__device__ __forceinline__ void tc_epilogue(const TcParams& p, uint32_t tmem_base, uint64_t* accum_bar,
+                                          volatile int* abort_flag_ptr, int warp, int lane, int m0, int n0,
+                                          int split, int n_iter) {
+  const int m = m0 + (warp & 3) * 32 + lane;
+  bool ok = mbar_wait_bounded(accum_bar, 0, abort_flag_ptr);
+  ok = __all_sync(0xffffffffu, ok);
+  tc_fence_after();
+  if (ok && n_iter > 0) {
+    tc_store_tile(p, tmem_base, warp, lane, m0, n0, split);
   } else if (ok && n_iter == 0 && m < p.M && p.out == OUT_F32) {
     // an empty K range still owns its partial: write zeros
     float* dst = (float*)p.C0 + (int64_t)split * p.split_stride + (int64_t)m * p.ldc + n0;
     for (int q = 0; q < min(p.bn, p.N - n0); ++q) dst[q] = 0.f;
   }
-  }
+}
 
 template <bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -508,6 +519,193 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   if (threadIdx.x == 0 && abort_flag && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_WAIT_EXPIRED);
 }
 
+// ------------------------------------------------------------------ many tiles per CTA pair, B resident
+// C = A B for a short contraction (K <= 512) and a large output, the shape of Reconstruct (X~ = U V): the
+// work per output tile is a handful of K blocks, so a kernel that lives for one tile spends its time on set-up,
+// one load round trip and one store round trip, none of them overlapped.  Here a CTA pair is persistent:
+//   * the tiles are numbered column tile first; pair p takes the contiguous range [p U / P, (p + 1) U / P), so
+//     it stays on one column tile for many tiles (and changes it once or twice at most);
+//   * its half of the B tile (all K blocks) stays in shared memory while the column tile does not change;
+//     only A is streamed through a ring of 128 x 64 stages;
+//   * the accumulator is double buffered in tensor memory (2 x bn columns): the tensor cores work on tile
+//     i + 1 while the four epilogue warps read and store tile i.
+// Barriers.  a_full / a_empty: the ring, as in the pair kernel.  b_full (leader): both halves of B have
+// landed; b_empty (each CTA, by commit): every MMA that reads the resident B is done, it may be replaced.
+// acc_full[j] (each CTA, by commit): buffer j holds a finished tile; acc_empty[j] (leader, 8 arrivals: the
+// four epilogue warps of both CTAs): buffer j has been read in both CTAs.  No load uses cluster multicast.
+constexpr int kStreamStages = 6;
+
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t spin = 1;; ++spin) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if ((spin & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  __shared__ __align__(8) uint64_t a_full[kStreamStages];
+  __shared__ __align__(8) uint64_t a_empty[kStreamStages];
+  __shared__ __align__(8) uint64_t b_full, b_empty;
+  __shared__ __align__(8) uint64_t acc_full[2];
+  __shared__ __align__(8) uint64_t acc_empty[2];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+
+  uint32_t cta_rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(cta_rank));
+  const bool leader = cta_rank == 0;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_pairs = (int)(gridDim.x >> 1), pair = (int)(blockIdx.x >> 1);
+  const int u_begin = (int)((long long)pair * p.st_units / n_pairs);
+  const int u_end = (int)((long long)(pair + 1) * p.st_units / n_pairs);
+  const int half_n = p.bn / 2;
+  const uint32_t b_kb_bytes = p.b_bytes;                     // this CTA's half of B, one K block
+  unsigned char* tiles = (unsigned char*)(((uintptr_t)smem + 1023) & ~(uintptr_t)1023);
+  unsigned char* b_res = tiles;
+  unsigned char* ring = tiles + (size_t)p.kb_total * b_kb_bytes;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStreamStages; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1); }
+    mbar_init(&b_full, 1);
+    mbar_init(&b_empty, 1);
+    for (int j = 0; j < 2; ++j) { mbar_init(&acc_full[j], 1); mbar_init(&acc_empty[j], 8); }
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                 "r"(p.tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_slot;
+  pdl_wait();
+  pdl_launch_dependents();
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const uint32_t bar_b = map_to_rank(smem_u32(&b_full), 0u);
+      int it = 0, nb = 0, cur_nt = -1;
+      bool ok = true;
+      for (int u = u_begin; u < u_end && ok; ++u) {
+        const int nt = u / p.st_m_tiles, mt = u - nt * p.st_m_tiles;
+        if (nt != cur_nt) {
+          // the MMAs that read the previous column tile's B are done in both CTAs before it is replaced
+          if (nb > 0) ok = mbar_wait_bounded(&b_empty, (uint32_t)((nb - 1) & 1), &abort_flag);
+          if (!ok) break;
+          if (leader) mbar_arrive_expect_tx(&b_full, 2u * (uint32_t)p.kb_total * b_kb_bytes);
+          const int nb0 = nt * p.bn + (int)cta_rank * half_n;
+          for (int kb = 0; kb < p.kb_total; ++kb)
+            for (uint32_t q = 0; q * 8192u < b_kb_bytes; ++q)
+              tma_load_2d_pair(b_res + (size_t)kb * b_kb_bytes + q * 8192u, &maps.b[0], bar_b, nb0 + (int)q * 64,
+                               kb * kBK);
+          ++nb;
+          cur_nt = nt;
+        }
+        const int m0 = mt * 2 * kBM + (int)cta_rank * kBM;
+        for (int kb = 0; kb < p.kb_total; ++kb, ++it) {
+          const int s = it % kStreamStages;
+          ok = mbar_wait_bounded(&a_empty[s], (uint32_t)(((it / kStreamStages) & 1) ^ 1), &abort_flag);
+          if (!ok) break;
+          if (leader) mbar_arrive_expect_tx(&a_full[s], 2u * kABytes);
+          tma_load_2d_pair(ring + (size_t)s * kABytes, &maps.a[0], map_to_rank(smem_u32(&a_full[s]), 0u), kb * kBK, m0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && leader) {
+      // instruction descriptor: fp32 accumulator, bf16 A (K-major) and B (MN-major), N >> 3, M = 256 >> 4
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(p.bn >> 3) << 17) |
+                             ((uint32_t)((2 * kBM) >> 4) << 24);
+      int it = 0, nb = 0, cur_nt = -1;
+      bool ok = true;
+      for (int u = u_begin, ui = 0; u < u_end && ok; ++u, ++ui) {
+        const int j = ui & 1;
+        const int nt = u / p.st_m_tiles;
+        // buffer j was read by both epilogues (the first use of each buffer passes at once)
+        ok = mbar_wait_cluster_bounded(&acc_empty[j], (uint32_t)(((ui >> 1) & 1) ^ 1), &abort_flag);
+        if (!ok) break;
+        if (nt != cur_nt) {
+          ok = mbar_wait_bounded(&b_full, (uint32_t)(nb & 1), &abort_flag);
+          if (!ok) break;
+          ++nb;
+          cur_nt = nt;
+        }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(j * p.bn);
+        for (int kb = 0; kb < p.kb_total; ++kb, ++it) {
+          const int s = it % kStreamStages;
+          ok = mbar_wait_bounded(&a_full[s], (uint32_t)((it / kStreamStages) & 1), &abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t a_desc = make_smem_desc(smem_u32(ring + (size_t)s * kABytes), false);
+          const uint64_t b_desc = make_smem_desc(smem_u32(b_res + (size_t)kb * b_kb_bytes), true);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k)
+            tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(32u >> 4) * k, b_desc + (uint64_t)(2048u >> 4) * k, idesc,
+                             (kb > 0 || k > 0) ? 1u : 0u);
+          tc_commit_pair(&a_empty[s]);
+        }
+        if (!ok) break;
+        tc_commit_pair(&acc_full[j]);
+        if (u + 1 == u_end || (u + 1) / p.st_m_tiles != nt) tc_commit_pair(&b_empty);
+      }
+    }
+  } else {
+    bool ok = true;
+    for (int u = u_begin, ui = 0; u < u_end; ++u, ++ui) {
+      const int j = ui & 1;
+      const int nt = u / p.st_m_tiles, mt = u - nt * p.st_m_tiles;
+      ok = mbar_wait_bounded(&acc_full[j], (uint32_t)((ui >> 1) & 1), &abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      tc_store_tile(p, tmem_base + (uint32_t)(j * p.bn), warp, lane, mt * 2 * kBM + (int)cta_rank * kBM, nt * p.bn, 0);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&acc_empty[j]), 0u));
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  // neither CTA frees tensor memory or leaves while the other may still use its shared or tensor memory
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols)
+                 : "memory");
+  }
+  if (threadIdx.x == 0 && abort_flag && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_WAIT_EXPIRED);
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -619,7 +817,54 @@ cudaError_t launch_pair_variant(const TmapPack& maps, const TcParams& p, dim3 gr
   return cudaGetLastError();
 }
 
-int g_pair_mode = 1;   // 0: never use the two-CTA kernel (test hook)
+// Pairs the streaming kernel is launched with: as many as can be resident at once (one CTA per SM).
+cudaError_t launch_stream(const TmapPack& maps, TcParams p, size_t smem, cudaStream_t stream) {
+  static bool configured[64] = {};
+  static int max_pairs[64] = {};
+  int dev = 0;
+  LORACT_CUDA_TRY(cudaGetDevice(&dev));
+  const bool cached = dev >= 0 && dev < 64 && configured[dev];
+  int pairs = cached ? max_pairs[dev] : 0;
+  if (!cached) {
+    const int smem_max = 8 * 8192 + kStreamStages * (int)kABytes + 1024;
+    LORACT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
+    cudaLaunchConfig_t q = {};
+    q.gridDim = dim3(2); q.blockDim = dim3(kThreads); q.dynamicSmemBytes = smem_max;
+    cudaLaunchAttribute qa[1];
+    qa[0].id = cudaLaunchAttributeClusterDimension;
+    qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+    q.attrs = qa; q.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_stream_kernel, &q) != cudaSuccess || n < 1) {
+      (void)cudaGetLastError();
+      cudaDeviceProp prop;
+      LORACT_CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+      n = prop.multiProcessorCount / 2;
+    }
+    pairs = n < 1 ? 1 : n;
+    if (dev >= 0 && dev < 64) { max_pairs[dev] = pairs; configured[dev] = true; }
+  }
+  if (pairs > p.st_units) pairs = p.st_units;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  LORACT_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_stream_kernel, maps, p));
+  count_launch(__func__, stream);
+  return cudaGetLastError();
+}
+
+int g_pair_mode = 1;   // 0: never use the two-CTA kernels (test hook); 1: by shape; 2: as 1, but no streaming kernel
 
 }  // namespace
 
@@ -668,6 +913,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   p.accumulate = g.accumulate ? 1 : 0;
   p.ep_E = g.ep_E; p.ep_ld = g.ep_ld; p.ep_row_a = g.ep_row_a; p.ep_row_b = g.ep_row_b; p.ep_col = g.ep_col;
   p.dev_status = dev_status;
+  p.st_m_tiles = 0; p.st_units = 0;
 
   TmapPack maps;
   for (int t = 0; t < g.n_terms; ++t) {
@@ -678,6 +924,22 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   }
   for (int t = g.n_terms; t < 3; ++t) { maps.a[t] = maps.a[0]; maps.b[t] = maps.b[0]; }
 
+  // Short contraction, large output, A K-major, B MN-major, one term (Reconstruct and the pre-norm backward):
+  // the persistent kernel with B resident, when there is more than one tile per resident pair.
+  if (g_pair_mode == 1 && g.M >= 2 * kBM && !g.a_mn && g.b_mn && g.n_terms == 1 && splits == 1 && p.kb_total <= 8 &&
+      g.N >= 256) {
+    TcParams sp = p;
+    sp.bn = p.kb_total <= 4 ? 256 : 128;
+    sp.b_bytes = (uint32_t)(sp.bn / 2 / 64) * 8192u;
+    sp.tmem_cols = 2u * (uint32_t)sp.bn;
+    sp.st_m_tiles = (g.M + 2 * kBM - 1) / (2 * kBM);
+    const long long units = (long long)sp.st_m_tiles * ((g.N + sp.bn - 1) / sp.bn);
+    if (units >= 148 && units < (1ll << 30)) {
+      sp.st_units = (int)units;
+      const size_t ssmem = (size_t)sp.kb_total * sp.b_bytes + (size_t)kStreamStages * kABytes + 1024;
+      return launch_stream(maps, sp, ssmem, stream);
+    }
+  }
   if (pair) {
     dim3 pgrid(2 * ((g.M + 2 * kBM - 1) / (2 * kBM)), (g.N + p.bn - 1) / p.bn, splits);
     const size_t psmem = (size_t)kPairStages * (kABytes + p.b_bytes) + 1024;

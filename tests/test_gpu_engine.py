@@ -86,3 +86,29 @@ def test_both_forms_agree_bit_for_bit_on_a_gram_product(dev):
     C2 = B.debug_gemm(As, Bs, M, N, K, True, True, out_mode=B.OUT_F32)
     torch.cuda.synchronize()
     assert float((C1 - C2).abs().max()) <= 1e-5 * float(C1.abs().max())
+
+
+@pytest.mark.parametrize("M,N,K,out_mode", [
+    (8192, 4096, 256, "bf16"),     # 32 x 16 tiles of 256 x 256, four K blocks: two or three column tiles per pair
+    (7000, 1288, 96, "f32"),       # ragged rows, ragged last column tile, K not a multiple of 64
+    (4100, 2560, 512, "bf16"),     # eight K blocks: 128-wide column tiles
+    (40000, 256, 48, "f32"),       # one column tile, many row tiles
+])
+def test_persistent_form_for_short_contractions_with_a_large_output(dev, M, N, K, out_mode):
+    # The shape of Reconstruct (A K-major, B N-major, K <= 512, far more tiles than SMs) is served by the
+    # persistent pair kernel: B resident, A streamed, double-buffered accumulator.  Checked against the
+    # definition and, bit for bit, against the one-tile-per-CTA form (same products in the same order).
+    As, Bs, ref = operands(M, N, K, False, True, 1, dev, seed=M + K)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    mode = B.OUT_BF16 if out_mode == "bf16" else B.OUT_F32
+    B.debug_set_pair_mode(True)
+    C = B.debug_gemm(As, Bs, M, N, K, False, True, out_mode=mode, status=status)
+    B.debug_set_pair_mode(False)
+    C1 = B.debug_gemm(As, Bs, M, N, K, False, True, out_mode=mode, status=status)
+    B.debug_set_pair_mode(True)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    scale = float(ref.abs().max())
+    tol = (2.0 ** -8 if out_mode == "bf16" else 2e-5 * max(1.0, (K / 64) ** 0.5)) * scale
+    assert float((C.double() - ref).abs().max()) <= tol
+    assert torch.equal(C, C1)
