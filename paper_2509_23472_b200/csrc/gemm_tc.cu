@@ -33,6 +33,7 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
 struct alignas(64) TmapPack {
   CUtensorMap a[3];
   CUtensorMap b[3];
+  CUtensorMap c[2];   // outputs (C0, C1) for the staged epilogue: boxes of 128 bytes x 32 rows
 };
 
 struct TcParams {
@@ -55,6 +56,7 @@ struct TcParams {
   const float* ep_row_b;
   const void* ep_col;
   uint32_t* dev_status;
+  int tma_store;      // 1: the epilogue stages 32-row boxes in shared memory and writes them with TMA stores
   int st_m_tiles;     // streaming kernel: 256-row tiles along M
   int st_units;       // streaming kernel: tiles in all (column tile major, then M)
 };
@@ -150,13 +152,165 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
+// ---- staged epilogue.  A thread owns one accumulator row, so a direct store instruction of a warp touches 32
+// different rows, 16 bytes each: every 128-byte line of the output is written in eight pieces by eight
+// instructions.  Instead each epilogue warp puts its 32 rows x 128 bytes into shared memory in the layout of a
+// 128-byte-swizzled TMA box (conflict free: the 16-byte chunk c of row i goes to chunk c ^ (i & 7)) and one
+// lane sends the box with a TMA store, which writes whole lines and clips at the edges of the output.  Each
+// warp cycles through kStoreBufs boxes of its own, so no barrier between warps is needed.
+constexpr int kStoreBufs = 4;
+constexpr uint32_t kStoreBoxBytes = 4096;                    // 32 rows x 128 bytes
+constexpr uint32_t kStoreWarpBytes = kStoreBufs * kStoreBoxBytes;
+
+struct StoreStage {
+  unsigned char* base;   // this warp's boxes (1024-byte aligned); nullptr: direct stores only
+  uint32_t cnt;          // boxes sent so far
+};
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"((uint64_t)map), "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+               : "memory");
+}
+template <int kPending>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kPending) : "memory");
+}
+// Boxes cnt .. cnt + kNeed - 1 may be written once the stores that last used them have read shared memory.
+template <int kNeed>
+__device__ __forceinline__ void stage_acquire(const StoreStage& st, int lane) {
+  if (st.cnt + kNeed > kStoreBufs) {
+    if (lane == 0) bulk_wait_read<kStoreBufs - kNeed>();
+    __syncwarp();
+  }
+}
+__device__ __forceinline__ unsigned char* stage_box(const StoreStage& st, uint32_t k) {
+  return st.base + ((st.cnt + k) % kStoreBufs) * kStoreBoxBytes;
+}
+__device__ __forceinline__ void stage_write16(unsigned char* box, int lane, int chunk, uint4 v) {
+  *reinterpret_cast<uint4*>(box + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = v;
+}
+// All lanes have written their rows of `box`: make them visible to the async proxy and send the box.
+__device__ __forceinline__ void stage_send(const CUtensorMap* map, unsigned char* box, int lane, int x, int y) {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncwarp();
+  if (lane == 0) {
+    tma_store_2d(map, box, x, y);
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  }
+}
+// Before the shared memory goes away (or at the end of the kernel): every store of this warp is complete.
+__device__ __forceinline__ void stage_drain(const StoreStage& st, int lane) {
+  if (st.base && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  __syncwarp();
+}
+
+__device__ __forceinline__ void tc_store_tile_staged(const TcParams& p, const TmapPack& maps, uint32_t tmem_base,
+                                                     int quad, int lane, int m0, int n0, int split,
+                                                     StoreStage& st) {
+  const int row0 = m0 + quad * 32;
+  const int m = row0 + lane;
+  const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+  const int y = split * p.M + row0;
+  if (p.out == OUT_F32) {
+    for (int c0 = 0; c0 < p.bn && n0 + c0 < p.N; c0 += 32) {
+      uint32_t v[32];
+      tc_ld32(taddr + (uint32_t)c0, v);
+      tc_wait_ld();
+      stage_acquire<1>(st, lane);
+      unsigned char* box = stage_box(st, 0);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) stage_write16(box, lane, q, make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]));
+      stage_send(&maps.c[0], box, lane, n0 + c0, y);
+      st.cnt += 1;
+    }
+    return;
+  }
+  const bool split_out = p.out == OUT_SPLIT;
+  const bool rms = p.out == OUT_RMS_BWD;
+  const bool live = m < p.M;                                 // rows past M are clipped by the store
+  float ra = 0.f, rb = 0.f;
+  if (rms && live) { ra = p.ep_row_a[m]; rb = p.ep_row_b[m]; }
+  for (int c0 = 0; c0 < p.bn && n0 + c0 < p.N; c0 += 64) {
+    if (split_out) stage_acquire<2>(st, lane); else stage_acquire<1>(st, lane);
+    unsigned char* box_hi = stage_box(st, 0);
+    unsigned char* box_lo = stage_box(st, 1);
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      uint32_t v[32];
+      tc_ld32(taddr + (uint32_t)(c0 + 32 * half), v);
+      tc_wait_ld();
+      const int n = n0 + c0 + 32 * half;
+      if (rms) {
+        const bool cols_ok = n + 32 <= p.N;                  // a partial group is clipped anyway; read nothing past N
+        const __nv_bfloat16* e = (const __nv_bfloat16*)p.ep_E + (int64_t)m * p.ep_ld + n;
+        const __nv_bfloat16* col = (const __nv_bfloat16*)p.ep_col + n;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t ow[4] = {0u, 0u, 0u, 0u};
+          if (live && cols_ok) {
+            const uint4 ev = reinterpret_cast<const uint4*>(e)[q];
+            const uint4 cv = __ldg(reinterpret_cast<const uint4*>(col) + q);
+            const uint32_t ew[4] = {ev.x, ev.y, ev.z, ev.w}, cw[4] = {cv.x, cv.y, cv.z, cv.w};
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              const float e0 = __uint_as_float(ew[h] << 16), e1 = __uint_as_float(ew[h] & 0xffff0000u);
+              const float c0f = __uint_as_float(cw[h] << 16), c1f = __uint_as_float(cw[h] & 0xffff0000u);
+              const float a0 = __uint_as_float(v[8 * q + 2 * h]), a1 = __uint_as_float(v[8 * q + 2 * h + 1]);
+              ow[h] = pack_bf16x2(ra * c0f * e0 - rb * a0 / c0f, ra * c1f * e1 - rb * a1 / c1f);
+            }
+          } else if (live) {
+            for (int h = 0; h < 8; ++h) {
+              const int nn = n + 8 * q + h;
+              if (nn < p.N) {
+                const float c = __bfloat162float(col[8 * q + h]);
+                const float r = ra * c * __bfloat162float(e[8 * q + h]) - rb * __uint_as_float(v[8 * q + h]) / c;
+                const uint32_t bits = (uint32_t)__bfloat16_as_ushort(__float2bfloat16(r));
+                ow[h >> 1] |= (h & 1) ? (bits << 16) : bits;
+              }
+            }
+          }
+          stage_write16(box_hi, lane, 4 * half + q, make_uint4(ow[0], ow[1], ow[2], ow[3]));
+        }
+      } else {
+        uint32_t hi[16], lo[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+          const float x0 = __uint_as_float(v[2 * q]), x1 = __uint_as_float(v[2 * q + 1]);
+          const __nv_bfloat16 h0 = __float2bfloat16(x0), h1 = __float2bfloat16(x1);
+          hi[q] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+          lo[q] = pack_bf16x2(x0 - __bfloat162float(h0), x1 - __bfloat162float(h1));
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          stage_write16(box_hi, lane, 4 * half + q, make_uint4(hi[4 * q], hi[4 * q + 1], hi[4 * q + 2], hi[4 * q + 3]));
+        if (split_out) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            stage_write16(box_lo, lane, 4 * half + q, make_uint4(lo[4 * q], lo[4 * q + 1], lo[4 * q + 2], lo[4 * q + 3]));
+        }
+      }
+    }
+    stage_send(&maps.c[0], box_hi, lane, n0 + c0, y);
+    if (split_out) stage_send(&maps.c[1], box_lo, lane, n0 + c0, y);
+    st.cnt += split_out ? 2 : 1;
+  }
+}
+
 // Writes one finished accumulator tile (128 rows of this CTA x bn columns, starting at tensor-memory column
 // tmem_base) in the output mode of p.  Warp w may touch the lanes 32 * (w % 4) .. + 31.
-__device__ __forceinline__ void tc_store_tile(const TcParams& p, uint32_t tmem_base, int warp, int lane, int m0,
-                                              int n0, int split) {
+__device__ __forceinline__ void tc_store_tile(const TcParams& p, const TmapPack& maps, uint32_t tmem_base, int warp,
+                                              int lane, int m0, int n0, int split, StoreStage& st) {
   const int quad = warp & 3;
   const int row = quad * 32 + lane;
   const int m = m0 + row;
+  if (m0 + quad * 32 >= p.M) return;                         // none of this warp's rows exists
+  // staged unless the output needs read-modify-write, or (split-K partials stacked along the rows of one
+  // tensor map) the warp's 32 rows are not all inside M
+  if (st.base && p.tma_store && !p.accumulate && (p.split_stride == 0 || m0 + quad * 32 + 32 <= p.M)) {
+    tc_store_tile_staged(p, maps, tmem_base, quad, lane, m0, n0, split, st);
+    return;
+  }
   {
     for (int c0 = 0; c0 < p.bn; c0 += 32) {
       uint32_t v[32];
@@ -241,15 +395,21 @@ __device__ __forceinline__ void tc_store_tile(const TcParams& p, uint32_t tmem_b
 }
 
 // Epilogue of one CTA (four warps) of the one-tile kernels: waits for the accumulator, then writes it.
-__device__ __forceinline__ void tc_epilogue(const TcParams& p, uint32_t tmem_base, uint64_t* accum_bar,
-                                          volatile int* abort_flag_ptr, int warp, int lane, int m0, int n0,
-                                          int split, int n_iter) {
+// `ring` is the operand ring: once the accumulator is complete every load has landed and every MMA has read
+// its stage, so the epilogue warps take the ring over as staging space (16 KB per warp).
+__device__ __forceinline__ void tc_epilogue(const TcParams& p, const TmapPack& maps, uint32_t tmem_base,
+                                          uint64_t* accum_bar, volatile int* abort_flag_ptr, int warp, int lane,
+                                          int m0, int n0, int split, int n_iter, unsigned char* ring) {
   const int m = m0 + (warp & 3) * 32 + lane;
   bool ok = mbar_wait_bounded(accum_bar, 0, abort_flag_ptr);
   ok = __all_sync(0xffffffffu, ok);
   tc_fence_after();
   if (ok && n_iter > 0) {
-    tc_store_tile(p, tmem_base, warp, lane, m0, n0, split);
+    StoreStage st;
+    st.base = ring + (uint32_t)(warp & 3) * kStoreWarpBytes;
+    st.cnt = 0;
+    tc_store_tile(p, maps, tmem_base, warp, lane, m0, n0, split, st);
+    stage_drain(st, lane);
   } else if (ok && n_iter == 0 && m < p.M && p.out == OUT_F32) {
     // an empty K range still owns its partial: write zeros
     float* dst = (float*)p.C0 + (int64_t)split * p.split_stride + (int64_t)m * p.ldc + n0;
@@ -350,7 +510,7 @@ gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
       tc_commit(&accum_bar);       // accumulator complete (or nothing was issued)
     }
   } else {
-    tc_epilogue(p, tmem_base, &accum_bar, &abort_flag, warp, lane, m0, n0, split, n_iter);
+    tc_epilogue(p, maps, tmem_base, &accum_bar, &abort_flag, warp, lane, m0, n0, split, n_iter, tiles);
   }
   tc_fence_before();
   __syncthreads();
@@ -504,7 +664,7 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
       tc_commit_pair(&accum_bar);        // accumulator complete in both CTAs (or nothing was issued)
     }
   } else {
-    tc_epilogue(p, tmem_base, &accum_bar, &abort_flag, warp, lane, m0, n0, split, n_iter);
+    tc_epilogue(p, maps, tmem_base, &accum_bar, &abort_flag, warp, lane, m0, n0, split, n_iter, tiles);
   }
   tc_fence_before();
   __syncthreads();
@@ -680,6 +840,9 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
     }
   } else {
     bool ok = true;
+    StoreStage st;
+    st.base = ring + (size_t)kStreamStages * kABytes + (uint32_t)(warp & 3) * kStoreWarpBytes;
+    st.cnt = 0;
     for (int u = u_begin, ui = 0; u < u_end; ++u, ++ui) {
       const int j = ui & 1;
       const int nt = u / p.st_m_tiles, mt = u - nt * p.st_m_tiles;
@@ -687,11 +850,14 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      tc_store_tile(p, tmem_base + (uint32_t)(j * p.bn), warp, lane, mt * 2 * kBM + (int)cta_rank * kBM, nt * p.bn, 0);
+      tc_store_tile(p, maps, tmem_base + (uint32_t)(j * p.bn), warp, lane, mt * 2 * kBM + (int)cta_rank * kBM,
+                    nt * p.bn, 0, st);
+      // the tile is in registers / shared memory now: hand the buffer back before the stores have drained
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&acc_empty[j]), 0u));
     }
+    stage_drain(st, lane);
   }
   tc_fence_before();
   __syncthreads();
@@ -727,14 +893,15 @@ EncodeTiledFn get_encode_fn() {
 
 // Tensor maps depend only on (pointer, extents, stride, box); they are cached so that a repeated call
 // on the same buffers encodes nothing.
-typedef std::tuple<const void*, uint64_t, uint64_t, uint64_t, uint32_t, uint32_t> TmapKey;
+typedef std::tuple<const void*, uint64_t, uint64_t, uint64_t, uint32_t, uint32_t, int> TmapKey;
 std::mutex g_tmap_mutex;
 std::map<TmapKey, CUtensorMap> g_tmap_cache;
 
-// 2-D bf16 tensor: `inner` contiguous elements, `outer` rows `ld` elements apart; box inner x outer.
+// 2-D tensor of bf16 (es = 2) or fp32 (es = 4): `inner` contiguous elements, `outer` rows `ld` elements apart;
+// box inner x outer.
 cudaError_t get_tmap(const void* ptr, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_inner,
-                     uint32_t box_outer, CUtensorMap* out) {
-  const TmapKey key(ptr, inner, outer, ld, box_inner, box_outer);
+                     uint32_t box_outer, CUtensorMap* out, int es = 2) {
+  const TmapKey key(ptr, inner, outer, ld, box_inner, box_outer, es);
   {
     std::lock_guard<std::mutex> lock(g_tmap_mutex);
     auto it = g_tmap_cache.find(key);
@@ -743,11 +910,11 @@ cudaError_t get_tmap(const void* ptr, uint64_t inner, uint64_t outer, uint64_t l
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return cudaErrorNotSupported;
   cuuint64_t dims[2] = {inner, outer};
-  cuuint64_t strides[1] = {ld * 2};
+  cuuint64_t strides[1] = {ld * (uint64_t)es};
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t elem[2] = {1, 1};
   CUtensorMap m;
-  const CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box,
+  const CUresult r = fn(&m, es == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box,
                         elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
                         CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -826,7 +993,7 @@ cudaError_t launch_stream(const TmapPack& maps, TcParams p, size_t smem, cudaStr
   const bool cached = dev >= 0 && dev < 64 && configured[dev];
   int pairs = cached ? max_pairs[dev] : 0;
   if (!cached) {
-    const int smem_max = 8 * 8192 + kStreamStages * (int)kABytes + 1024;
+    const int smem_max = 8 * 8192 + kStreamStages * (int)kABytes + 4 * (int)kStoreWarpBytes + 1024;
     LORACT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
     cudaLaunchConfig_t q = {};
     q.gridDim = dim3(2); q.blockDim = dim3(kThreads); q.dynamicSmemBytes = smem_max;
@@ -913,7 +1080,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   p.accumulate = g.accumulate ? 1 : 0;
   p.ep_E = g.ep_E; p.ep_ld = g.ep_ld; p.ep_row_a = g.ep_row_a; p.ep_row_b = g.ep_row_b; p.ep_col = g.ep_col;
   p.dev_status = dev_status;
-  p.st_m_tiles = 0; p.st_units = 0;
+  p.st_m_tiles = 0; p.st_units = 0; p.tma_store = 0;
 
   TmapPack maps;
   for (int t = 0; t < g.n_terms; ++t) {
@@ -923,6 +1090,26 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
     else LORACT_CUDA_TRY(get_tmap(g.terms[t].B, g.K, g.N, g.ldb, 64, (uint32_t)b_rows, &maps.b[t]));
   }
   for (int t = g.n_terms; t < 3; ++t) { maps.a[t] = maps.a[0]; maps.b[t] = maps.b[0]; }
+  maps.c[0] = maps.a[0]; maps.c[1] = maps.a[0];
+  if (splits == 1) p.split_stride = 0;
+  // Output maps for the staged epilogue (boxes of 128 bytes x 32 rows).  Split-K partials are stacked along the
+  // rows of one map, which needs them back to back in memory.
+  auto staged_ok = [&](int bn) {
+    const int es = g.out == OUT_F32 ? 4 : 2;
+    if (g.accumulate || bn % (128 / es)) return false;
+    if (((uintptr_t)g.C0 & 15) || (g.ldc * es) % 16) return false;
+    if (g.out == OUT_SPLIT && ((uintptr_t)g.C1 & 15)) return false;
+    if (splits > 1 && g.split_stride != (int64_t)g.M * g.ldc) return false;
+    if (g.out == OUT_RMS_BWD && (((uintptr_t)g.ep_E & 15) || ((uintptr_t)g.ep_col & 15) || g.ep_ld % 8)) return false;
+    return true;
+  };
+  auto make_out_maps = [&]() -> cudaError_t {
+    const int es = g.out == OUT_F32 ? 4 : 2;
+    const uint32_t box = (uint32_t)(128 / es);
+    LORACT_CUDA_TRY(get_tmap(g.C0, g.N, (uint64_t)splits * g.M, g.ldc, box, 32, &maps.c[0], es));
+    if (g.out == OUT_SPLIT) LORACT_CUDA_TRY(get_tmap(g.C1, g.N, g.M, g.ldc, box, 32, &maps.c[1], es));
+    return cudaSuccess;
+  };
 
   // Short contraction, large output, A K-major, B MN-major, one term (Reconstruct and the pre-norm backward):
   // the persistent kernel with B resident, when there is more than one tile per resident pair.
@@ -936,10 +1123,14 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
     const long long units = (long long)sp.st_m_tiles * ((g.N + sp.bn - 1) / sp.bn);
     if (units >= 148 && units < (1ll << 30)) {
       sp.st_units = (int)units;
-      const size_t ssmem = (size_t)sp.kb_total * sp.b_bytes + (size_t)kStreamStages * kABytes + 1024;
+      sp.tma_store = staged_ok(sp.bn) ? 1 : 0;
+      if (sp.tma_store) LORACT_CUDA_TRY(make_out_maps());
+      const size_t ssmem = (size_t)sp.kb_total * sp.b_bytes + (size_t)kStreamStages * kABytes + 4 * kStoreWarpBytes + 1024;
       return launch_stream(maps, sp, ssmem, stream);
     }
   }
+  p.tma_store = staged_ok(p.bn) ? 1 : 0;
+  if (p.tma_store) LORACT_CUDA_TRY(make_out_maps());
   if (pair) {
     dim3 pgrid(2 * ((g.M + 2 * kBM - 1) / (2 * kBM)), (g.N + p.bn - 1) / p.bn, splits);
     const size_t psmem = (size_t)kPairStages * (kABytes + p.b_bytes) + 1024;
