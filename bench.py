@@ -141,8 +141,9 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="loract", choices=["loract", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--kernel-only", action="store_true",
-                    help="run only the dominant kernel (pass 1) a few times: the small case for profiler captures")
+    ap.add_argument("--kernel-only", nargs="?", const="pass1", default=None, choices=["pass1", "reconstruct"],
+                    help="run only one kernel a few times (pass 1 of Algorithm 1, or Reconstruct): the small case "
+                         "for profiler captures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "loract" else args.warmup
     if args.impl == "reference":
@@ -214,9 +215,14 @@ def main():
 
     if args.kernel_only:
         Om = torch.randn(r, d, device=dev).to(X.dtype)
+        Uk = torch.randn(N, r, device=dev).to(X.dtype)
+        Xt = torch.empty_like(X)
         for _ in range(args.warmup + args.steps):
             flush.zero_()
-            B.debug_gemm([X], [Om], N, r, d, False, False, out_mode=B.OUT_SPLIT, engine=1)
+            if args.kernel_only == "pass1":
+                B.debug_gemm([X], [Om], N, r, d, False, False, out_mode=B.OUT_SPLIT, engine=1)
+            else:
+                B.reconstruct(Uk, Om, out=Xt)
         torch.cuda.synchronize()
         print(json.dumps({"kernel_only": True, "launches": args.warmup + args.steps}))
         return

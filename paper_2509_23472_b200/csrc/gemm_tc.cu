@@ -26,7 +26,8 @@ namespace {
 constexpr int kBM = 128;
 constexpr int kBK = 64;          // bf16 elements = one 128-byte swizzle row
 constexpr int kStages = 4;
-constexpr int kThreads = 192;    // warp 0: TMA, warp 1: MMA + tensor memory, warps 2..5: epilogue
+constexpr int kThreads = 320;    // warp 0: TMA, warp 1: MMA + tensor memory, warps 2..9: epilogue
+constexpr int kEpiWarps = 8;     // two per quarter of the tensor-memory lanes: they take alternate column groups
 constexpr uint32_t kABytes = kBM * kBK * 2;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
 
@@ -157,8 +158,10 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // instructions.  Instead each epilogue warp puts its 32 rows x 128 bytes into shared memory in the layout of a
 // 128-byte-swizzled TMA box (conflict free: the 16-byte chunk c of row i goes to chunk c ^ (i & 7)) and one
 // lane sends the box with a TMA store, which writes whole lines and clips at the edges of the output.  Each
-// warp cycles through kStoreBufs boxes of its own, so no barrier between warps is needed.
-constexpr int kStoreBufs = 4;
+// warp cycles through kStoreBufs boxes of its own, so no barrier between warps is needed.  Two warps share each
+// quarter of the accumulator rows (a warp may only read the tensor-memory lanes 32 * (warp % 4) .. + 31); they
+// take alternate column groups.
+constexpr int kStoreBufs = 2;
 constexpr uint32_t kStoreBoxBytes = 4096;                    // 32 rows x 128 bytes
 constexpr uint32_t kStoreWarpBytes = kStoreBufs * kStoreBoxBytes;
 
@@ -206,14 +209,14 @@ __device__ __forceinline__ void stage_drain(const StoreStage& st, int lane) {
 }
 
 __device__ __forceinline__ void tc_store_tile_staged(const TcParams& p, const TmapPack& maps, uint32_t tmem_base,
-                                                     int quad, int lane, int m0, int n0, int split,
-                                                     StoreStage& st) {
+                                                     int quad, int half_id, int lane, int m0, int n0,
+                                                     int split, StoreStage& st) {
   const int row0 = m0 + quad * 32;
   const int m = row0 + lane;
   const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
   const int y = split * p.M + row0;
   if (p.out == OUT_F32) {
-    for (int c0 = 0; c0 < p.bn && n0 + c0 < p.N; c0 += 32) {
+    for (int c0 = 32 * half_id; c0 < p.bn && n0 + c0 < p.N; c0 += 64) {
       uint32_t v[32];
       tc_ld32(taddr + (uint32_t)c0, v);
       tc_wait_ld();
@@ -231,7 +234,7 @@ __device__ __forceinline__ void tc_store_tile_staged(const TcParams& p, const Tm
   const bool live = m < p.M;                                 // rows past M are clipped by the store
   float ra = 0.f, rb = 0.f;
   if (rms && live) { ra = p.ep_row_a[m]; rb = p.ep_row_b[m]; }
-  for (int c0 = 0; c0 < p.bn && n0 + c0 < p.N; c0 += 64) {
+  for (int c0 = 64 * half_id; c0 < p.bn && n0 + c0 < p.N; c0 += 128) {
     if (split_out) stage_acquire<2>(st, lane); else stage_acquire<1>(st, lane);
     unsigned char* box_hi = stage_box(st, 0);
     unsigned char* box_lo = stage_box(st, 1);
@@ -257,7 +260,8 @@ __device__ __forceinline__ void tc_store_tile_staged(const TcParams& p, const Tm
               const float e0 = __uint_as_float(ew[h] << 16), e1 = __uint_as_float(ew[h] & 0xffff0000u);
               const float c0f = __uint_as_float(cw[h] << 16), c1f = __uint_as_float(cw[h] & 0xffff0000u);
               const float a0 = __uint_as_float(v[8 * q + 2 * h]), a1 = __uint_as_float(v[8 * q + 2 * h + 1]);
-              ow[h] = pack_bf16x2(ra * c0f * e0 - rb * a0 / c0f, ra * c1f * e1 - rb * a1 / c1f);
+              // the quotient is rounded to bf16 below: the fast division (2 ulp in fp32) is exact enough
+              ow[h] = pack_bf16x2(ra * c0f * e0 - __fdividef(rb * a0, c0f), ra * c1f * e1 - __fdividef(rb * a1, c1f));
             }
           } else if (live) {
             for (int h = 0; h < 8; ++h) {
@@ -272,22 +276,28 @@ __device__ __forceinline__ void tc_store_tile_staged(const TcParams& p, const Tm
           }
           stage_write16(box_hi, lane, 4 * half + q, make_uint4(ow[0], ow[1], ow[2], ow[3]));
         }
+      } else if (!split_out) {
+        // one conversion instruction per pair of columns: this loop runs on a single warp per scheduler, so
+        // its length in instructions is its duration
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          stage_write16(box_hi, lane, 4 * half + q,
+                        make_uint4(pack_bf16x2(__uint_as_float(v[8 * q]), __uint_as_float(v[8 * q + 1])),
+                                   pack_bf16x2(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3])),
+                                   pack_bf16x2(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5])),
+                                   pack_bf16x2(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7]))));
       } else {
         uint32_t hi[16], lo[16];
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
           const float x0 = __uint_as_float(v[2 * q]), x1 = __uint_as_float(v[2 * q + 1]);
-          const __nv_bfloat16 h0 = __float2bfloat16(x0), h1 = __float2bfloat16(x1);
-          hi[q] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-          lo[q] = pack_bf16x2(x0 - __bfloat162float(h0), x1 - __bfloat162float(h1));
+          hi[q] = pack_bf16x2(x0, x1);
+          lo[q] = pack_bf16x2(x0 - __uint_as_float(hi[q] << 16), x1 - __uint_as_float(hi[q] & 0xffff0000u));
         }
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
+        for (int q = 0; q < 4; ++q) {
           stage_write16(box_hi, lane, 4 * half + q, make_uint4(hi[4 * q], hi[4 * q + 1], hi[4 * q + 2], hi[4 * q + 3]));
-        if (split_out) {
-#pragma unroll
-          for (int q = 0; q < 4; ++q)
-            stage_write16(box_lo, lane, 4 * half + q, make_uint4(lo[4 * q], lo[4 * q + 1], lo[4 * q + 2], lo[4 * q + 3]));
+          stage_write16(box_lo, lane, 4 * half + q, make_uint4(lo[4 * q], lo[4 * q + 1], lo[4 * q + 2], lo[4 * q + 3]));
         }
       }
     }
@@ -302,17 +312,18 @@ __device__ __forceinline__ void tc_store_tile_staged(const TcParams& p, const Tm
 __device__ __forceinline__ void tc_store_tile(const TcParams& p, const TmapPack& maps, uint32_t tmem_base, int warp,
                                               int lane, int m0, int n0, int split, StoreStage& st) {
   const int quad = warp & 3;
+  const int half_id = (warp - 2) >> 2;                       // which of the two warps of this quarter
   const int row = quad * 32 + lane;
   const int m = m0 + row;
   if (m0 + quad * 32 >= p.M) return;                         // none of this warp's rows exists
   // staged unless the output needs read-modify-write, or (split-K partials stacked along the rows of one
   // tensor map) the warp's 32 rows are not all inside M
   if (st.base && p.tma_store && !p.accumulate && (p.split_stride == 0 || m0 + quad * 32 + 32 <= p.M)) {
-    tc_store_tile_staged(p, maps, tmem_base, quad, lane, m0, n0, split, st);
+    tc_store_tile_staged(p, maps, tmem_base, quad, half_id, lane, m0, n0, split, st);
     return;
   }
   {
-    for (int c0 = 0; c0 < p.bn; c0 += 32) {
+    for (int c0 = 32 * half_id; c0 < p.bn; c0 += 64) {
       uint32_t v[32];
       tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
       tc_wait_ld();
@@ -394,9 +405,9 @@ __device__ __forceinline__ void tc_store_tile(const TcParams& p, const TmapPack&
   }
 }
 
-// Epilogue of one CTA (four warps) of the one-tile kernels: waits for the accumulator, then writes it.
+// Epilogue of one CTA (eight warps) of the one-tile kernels: waits for the accumulator, then writes it.
 // `ring` is the operand ring: once the accumulator is complete every load has landed and every MMA has read
-// its stage, so the epilogue warps take the ring over as staging space (16 KB per warp).
+// its stage, so the epilogue warps take the ring over as staging space (8 KB per warp).
 __device__ __forceinline__ void tc_epilogue(const TcParams& p, const TmapPack& maps, uint32_t tmem_base,
                                           uint64_t* accum_bar, volatile int* abort_flag_ptr, int warp, int lane,
                                           int m0, int n0, int split, int n_iter, unsigned char* ring) {
@@ -406,11 +417,11 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const TmapPack& m
   tc_fence_after();
   if (ok && n_iter > 0) {
     StoreStage st;
-    st.base = ring + (uint32_t)(warp & 3) * kStoreWarpBytes;
+    st.base = ring + (uint32_t)(warp - 2) * kStoreWarpBytes;
     st.cnt = 0;
     tc_store_tile(p, maps, tmem_base, warp, lane, m0, n0, split, st);
     stage_drain(st, lane);
-  } else if (ok && n_iter == 0 && m < p.M && p.out == OUT_F32) {
+  } else if (ok && n_iter == 0 && m < p.M && p.out == OUT_F32 && warp < 6) {
     // an empty K range still owns its partial: write zeros
     float* dst = (float*)p.C0 + (int64_t)split * p.split_stride + (int64_t)m * p.ldc + n0;
     for (int q = 0; q < min(p.bn, p.N - n0); ++q) dst[q] = 0.f;
@@ -688,11 +699,11 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
 //   * its half of the B tile (all K blocks) stays in shared memory while the column tile does not change;
 //     only A is streamed through a ring of 128 x 64 stages;
 //   * the accumulator is double buffered in tensor memory (2 x bn columns): the tensor cores work on tile
-//     i + 1 while the four epilogue warps read and store tile i.
+//     i + 1 while the eight epilogue warps read and store tile i.
 // Barriers.  a_full / a_empty: the ring, as in the pair kernel.  b_full (leader): both halves of B have
 // landed; b_empty (each CTA, by commit): every MMA that reads the resident B is done, it may be replaced.
-// acc_full[j] (each CTA, by commit): buffer j holds a finished tile; acc_empty[j] (leader, 8 arrivals: the
-// four epilogue warps of both CTAs): buffer j has been read in both CTAs.  No load uses cluster multicast.
+// acc_full[j] (each CTA, by commit): buffer j holds a finished tile; acc_empty[j] (leader, 16 arrivals: the
+// eight epilogue warps of both CTAs): buffer j has been read in both CTAs.  No load uses cluster multicast.
 constexpr int kStreamStages = 6;
 
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
@@ -749,7 +760,7 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
     for (int s = 0; s < kStreamStages; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1); }
     mbar_init(&b_full, 1);
     mbar_init(&b_empty, 1);
-    for (int j = 0; j < 2; ++j) { mbar_init(&acc_full[j], 1); mbar_init(&acc_empty[j], 8); }
+    for (int j = 0; j < 2; ++j) { mbar_init(&acc_full[j], 1); mbar_init(&acc_empty[j], 2 * kEpiWarps); }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -841,7 +852,7 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   } else {
     bool ok = true;
     StoreStage st;
-    st.base = ring + (size_t)kStreamStages * kABytes + (uint32_t)(warp & 3) * kStoreWarpBytes;
+    st.base = ring + (size_t)kStreamStages * kABytes + (uint32_t)(warp - 2) * kStoreWarpBytes;
     st.cnt = 0;
     for (int u = u_begin, ui = 0; u < u_end; ++u, ++ui) {
       const int j = ui & 1;
@@ -993,7 +1004,7 @@ cudaError_t launch_stream(const TmapPack& maps, TcParams p, size_t smem, cudaStr
   const bool cached = dev >= 0 && dev < 64 && configured[dev];
   int pairs = cached ? max_pairs[dev] : 0;
   if (!cached) {
-    const int smem_max = 8 * 8192 + kStreamStages * (int)kABytes + 4 * (int)kStoreWarpBytes + 1024;
+    const int smem_max = 8 * 8192 + kStreamStages * (int)kABytes + kEpiWarps * (int)kStoreWarpBytes + 1024;
     LORACT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
     cudaLaunchConfig_t q = {};
     q.gridDim = dim3(2); q.blockDim = dim3(kThreads); q.dynamicSmemBytes = smem_max;
@@ -1125,7 +1136,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
       sp.st_units = (int)units;
       sp.tma_store = staged_ok(sp.bn) ? 1 : 0;
       if (sp.tma_store) LORACT_CUDA_TRY(make_out_maps());
-      const size_t ssmem = (size_t)sp.kb_total * sp.b_bytes + (size_t)kStreamStages * kABytes + 4 * kStoreWarpBytes + 1024;
+      const size_t ssmem = (size_t)sp.kb_total * sp.b_bytes + (size_t)kStreamStages * kABytes + kEpiWarps * kStoreWarpBytes + 1024;
       return launch_stream(maps, sp, ssmem, stream);
     }
   }
