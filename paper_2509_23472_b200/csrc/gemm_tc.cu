@@ -92,12 +92,16 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // Bounded wait.  Returns false if the limit expired (or another role already gave up).
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
+  // the wall clock is read only once in a while, and first after 1024 failed polls: a read of %globaltimer is
+  // slow enough to matter on the hand-offs of the operand ring, which all pass through here
+  uint64_t t0 = 0;
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((spin & 255u) == 0u) {
+    if ((spin & 1023u) == 0u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      const uint64_t now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
     }
   }
 }
@@ -702,12 +706,18 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
 //     i + 1 while the eight epilogue warps read and store tile i.
 // Barriers.  a_full / a_empty: the ring, as in the pair kernel.  b_full (leader): both halves of B have
 // landed; b_empty (each CTA, by commit): every MMA that reads the resident B is done, it may be replaced.
-// acc_full[j] (each CTA, by commit): buffer j holds a finished tile; acc_empty[j] (leader, 16 arrivals: the
-// eight epilogue warps of both CTAs): buffer j has been read in both CTAs.  No load uses cluster multicast.
+// acc_full[j] (each CTA, by commit): buffer j holds a finished tile; acc_empty[j] (leader, one arrival
+// per CTA, sent by the first epilogue warp once all eight have arrived on the CTA's own epi_done[j]): buffer j has been read in both CTAs.  No load uses cluster multicast.
 constexpr int kStreamStages = 6;
 
+// An arrival on a barrier of the peer CTA.  Relaxed: it announces that tensor-memory reads have completed
+// (tcgen05.wait::ld has returned), no memory written by this thread has to become visible with it, and a
+// releasing arrival at cluster scope costs most of a microsecond.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_local(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
@@ -722,12 +732,14 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
 }
 __device__ __forceinline__ bool mbar_wait_cluster_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait_cluster(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
+  uint64_t t0 = 0;
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try_wait_cluster(bar, parity)) return true;
-    if ((spin & 255u) == 0u) {
+    if ((spin & 1023u) == 0u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      const uint64_t now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
     }
   }
 }
@@ -740,6 +752,7 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   __shared__ __align__(8) uint64_t b_full, b_empty;
   __shared__ __align__(8) uint64_t acc_full[2];
   __shared__ __align__(8) uint64_t acc_empty[2];
+  __shared__ __align__(8) uint64_t epi_done[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
@@ -760,7 +773,11 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
     for (int s = 0; s < kStreamStages; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1); }
     mbar_init(&b_full, 1);
     mbar_init(&b_empty, 1);
-    for (int j = 0; j < 2; ++j) { mbar_init(&acc_full[j], 1); mbar_init(&acc_empty[j], 2 * kEpiWarps); }
+    for (int j = 0; j < 2; ++j) {
+      mbar_init(&acc_full[j], 1);
+      mbar_init(&acc_empty[j], 2);
+      mbar_init(&epi_done[j], kEpiWarps);
+    }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -866,7 +883,17 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
       // the tile is in registers / shared memory now: hand the buffer back before the stores have drained
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&acc_empty[j]), 0u));
+      if (lane == 0) {
+        mbar_arrive_local(&epi_done[j]);
+        if (warp == 2) {
+          // one signal per CTA and tile: the first epilogue warp collects the eight and tells the leader
+          if (mbar_wait_bounded(&epi_done[j], (uint32_t)((ui >> 1) & 1), &abort_flag)) {
+            if (leader) mbar_arrive_local(&acc_empty[j]);
+            else mbar_arrive_cluster(map_to_rank(smem_u32(&acc_empty[j]), 0u));
+          }
+        }
+      }
+      __syncwarp();
     }
     stage_drain(st, lane);
   }
