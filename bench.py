@@ -153,7 +153,7 @@ def main():
     import torch
     import __graft_entry__ as entry
     from paper_2509_23472_b200 import binding as B
-    from paper_2509_23472_b200 import synth
+    from paper_2509_23472_b200 import dp, synth
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -174,13 +174,12 @@ def main():
 
     w = synth.get_workload(args.workload)
     # data-parallel replicas: every rank draws its own batch and samples its own rows
-    w_rank = synth.scaled(w, name=w.name) if rank == 0 else \
-        synth.Workload(**{**w.__dict__, "seed": w.seed + 7919 * rank})
+    w_rank = dp.rank_workload(w, rank)
     inp = synth.make_inputs(w_rank, device=dev)
     X, G = inp["X"], inp["G"]
     N, d, r, g = w.n_tokens, w.d, w.rank, w.g
     es = w.elem_bytes
-    desc = B.make_desc(X, r, seed=w_rank.seed, call_id=rank)
+    desc = B.make_desc(X, r, seed=w_rank.seed, call_id=dp.rank_call_id(rank))
     ws = B.alloc_workspace(desc, dev)
     U = torch.empty(N, r, dtype=X.dtype, device=dev)
     V = torch.empty(r, d, dtype=X.dtype, device=dev)
@@ -323,10 +322,7 @@ def main():
         k_times = timed(pass1_group, 6)
         k_ms = statistics.mean(k_times) / group
 
-    if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
+    total_ms, e2e_ms = dp.max_over_ranks([total_ms, e2e_ms], dist, dev)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -335,8 +331,8 @@ def main():
     peaks = measured_peaks()
     ms_per_step = total_ms / args.steps
     x_bytes = N * d * es
-    value = world * x_bytes / (ms_per_step * 1e-3) / 1e9
-    e2e_value = world * x_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9
+    value = dp.whole_job_gbs(world, x_bytes, ms_per_step)
+    e2e_value = dp.whole_job_gbs(world, x_bytes, e2e_ms / e2e_steps)
     # algorithmic bytes of pass 1: X read once, the test matrix read once, Y written once as a bf16 pair
     k_bytes = N * d * es + r * d * es + N * r * 4
     roofline = None

@@ -1,0 +1,67 @@
+"""The N > 1 layout of the benchmark on a CPU process group (gloo, world size 2).
+
+The hot path shards by batch with no collective, so what there is to check across ranks is the bookkeeping:
+every rank draws a batch and a row sample of its own, rank 0 keeps the single-GPU workload, and the per-rank
+times become one whole-job number through a maximum over ranks.  The row samples come from the oracle's
+sampler (the device's is checked bit for bit against it in the GPU tests)."""
+import os
+import socket
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from oracle import loract_oracle as orc
+from paper_2509_23472_b200 import dp, synth
+
+
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank: int, world: int, port: int, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        base = synth.scaled(synth.get_workload("llama7b_block"), n_tokens=256, d=64, rank=16, signal_rank=32)
+        w = dp.rank_workload(base, rank)
+        X = synth.make_inputs(w)["X"]
+        idx = torch.from_numpy(orc.sample_indices(w.n_tokens, w.rank, w.seed, dp.rank_call_id(rank)).astype(np.int64))
+        head = X[:4, :8].float().contiguous()
+        idxs = [torch.empty_like(idx) for _ in range(world)]
+        heads = [torch.empty_like(head) for _ in range(world)]
+        dist.all_gather(idxs, idx)
+        dist.all_gather(heads, head)
+        # per-rank step times: rank r is the slowest in entry r
+        times = [1.0 + (rank == 0), 1.0 + (rank == 1)]
+        agg = dp.max_over_ranks(times, dist)
+        out[rank] = dict(seed=w.seed, idx_differ=not torch.equal(idxs[0], idxs[1]),
+                         data_differ=not torch.equal(heads[0], heads[1]),
+                         rank0_is_base=(w.seed == base.seed) if rank == 0 else None, agg=agg,
+                         shape=(w.n_tokens, w.d, w.rank))
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_get_their_own_batches_and_one_whole_job_number():
+    world = 2
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_worker, args=(world, _free_port(), out), nprocs=world, join=True)
+        res = {k: dict(v) for k, v in out.items()}
+    assert set(res) == {0, 1}
+    assert res[0]["rank0_is_base"] is True
+    assert res[1]["seed"] - res[0]["seed"] == dp.SEED_STRIDE
+    for r in (0, 1):
+        assert res[r]["idx_differ"] and res[r]["data_differ"]
+        assert res[r]["agg"] == [2.0, 2.0]            # the maximum over ranks, seen by every rank
+        assert res[r]["shape"] == (256, 64, 16)       # weak scaling: the per-rank shape does not change
+    # whole-job throughput: both ranks' bytes over the slowest rank's time
+    assert dp.whole_job_gbs(2, 10 ** 9, 1000.0) == 2.0
+    # without a process group the aggregate is the identity
+    assert dp.max_over_ranks([3.0, 1.5]) == [3.0, 1.5]
