@@ -308,19 +308,31 @@ __device__ __forceinline__ bool factor_diag_half(const float* slot, float* lcol,
                          c0 + 2 * pp + 1 < lane ? slot[lane * kLd + c0 + 2 * pp + 1] : 0.f);
   float diag = slot[lane * kLd + lane];   // used by the lanes whose diagonal lies in this warp's columns
   if (half == 1) {
+    // Two columns per round trip: one column at a time costs a shared-memory latency for the word, one for
+    // the column and the dependent FMAs -- about 200 cycles against the 115 a pivot takes -- and this warp
+    // ended each block 1300 cycles behind the one it follows.  The updates of two columns commute (both use
+    // final values of L), and their loads overlap.
 #pragma unroll
-    for (int k = 0; k < kHalf; ++k) {
-      const float v = wait_word(lcol + k * kLcolLd + lane, gave_up);
-      const float lik = (lane >= kHalf) ? v : 0.f;   // L[lane][k]
+    for (int k = 0; k < kHalf; k += 2) {
+      const float v0 = wait_word(lcol + k * kLcolLd + lane, gave_up);
+      const float v1 = wait_word(lcol + (k + 1) * kLcolLd + lane, gave_up);
+      const float l0 = (lane >= kHalf) ? v0 : 0.f;   // L[lane][k]
+      const float l1 = (lane >= kHalf) ? v1 : 0.f;   // L[lane][k + 1]
       __syncwarp();
-      const float2 nl = make_float2(-lik, -lik);
-      const float4* col = reinterpret_cast<const float4*>(lcol + k * kLcolLd + kHalf);
-      diag = fmaf(-lik, lik, diag);
+      const float2 n0 = make_float2(-l0, -l0), n1 = make_float2(-l1, -l1);
+      const float4* c0p = reinterpret_cast<const float4*>(lcol + k * kLcolLd + kHalf);
+      const float4* c1p = reinterpret_cast<const float4*>(lcol + (k + 1) * kLcolLd + kHalf);
+      float4 la[kHalf / 4], lb[kHalf / 4];
+#pragma unroll
+      for (int q = 0; q < kHalf / 4; ++q) { la[q] = c0p[q]; lb[q] = c1p[q]; }
+      diag = fmaf(-l0, l0, diag);
+      diag = fmaf(-l1, l1, diag);
 #pragma unroll
       for (int q = 0; q < kHalf / 4; ++q) {
-        const float4 l = col[q];
-        a2[2 * q] = __ffma2_rn(nl, make_float2(l.x, l.y), a2[2 * q]);
-        a2[2 * q + 1] = __ffma2_rn(nl, make_float2(l.z, l.w), a2[2 * q + 1]);
+        a2[2 * q] = __ffma2_rn(n0, make_float2(la[q].x, la[q].y), a2[2 * q]);
+        a2[2 * q + 1] = __ffma2_rn(n0, make_float2(la[q].z, la[q].w), a2[2 * q + 1]);
+        a2[2 * q] = __ffma2_rn(n1, make_float2(lb[q].x, lb[q].y), a2[2 * q]);
+        a2[2 * q + 1] = __ffma2_rn(n1, make_float2(lb[q].z, lb[q].w), a2[2 * q + 1]);
       }
     }
   }
