@@ -158,6 +158,7 @@ cudaError_t gram_rows(const void* S, int l, int64_t d, bool bf16, const BasisWs&
   return run_gemm(g, status, stream);
 }
 
+constexpr int kReduceFirst = 8;    // partial count from which a separate, all-SM reduction pays
 cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs& w, uint32_t* status,
                    cudaStream_t stream) {
   SmallBlockArgs a;
@@ -167,6 +168,14 @@ cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs&
   if (bf16) {
     a.partials = w.gram_partials; a.partial_type = ELEM_F32; a.n_partials = n_partials;
     a.partial_stride = (int64_t)l * l;
+    if (l <= 256 && n_partials >= kReduceFirst) {
+      // The factorisation runs on eight SMs; summing many partials there is a read of several MB through
+      // eight SMs' worth of bandwidth.  All SMs sum them first (same order of additions, so the same bits).
+      float* W = (float*)w.sb_scratch;
+      LORACT_CUDA_TRY(reduce_partials_launch(w.gram_partials, n_partials, a.partial_stride, (int64_t)l * l, W, nullptr,
+                                             stream));
+      a.partials = W; a.n_partials = 1; a.partial_stride = 0;
+    }
     a.use_f64 = false; a.shift_rel = shift;
     a.linv_hi = w.Lh; a.linv_lo = w.Ll;
   } else {
