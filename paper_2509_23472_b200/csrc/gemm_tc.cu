@@ -625,33 +625,42 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   pdl_wait();
   pdl_launch_dependents();
 
-  if (warp == 0) {
+  if (warp == 0 || warp == 2) {
     if (lane == 0) {
       const int nb0 = n0 + (int)cta_rank * half_n;           // this CTA's half of the B tile
-      for (int it = 0; it < n_iter; ++it) {
-        const int s = it % kPairStages;
-        if (!mbar_wait_bounded(&empty_bar[s], ((it / kPairStages) & 1) ^ 1, &abort_flag)) break;
-        const int term = it / kb_count;
-        const int k0 = (kb_begin + (it - term * kb_count)) * kBK;
+      // stage, parity, term and K block are carried along (no division in the loop)
+      int s = (warp == 0 ? 0 : 1) % kPairStages;
+      uint32_t parity = 1u;
+      int term = 0, kb = (warp == 0 ? 0 : 1);
+      while (kb >= kb_count && kb_count > 0) { kb -= kb_count; ++term; }
+      for (int it = (warp == 0 ? 0 : 1); it < n_iter; it += 2) {
+        if (!mbar_wait_bounded(&empty_bar[s], parity, &abort_flag)) break;
+        const int k0 = (kb_begin + kb) * kBK;
         unsigned char* a_dst = tiles + (size_t)s * stage_bytes;
         unsigned char* b_dst = a_dst + kABytes;
         // the leader expects the bytes of both CTAs on its barrier
         if (leader) mbar_arrive_expect_tx(&full_bar[s], 2u * stage_bytes);
         const uint32_t bar = map_to_rank(smem_u32(&full_bar[s]), 0u);
+        const int term_now = term;
+        s += 2; if (s >= kPairStages) { s -= kPairStages; parity ^= 1u; }
+        kb += 2; if (kb >= kb_count) { kb -= kb_count; ++term; if (kb >= kb_count) { kb -= kb_count; ++term; } }
         if (A_MN) {
-          tma_load_2d_pair(a_dst, &maps.a[term], bar, m0, k0);
-          tma_load_2d_pair(a_dst + 8192, &maps.a[term], bar, m0 + 64, k0);
+          tma_load_2d_pair(a_dst, &maps.a[term_now], bar, m0, k0);
+          tma_load_2d_pair(a_dst + 8192, &maps.a[term_now], bar, m0 + 64, k0);
         } else {
-          tma_load_2d_pair(a_dst, &maps.a[term], bar, k0, m0);
+          tma_load_2d_pair(a_dst, &maps.a[term_now], bar, k0, m0);
         }
         if (B_MN) {
           for (uint32_t q = 0; q * 8192u < p.b_bytes; ++q)
-            tma_load_2d_pair(b_dst + q * 8192u, &maps.b[term], bar, nb0 + (int)q * 64, k0);
+            tma_load_2d_pair(b_dst + q * 8192u, &maps.b[term_now], bar, nb0 + (int)q * 64, k0);
         } else {
-          tma_load_2d_pair(b_dst, &maps.b[term], bar, k0, nb0);
+          tma_load_2d_pair(b_dst, &maps.b[term_now], bar, k0, nb0);
         }
       }
     }
+    __syncwarp();
+  }
+  if (warp == 0) {
   } else if (warp == 1) {
     if (lane == 0 && leader) {
       // instruction descriptor: fp32 accumulator, bf16 A and B, operand majors, N >> 3, M = 256 >> 4
@@ -659,12 +668,14 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
                              ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(p.bn >> 3) << 17) |
                              ((uint32_t)((2 * kBM) >> 4) << 24);
       bool ok = true;
+      int s = 0;
+      uint32_t parity = 0u;
+      const uint32_t tiles_u32 = smem_u32(tiles);
       for (int it = 0; it < n_iter && ok; ++it) {
-        const int s = it % kPairStages;
-        ok = mbar_wait_bounded(&full_bar[s], (it / kPairStages) & 1, &abort_flag);
+        ok = mbar_wait_bounded(&full_bar[s], parity, &abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t a_addr = smem_u32(tiles + (size_t)s * stage_bytes);
+        const uint32_t a_addr = tiles_u32 + (uint32_t)s * stage_bytes;
         const uint32_t b_addr = a_addr + kABytes;
         const uint64_t a_desc = make_smem_desc(a_addr, A_MN);
         const uint64_t b_desc = make_smem_desc(b_addr, B_MN);
@@ -675,6 +686,7 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
           tc_mma_bf16_pair(tmem_base, a_k, b_k, idesc, (it > 0 || k > 0) ? 1u : 0u);
         }
         tc_commit_pair(&empty_bar[s]);   // frees the stage in both CTAs once these MMAs have read it
+        if (++s == kPairStages) { s = 0; parity ^= 1u; }
       }
       tc_commit_pair(&accum_bar);        // accumulator complete in both CTAs (or nothing was issued)
     }

@@ -112,3 +112,40 @@ def test_persistent_form_for_short_contractions_with_a_large_output(dev, M, N, K
     tol = (2.0 ** -8 if out_mode == "bf16" else 2e-5 * max(1.0, (K / 64) ** 0.5)) * scale
     assert float((C.double() - ref).abs().max()) <= tol
     assert torch.equal(C, C1)
+
+
+@pytest.mark.parametrize("a_mn,b_mn,M,N,K,splits", [(True, True, 256, 256, 4096, 8),      # Gram of a hi/lo pair
+                                                    (False, False, 1024, 256, 256, 1),   # apply L^-T
+                                                    (False, True, 256, 1024, 256, 1)])   # Omega = L^-1 T
+@pytest.mark.parametrize("pattern", ["hl3", "a2", "b2"])
+def test_terms_that_share_operands(dev, a_mn, b_mn, M, N, K, splits, pattern):
+    # hi/lo products repeat operands: (Ah Bh + Ah Bl + Al Bh), (A0 B + A1 B), (A B0 + A B1).  The two-CTA form
+    # then loads every distinct operand once per K block and issues all the products from that stage; the result
+    # must be the definition, and agree with the one-CTA form (which runs the terms one after the other) to
+    # fp32 rounding of a different order of additions.
+    g = torch.Generator(device=dev)
+    g.manual_seed(17)
+    mk_a = lambda: torch.randn((K, M) if a_mn else (M, K), generator=g, device=dev).bfloat16()
+    mk_b = lambda: torch.randn((K, N) if b_mn else (N, K), generator=g, device=dev).bfloat16()
+    A0, A1, B0, B1 = mk_a(), (mk_a().float() * 2.0 ** -8).bfloat16(), mk_b(), (mk_b().float() * 2.0 ** -8).bfloat16()
+    if pattern == "hl3":
+        As, Bs = [A0, A0, A1], [B0, B1, B0]
+    elif pattern == "a2":
+        As, Bs = [A0, A1], [B0, B0]
+    else:
+        As, Bs = [A0, A0], [B0, B1]
+    ref = torch.zeros(M, N, dtype=torch.float64, device=dev)
+    for a, b in zip(As, Bs):
+        ref += (a.double().t() if a_mn else a.double()) @ (b.double() if b_mn else b.double().t())
+    out = {}
+    for pair in (True, False):
+        B.debug_set_pair_mode(pair)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        C = B.debug_gemm(As, Bs, M, N, K, a_mn, b_mn, out_mode=B.OUT_F32, splits=splits, status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        out[pair] = C.double().sum(0) if splits > 1 else C.double()
+    B.debug_set_pair_mode(True)
+    scale = float(ref.abs().max())
+    assert float((out[True] - ref).abs().max()) <= 1e-4 * scale
+    assert float((out[True] - out[False]).abs().max()) <= 1e-5 * scale
