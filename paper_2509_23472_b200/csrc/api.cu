@@ -311,12 +311,11 @@ cudaError_t compress_core(const loract_desc_t* desc, const void* X, int64_t ldx,
                           int32_t* idx_out, const CompressWs& w, const Plan& plan, cudaStream_t stream) {
   const bool bf16 = plan.bf16;
   const int r = desc->rank;
-  LORACT_CUDA_TRY(cudaMemsetAsync(w.status, 0, 4, stream));
-  // line 1: sample rows, gather them
+  // line 1: sample rows, gather them.  The sampler is the first kernel of the call: it clears the status word
+  // and writes the caller's copy of the indices itself.
   trace_label("sample");
   LORACT_CUDA_TRY(sample_indices_launch(desc->seed, desc->call_id, (uint32_t)desc->n_tokens, r, w.idx,
-                                        w.status, stream));
-  if (idx_out) LORACT_CUDA_TRY(cudaMemcpyAsync(idx_out, w.idx, (size_t)r * 4, cudaMemcpyDeviceToDevice, stream));
+                                        w.status, stream, idx_out, true));
   trace_label("gather");
   LORACT_CUDA_TRY(gather_rows_launch(X, ldx, w.idx, r, desc->d, elem_bytes(desc), w.S, stream));
   // Lines 2 to 7.  The test matrix (the sampled rows A_k at first, Q^T X in the power iterations of lines

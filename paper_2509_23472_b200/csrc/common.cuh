@@ -108,8 +108,11 @@ cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t stream);
 cudaError_t gemm_f32_small_launch(const GemmDesc& g, cudaStream_t stream);
 
 // ---------------------------------------------------------------- sampler and gather
+// idx_copy (optional) receives the same indices; clear_status: the kernel sets the status word instead of OR-ing
+// into it (for the first kernel of a call).
 cudaError_t sample_indices_launch(uint64_t seed, uint64_t call_id, uint32_t n_rows, int rank,
-                                  int32_t* idx_dev, uint32_t* dev_status, cudaStream_t stream);
+                                  int32_t* idx_dev, uint32_t* dev_status, cudaStream_t stream,
+                                  int32_t* idx_copy = nullptr, bool clear_status = false);
 // dst (rank x d, stride d) = src[idx, :] (stride ld); 16-byte loads.  elem_bytes 2 or 4.
 cudaError_t gather_rows_launch(const void* src, int64_t ld, const int32_t* idx, int rank, int64_t d,
                                int elem_bytes, void* dst, cudaStream_t stream);

@@ -38,7 +38,7 @@ constexpr int kTableSlots = 2048;
 __global__ void __launch_bounds__(kSamplerThreads)
 sample_indices_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_t call_lo, uint32_t call_hi,
                       uint32_t n_rows, int rank, int32_t* __restrict__ idx_out,
-                      uint32_t* __restrict__ dev_status) {
+                      int32_t* __restrict__ idx_copy, uint32_t* __restrict__ dev_status, int clear_status) {
   __shared__ uint32_t accepted[kMaxRank];
   __shared__ uint32_t tab_key[kTableSlots];   // value + 1, 0 = empty
   __shared__ uint32_t tab_pos[kTableSlots];   // smallest stream position of that value
@@ -83,8 +83,16 @@ sample_indices_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_t call_lo, uint
   }
   const int found = s_count;
   pdl_wait();   // the index array may still be read by the previous call's kernels
-  for (int j = tid; j < rank; j += kSamplerThreads) idx_out[j] = (j < found) ? (int32_t)accepted[j] : 0;
-  if (tid == 0 && found < rank && dev_status) atomicOr(dev_status, LORACT_DEV_SAMPLER_SHORT);
+  for (int j = tid; j < rank; j += kSamplerThreads) {
+    const int32_t v = (j < found) ? (int32_t)accepted[j] : 0;
+    idx_out[j] = v;
+    if (idx_copy) idx_copy[j] = v;     // the caller's copy: no separate copy node between this kernel and the gather
+  }
+  // first kernel of a call: it also clears the status word (no memset node in front of it)
+  if (tid == 0 && dev_status) {
+    if (clear_status) *dev_status = (found < rank) ? LORACT_DEV_SAMPLER_SHORT : 0u;
+    else if (found < rank) atomicOr(dev_status, LORACT_DEV_SAMPLER_SHORT);
+  }
 }
 
 // dst[row, :] = src[idx[row], :], 16 bytes per thread per step.
@@ -135,10 +143,11 @@ __global__ void gaussian_rows_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_
 }  // namespace
 
 cudaError_t sample_indices_launch(uint64_t seed, uint64_t call_id, uint32_t n_rows, int rank,
-                                  int32_t* idx_dev, uint32_t* dev_status, cudaStream_t stream) {
+                                  int32_t* idx_dev, uint32_t* dev_status, cudaStream_t stream, int32_t* idx_copy,
+                                  bool clear_status) {
   LORACT_CUDA_TRY(launch_pdl(sample_indices_kernel, dim3(1), dim3(kSamplerThreads), 0, stream, (uint32_t)seed,
                              (uint32_t)(seed >> 32), (uint32_t)call_id, (uint32_t)(call_id >> 32), n_rows, rank,
-                             idx_dev, dev_status));
+                             idx_dev, idx_copy, dev_status, clear_status ? 1 : 0));
   count_launch(__func__, stream);
   return cudaGetLastError();
 }
