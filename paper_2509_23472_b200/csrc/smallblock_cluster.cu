@@ -302,38 +302,53 @@ __device__ __forceinline__ bool factor_diag_half(const float* slot, float* lcol,
                                                  volatile int* gave_up, int half, int lane) {
   const int c0 = half * kHalf;
   float2 a2[kHalf / 2];   // row `lane`, columns (c0 + 2p, c0 + 2p + 1), below the diagonal only
-#pragma unroll
-  for (int pp = 0; pp < kHalf / 2; ++pp)
-    a2[pp] = make_float2(c0 + 2 * pp < lane ? slot[lane * kLd + c0 + 2 * pp] : 0.f,
-                         c0 + 2 * pp + 1 < lane ? slot[lane * kLd + c0 + 2 * pp + 1] : 0.f);
   float diag = slot[lane * kLd + lane];   // used by the lanes whose diagonal lies in this warp's columns
-  if (half == 1) {
-    // Two columns per round trip: one column at a time costs a shared-memory latency for the word, one for
-    // the column and the dependent FMAs -- about 200 cycles against the 115 a pivot takes -- and this warp
-    // ended each block 1300 cycles behind the one it follows.  The updates of two columns commute (both use
-    // final values of L), and their loads overlap.
+  if (half == 0) {
+#pragma unroll
+    for (int pp = 0; pp < kHalf / 2; ++pp)
+      a2[pp] = make_float2(2 * pp < lane ? slot[lane * kLd + 2 * pp] : 0.f,
+                           2 * pp + 1 < lane ? slot[lane * kLd + 2 * pp + 1] : 0.f);
+  } else {
+    // The following warp.  Rows 0..15 have nothing below the diagonal in the columns 16..31, so their lanes
+    // would idle: instead lane i and lane i - 16 share row i while the columns of the first warp are taken
+    // off (lane i its columns 16..23, lane i - 16 the columns 24..31), which halves the instructions per
+    // followed column -- this warp ran a thousand cycles behind the one it follows -- and the upper lanes
+    // collect the whole row with eight shuffles before their own pivots start.  Two columns are taken per
+    // round trip: the updates commute (both use final values of L) and their loads overlap.
+    const int row = lane | kHalf;
+    const int cb = kHalf + ((lane < kHalf) ? kHalf / 2 : 0);   // first of this lane's eight columns
+    float2 f[kHalf / 4];
+#pragma unroll
+    for (int pp = 0; pp < kHalf / 4; ++pp)
+      f[pp] = make_float2(cb + 2 * pp < row ? slot[row * kLd + cb + 2 * pp] : 0.f,
+                          cb + 2 * pp + 1 < row ? slot[row * kLd + cb + 2 * pp + 1] : 0.f);
 #pragma unroll
     for (int k = 0; k < kHalf; k += 2) {
-      const float v0 = wait_word(lcol + k * kLcolLd + lane, gave_up);
-      const float v1 = wait_word(lcol + (k + 1) * kLcolLd + lane, gave_up);
-      const float l0 = (lane >= kHalf) ? v0 : 0.f;   // L[lane][k]
-      const float l1 = (lane >= kHalf) ? v1 : 0.f;   // L[lane][k + 1]
+      const float l0 = wait_word(lcol + k * kLcolLd + row, gave_up);         // L[row][k]
+      const float l1 = wait_word(lcol + (k + 1) * kLcolLd + row, gave_up);   // L[row][k + 1]
       __syncwarp();
       const float2 n0 = make_float2(-l0, -l0), n1 = make_float2(-l1, -l1);
-      const float4* c0p = reinterpret_cast<const float4*>(lcol + k * kLcolLd + kHalf);
-      const float4* c1p = reinterpret_cast<const float4*>(lcol + (k + 1) * kLcolLd + kHalf);
-      float4 la[kHalf / 4], lb[kHalf / 4];
+      const float4* c0p = reinterpret_cast<const float4*>(lcol + k * kLcolLd + cb);
+      const float4* c1p = reinterpret_cast<const float4*>(lcol + (k + 1) * kLcolLd + cb);
+      const float4 la0 = c0p[0], la1 = c0p[1], lb0 = c1p[0], lb1 = c1p[1];
+      if (lane >= kHalf) diag = fmaf(-l1, l1, fmaf(-l0, l0, diag));
+      f[0] = __ffma2_rn(n0, make_float2(la0.x, la0.y), f[0]);
+      f[1] = __ffma2_rn(n0, make_float2(la0.z, la0.w), f[1]);
+      f[2] = __ffma2_rn(n0, make_float2(la1.x, la1.y), f[2]);
+      f[3] = __ffma2_rn(n0, make_float2(la1.z, la1.w), f[3]);
+      f[0] = __ffma2_rn(n1, make_float2(lb0.x, lb0.y), f[0]);
+      f[1] = __ffma2_rn(n1, make_float2(lb0.z, lb0.w), f[1]);
+      f[2] = __ffma2_rn(n1, make_float2(lb1.x, lb1.y), f[2]);
+      f[3] = __ffma2_rn(n1, make_float2(lb1.z, lb1.w), f[3]);
+    }
 #pragma unroll
-      for (int q = 0; q < kHalf / 4; ++q) { la[q] = c0p[q]; lb[q] = c1p[q]; }
-      diag = fmaf(-l0, l0, diag);
-      diag = fmaf(-l1, l1, diag);
-#pragma unroll
-      for (int q = 0; q < kHalf / 4; ++q) {
-        a2[2 * q] = __ffma2_rn(n0, make_float2(la[q].x, la[q].y), a2[2 * q]);
-        a2[2 * q + 1] = __ffma2_rn(n0, make_float2(la[q].z, la[q].w), a2[2 * q + 1]);
-        a2[2 * q] = __ffma2_rn(n1, make_float2(lb[q].x, lb[q].y), a2[2 * q]);
-        a2[2 * q + 1] = __ffma2_rn(n1, make_float2(lb[q].z, lb[q].w), a2[2 * q + 1]);
-      }
+    for (int pp = 0; pp < kHalf / 4; ++pp) {
+      // columns 24..31 of row `lane` come up from lane - 16 (the source lane wraps for the lower lanes,
+      // whose registers are cleared right after)
+      const float tx = __shfl_sync(0xffffffffu, f[pp].x, (lane + kHalf) & 31);
+      const float ty = __shfl_sync(0xffffffffu, f[pp].y, (lane + kHalf) & 31);
+      a2[pp] = (lane >= kHalf) ? f[pp] : make_float2(0.f, 0.f);
+      a2[kHalf / 4 + pp] = (lane >= kHalf) ? make_float2(tx, ty) : make_float2(0.f, 0.f);
     }
   }
   bool clamped = false;
@@ -356,21 +371,35 @@ __device__ __forceinline__ void invert_diag_part(float* slot, const float* mcol,
   float2 x01 = make_float2(j0 == lane ? 1.f : 0.f, j0 + 1 == lane ? 1.f : 0.f);
   float2 x23 = make_float2(j0 + 2 == lane ? 1.f : 0.f, j0 + 3 == lane ? 1.f : 0.f);
   float my_rinv = 1.f;
-  // a real loop on purpose: straight-line code runs at the rate instructions can be fetched (several
-  // cycles each), a loop this small is served from the innermost instruction cache
-  // The word of the next column is read ahead (it may still be unset; then it is waited for at the top).
-  uint32_t ahead = *reinterpret_cast<const volatile uint32_t*>(mcol + j0 * kLcolLd + lane);
+  // Four columns per round: the words of all four are fetched together (and waited for only if one is still
+  // unset), then the four updates run back to back with nothing in them but the broadcast of row k and two
+  // packed FMAs.  One column per round cost about 180 cycles, a chain of load, compare, branch, select,
+  // shuffle and FMA latencies, which is more than the factoring warps need per pivot: the warp with all 32
+  // columns to go through finished 1400 cycles after the last pivot and held up the whole block step.
+  // The count of columns, 32 - 4 part, is a multiple of four.  A rolled loop: small enough to be served from
+  // the innermost instruction cache.
 #pragma unroll 1
-  for (int k = j0; k < kB; ++k) {
-    const float w = (ahead != kUnset) ? __uint_as_float(ahead) : wait_word(mcol + k * kLcolLd + lane, gave_up);
-    ahead = *reinterpret_cast<const volatile uint32_t*>(mcol + (k + 1 < kB ? k + 1 : k) * kLcolLd + lane);
-    my_rinv = (lane == k) ? w : my_rinv;
-    const float m = (lane > k) ? w : 0.f;
-    const float2 nm = make_float2(-m, -m);
-    const float2 r01 = make_float2(__shfl_sync(0xffffffffu, x01.x, k), __shfl_sync(0xffffffffu, x01.y, k));
-    const float2 r23 = make_float2(__shfl_sync(0xffffffffu, x23.x, k), __shfl_sync(0xffffffffu, x23.y, k));
-    x01 = __ffma2_rn(nm, r01, x01);
-    x23 = __ffma2_rn(nm, r23, x23);
+  for (int k = j0; k < kB; k += 4) {
+    uint32_t bits[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      bits[q] = *reinterpret_cast<const volatile uint32_t*>(mcol + (k + q) * kLcolLd + lane);
+    float w[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      w[q] = (bits[q] != kUnset) ? __uint_as_float(bits[q]) : wait_word(mcol + (k + q) * kLcolLd + lane, gave_up);
+    __syncwarp();
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int kk = k + q;
+      my_rinv = (lane == kk) ? w[q] : my_rinv;
+      const float m = (lane > kk) ? w[q] : 0.f;
+      const float2 nm = make_float2(-m, -m);
+      const float2 r01 = make_float2(__shfl_sync(0xffffffffu, x01.x, kk), __shfl_sync(0xffffffffu, x01.y, kk));
+      const float2 r23 = make_float2(__shfl_sync(0xffffffffu, x23.x, kk), __shfl_sync(0xffffffffu, x23.y, kk));
+      x01 = __ffma2_rn(nm, r01, x01);
+      x23 = __ffma2_rn(nm, r23, x23);
+    }
   }
   *reinterpret_cast<float4*>(slot + lane * kLd + j0) =
       make_float4(x01.x * my_rinv, x01.y * my_rinv, x23.x * my_rinv, x23.y * my_rinv);
