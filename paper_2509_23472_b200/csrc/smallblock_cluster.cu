@@ -413,6 +413,9 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
   __shared__ __align__(8) uint64_t dinv_bar[kMaxBlk];    // workers: D_k^{-1} has arrived
   __shared__ __align__(8) uint64_t panel_bar[kMaxBlk];   // workers: every L(i,k), i > k, has arrived
   __shared__ __align__(8) uint64_t chain_bar[kMaxBlk];   // CTA 0: blocks (j, j-1) and (j, j) have arrived
+  // workers: L(k+1, k) and L(k+2, k) have arrived -- all that the two blocks CTA 0 waits for next need, so
+  // their update does not wait for the whole panel (every worker's blocks, copied to every other worker)
+  __shared__ __align__(8) uint64_t urgent_bar[kMaxBlk];
   __shared__ float s_red[kCThreads / 32];
   __shared__ float s_shift, s_floor;
   __shared__ int s_gave_up;
@@ -443,14 +446,19 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
     bar_init(&dinv_bar[k], 1);
     bar_init(&panel_bar[k], 2);   // the byte count (below) and the CTA's own blocks of the column
     bar_init(&chain_bar[k], 1);
+    bar_init(&urgent_bar[k], 2);  // the byte count, and this CTA's own L(k+2, k) (at once if it owns none)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     if (k < nblk) {
       if (cta != 0) {
         bar_expect(&dinv_bar[k], kSlotTx);
         if (k + 1 < nblk) {
-          int from_peers = 1;   // L(k+1, k) comes from CTA 0
-          for (int bi = k + 2; bi < nblk; ++bi) from_peers += owner_of(bi, k, nblk) != cta ? 1 : 0;
+          int from_peers = 0;   // rows k + 3 and below; L(k+1, k) (from CTA 0) and L(k+2, k) count on urgent_bar
+          for (int bi = k + 3; bi < nblk; ++bi) from_peers += owner_of(bi, k, nblk) != cta ? 1 : 0;
           bar_expect(&panel_bar[k], (uint32_t)from_peers * kSlotTx);
+          const bool own_k2 = k + 2 < nblk && owner_of(k + 2, k, nblk) == cta;
+          const bool peer_k2 = k + 2 < nblk && !own_k2;
+          bar_expect(&urgent_bar[k], (peer_k2 ? 2u : 1u) * kSlotTx);
+          if (!own_k2) bar_arrive_local(&urgent_bar[k]);
         }
       } else if (k >= 2) {
         bar_expect(&chain_bar[k], 2 * kSlotTx);
@@ -623,7 +631,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
         if (lane >= 1 && lane < kCl) {
           const uint32_t src = smem_addr(blk);
           bulk_to_peer(map_to_cta(src, lane), src, kSlotTx,
-                       map_to_cta(smem_addr(is_dinv ? &dinv_bar[k] : &panel_bar[k]), lane));
+                       map_to_cta(smem_addr(is_dinv ? &dinv_bar[k] : &urgent_bar[k]), lane));
         }
       }
     }
@@ -654,13 +662,16 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
         group_sync(1);   // everyone has read the block
         tile_store<2, 2>(blk, acc, t2m, t2n, 1.f, false);
         fence_async_proxy();
-        send_rows(blk, warp * 4, 4, &panel_bar[k], 1, kCl - 1, cta, lane);
+        send_rows(blk, warp * 4, 4, bi == k + 2 ? &urgent_bar[k] : &panel_bar[k], 1, kCl - 1, cta, lane);
       }
-      // this CTA's own blocks of column k are in place: the second arrival on its own barrier
+      // this CTA's own blocks of column k are in place: the second arrival on its own barriers
       group_sync(1);
-      if (tid == 0 && k + 1 < nblk) bar_arrive_local(&panel_bar[k]);
+      if (tid == 0 && k + 1 < nblk) {
+        bar_arrive_local(&panel_bar[k]);
+        if (k + 2 < nblk && owner_of(k + 2, k, nblk) == cta) bar_arrive_local(&urgent_bar[k]);
+      }
       if (k + 1 >= nblk) { if (tid == 0) s_urgent = 0; break; }
-      if (tid == 0) bar_wait(&panel_bar[k], &s_gave_up);
+      if (tid == 0) bar_wait(&urgent_bar[k], &s_gave_up);
       group_sync(1);
       // trailing update with column k.  A diagonal block (j, j) takes columns k <= j - 2 here (CTA 0
       // applies column j - 1 itself), every other block (i, j) columns k <= j - 1.  First the two blocks
@@ -676,7 +687,8 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
         fence_async_proxy();
         send_rows(blk, warp * 4, 4, &chain_bar[k + 2], 0, 0, -1, lane);
       }
-      if (tid == 0) s_urgent = 0;
+      if (tid == 0) { s_urgent = 0; bar_wait(&panel_bar[k], &s_gave_up); }
+      group_sync(1);
       // ... then the rest, one block per pair of warps at a time
       int turn = 0;
       for (int q = 0; q < n_mine; ++q) {
@@ -763,7 +775,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
         }
       }
       if (k + 1 >= nblk) break;
-      if (gt == 0) bar_wait(&panel_bar[k], &s_gave_up);
+      if (gt == 0) { bar_wait(&urgent_bar[k], &s_gave_up); bar_wait(&panel_bar[k], &s_gave_up); }
       group_sync(2);
       // Tt(i,j)[b][a] (+)= sum_q Xt(k,j)[b][q] L(i,k)[a][q] for the rows below
       int turn = 0;
