@@ -343,7 +343,7 @@ def main():
                     "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
                     # dram__bytes_read.sum + dram__bytes_write.sum per launch of this kernel at this shape
                     # (profiles/pass1_llama7b_block_ncu.md); other shapes have not been captured
-                    "traffic": 141.3e6 if (N, d, r) == (16384, 4096, 256) else None,
+                    "traffic": 140.3e6 if (N, d, r) == (16384, 4096, 256) else None,
                     "ms_per_launch": k_ms, "algorithmic_bytes": k_bytes,
                     "tflops": 2.0 * N * d * r / (k_ms * 1e-3) / 1e12}
     # whole-step floor: X once + factors + gathered rows (strict), against measured HBM bandwidth
