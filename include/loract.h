@@ -17,9 +17,11 @@
  *   - rank: a multiple of 16, 16 <= rank <= 512, rank <= n_tokens and rank <= d.
  *   - Calls are asynchronous on the CUDA stream passed as `stream` (a cudaStream_t cast to void*;
  *     NULL is the default stream) and never synchronise, except loract_read_device_status.
- *   - Host-detectable errors return a status and launch nothing.  Conditions found on the device (a
- *     Cholesky pivot that had to be clamped, a bounded wait that expired) are recorded in a 32-bit word
- *     at the start of `ws`; outputs are still fully written.  Read it with loract_read_device_status.
+ *   - Host-detectable errors return a status and launch nothing.  Conditions found on the device are recorded
+ *     in a 32-bit word at the start of `ws`; read it with loract_read_device_status.  After a clamped pivot
+ *     or a non-finite input the outputs are still fully written (finite where the input was).  After an
+ *     expired wait (LORACT_DEV_WAIT_EXPIRED) the kernel that gave up has skipped its stores: the outputs
+ *     are unspecified and must not be used.
  *   - `ws` is scratch of at least loract_workspace_bytes(desc) bytes, 256-byte aligned, private to one
  *     in-flight call.  The same (seed, call_id, n_tokens, rank) always selects the same rows.
  */
@@ -140,21 +142,31 @@ loract_status_t loract_prenorm_backward(const loract_desc_t* desc, const void* U
  *     start at zero.  Two calls that overlap on the GPU (different streams, or different threads) race
  *     on it: serialise them.
  *   - The device status word of this entry point is the first word of that array; it is not readable
- *     through loract_read_device_status. */
+ *     through loract_read_device_status.  loract_weight_grad_static_status copies it to *out_host (a HOST
+ *     pointer) and synchronises `stream`; it allocates nothing either.  A non-zero word (an expired wait)
+ *     means dW of the last call is not valid. */
 loract_status_t loract_weight_grad_static(const loract_desc_t* desc, const void* U, const void* V,
                                           const void* G, int32_t g, int64_t ldg, float* dW, int accumulate,
                                           void* stream);
+loract_status_t loract_weight_grad_static_status(uint32_t* out_host, void* stream);
 
 /* Comparator of Section 3.2: randomized SVD at the same rank -- Algorithm 1 with a Gaussian test matrix
  * of rank + oversample columns (Philox + Box-Muller, counter word 1 set to 1) and `power_iters`
  * iterations of Y = X (X^T Q).  Writes the un-truncated pair: Uq (n_tokens x l), B (l x d), l = rank +
- * oversample (a multiple of 16, <= 512).  bf16 only.  ws must hold loract_rsvd_workspace_bytes. */
+ * oversample (a multiple of 8, <= 512).  The cut from l to `rank` columns (the singular value decomposition
+ * of the small matrix B) is left to the caller.  bf16 only.  ws must hold loract_rsvd_workspace_bytes. */
 size_t loract_rsvd_workspace_bytes(const loract_desc_t* desc, int32_t oversample);
 loract_status_t loract_rsvd(const loract_desc_t* desc, int32_t oversample, const void* X, void* Uq,
                             void* B, void* ws, size_t ws_bytes, void* stream);
 
 /* Copies the device status word at the start of `ws` to *out_host.  Synchronises `stream`. */
 loract_status_t loract_read_device_status(const void* ws, uint32_t* out_host, void* stream);
+
+/* What a device status word means for the call that produced it: LORACT_ERR_TIMEOUT if a bounded wait
+ * expired (outputs unspecified), LORACT_ERR_NUMERIC if a non-finite value reached the factorisation or the
+ * sampler ran short (outputs written but meaningless), LORACT_OK otherwise (a clamped pivot alone is a
+ * warning: the factors are valid).  Pure host function. */
+loract_status_t loract_status_from_device_word(uint32_t word);
 
 const char* loract_status_string(loract_status_t s);
 

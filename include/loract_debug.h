@@ -27,6 +27,12 @@ loract_status_t loract_debug_gemm(int32_t M, int32_t N, int32_t K, int32_t a_mn,
                                   void* C0, void* C1, int64_t ldc, int32_t splits, int64_t split_stride,
                                   int32_t acc64, int32_t engine, uint32_t* status_word, void* stream);
 
+/* Line 8 of Algorithm 1 alone, exactly as loract_compress runs it (same kernels, same launch shapes):
+ * V (rank x d) = U^T X from a stored U (n_tokens x rank).  ws as for loract_compress.  For timing that step in
+ * isolation. */
+loract_status_t loract_debug_project(const loract_desc_t* desc, const void* U, const void* X, void* V, void* ws,
+                                     size_t ws_bytes, void* stream);
+
 /* The tensor-core kernel exists in two forms: one CTA per 128-row tile, and a pair of CTAs (tcgen05
  * cta_group::2) per 256-row tile, chosen by shape.  on = 0 keeps every contraction on the one-CTA form, so
  * that a test can compare the two; on = 1 (the default) restores the choice by shape.  Process-wide. */
@@ -41,6 +47,13 @@ void loract_debug_set_pair_mode(int32_t on);
 void loract_debug_trace_begin(void* stream);
 int32_t loract_debug_trace_end(void* stream, char* names, float* micros, int32_t max_entries);
 
+/* The give-up path of the bounded device-side waits, exercised without a fault: launches one tiny kernel in
+ * which a thread waits on a barrier that nothing ever completes, using the same wait helper as the tensor-core
+ * engine (which = 0) or as the cluster factorisation kernel (which = 1, a cluster of two CTAs), with
+ * `limit_ns` (1 ns to 100 ms) in place of the built-in limit.  The wait gives up, the kernel ORs
+ * LORACT_DEV_WAIT_EXPIRED into *status_word (device uint32) and returns; the context stays usable. */
+loract_status_t loract_debug_wait_expiry(int32_t which, uint64_t limit_ns, uint32_t* status_word, void* stream);
+
 /* The cudaError_t behind the most recent LORACT_ERR_CUDA returned by any entry point (0 if none yet). */
 int32_t loract_debug_last_cuda_error(void);
 
@@ -48,7 +61,7 @@ int32_t loract_debug_last_cuda_error(void);
  * W = sum of n_partials r x r matrices (fp32 if partial_f64 == 0, else fp64; `partial_stride` elements
  * apart); L L^T = W + shift_rel * mean(diag W) * I; writes L^{-1} (lower triangular, row-major) as fp32
  * (linv_f32), as a bf16 hi/lo pair (linv_hi, linv_lo), any of which may be NULL.  use_f64 selects the
- * arithmetic.  scratch: 2*r*r + 2*256*256 elements of the compute type.  r a multiple of 16, <= 512. */
+ * arithmetic.  scratch: 2*r*r + 2*256*256 elements of the compute type.  r a multiple of 8, <= 512. */
 loract_status_t loract_debug_small_block(int32_t r, const void* partials, int32_t partial_f64,
                                          int32_t n_partials, int64_t partial_stride, int32_t use_f64,
                                          float shift_rel, void* scratch, float* linv_f32, void* linv_hi,

@@ -17,8 +17,8 @@ What follows the paper, and where:
                        Section 3.3, the pre-norm unit and its three gradient
                        equations
   * ``truncated_svd``  Section 3.2 (the Eckart-Young optimum, yardstick)
-  * ``rsvd``           Section 3.2: "the rest of the algorithm identical to
-                       RSVD" -- the same steps with a Gaussian test matrix
+  * ``rsvd``           Section 3.2: the same steps as Algorithm 1 with the
+                       sampled rows replaced by a Gaussian test matrix
   * ``halko_bound_sq`` the deterministic bound of Theorem 3.3
 
 Readings taken where the paper is silent (all listed in the design notes):

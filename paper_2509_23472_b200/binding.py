@@ -21,9 +21,10 @@ DEV_PIVOT_CLAMPED, DEV_WAIT_EXPIRED, DEV_SAMPLER_SHORT, DEV_NONFINITE = 1, 2, 4,
 
 EXPORTS = (
     "loract_workspace_bytes", "loract_sample_indices", "loract_compress", "loract_reconstruct",
-    "loract_weight_grad", "loract_weight_grad_static", "loract_compress_prenorm",
+    "loract_weight_grad", "loract_weight_grad_static", "loract_weight_grad_static_status", "loract_compress_prenorm",
     "loract_prenorm_backward_workspace_bytes", "loract_prenorm_backward", "loract_rsvd_workspace_bytes", "loract_rsvd",
-    "loract_read_device_status", "loract_status_string", "loract_kernel_launch_count",
+    "loract_read_device_status", "loract_status_from_device_word", "loract_status_string",
+    "loract_kernel_launch_count",
 )
 
 
@@ -69,6 +70,8 @@ def lib() -> ctypes.CDLL:
         l.loract_weight_grad.argtypes = [dp, vp, vp, vp, i32, i64, vp, ctypes.c_int, vp, sz, vp]
         l.loract_weight_grad_static.restype = ctypes.c_int
         l.loract_weight_grad_static.argtypes = [dp, vp, vp, vp, i32, i64, vp, ctypes.c_int, vp]
+        l.loract_weight_grad_static_status.restype = ctypes.c_int
+        l.loract_weight_grad_static_status.argtypes = [ctypes.POINTER(ctypes.c_uint32), vp]
         l.loract_compress_prenorm.restype = ctypes.c_int
         l.loract_compress_prenorm.argtypes = [dp, vp, vp, vp, ctypes.c_float, i32, vp, vp, vp, vp, vp, vp,
                                               vp, sz, vp]
@@ -82,6 +85,8 @@ def lib() -> ctypes.CDLL:
         l.loract_rsvd.argtypes = [dp, i32, vp, vp, vp, vp, sz, vp]
         l.loract_read_device_status.restype = ctypes.c_int
         l.loract_read_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
+        l.loract_status_from_device_word.restype = ctypes.c_int
+        l.loract_status_from_device_word.argtypes = [ctypes.c_uint32]
         l.loract_status_string.restype = ctypes.c_char_p
         l.loract_status_string.argtypes = [ctypes.c_int]
         l.loract_kernel_launch_count.restype = ctypes.c_uint64
@@ -92,6 +97,10 @@ def lib() -> ctypes.CDLL:
 
 def status_string(code: int) -> str:
     return lib().loract_status_string(code).decode()
+
+
+def status_from_device_word(word: int) -> int:
+    return int(lib().loract_status_from_device_word(word))
 
 
 def kernel_launch_count() -> int:
@@ -223,6 +232,14 @@ def weight_grad_static(U: torch.Tensor, V: torch.Tensor, G: torch.Tensor, dW: to
     return dW
 
 
+def weight_grad_static_status(device) -> int:
+    """Device status word of the last loract_weight_grad_static call on the current device (0 = clean)."""
+    out = ctypes.c_uint32(0)
+    _check(lib().loract_weight_grad_static_status(ctypes.byref(out), _stream(device)),
+           "loract_weight_grad_static_status")
+    return int(out.value)
+
+
 def compress_prenorm(X: torch.Tensor, gamma: torch.Tensor, beta: Optional[torch.Tensor], eps: float, kind: int,
                      rank: int, seed: int = 0, call_id: int = 0, want_A: bool = True,
                      ws: Optional[torch.Tensor] = None):
@@ -294,7 +311,8 @@ def read_device_status(ws: torch.Tensor) -> int:
 # ---------------------------------------------------------------------------------------------
 OUT_F32, OUT_BF16, OUT_SPLIT, OUT_F64 = 0, 1, 2, 3
 DEBUG_EXPORTS = ("loract_debug_gemm", "loract_debug_small_block", "loract_debug_set_pair_mode",
-                 "loract_debug_last_cuda_error", "loract_debug_trace_begin", "loract_debug_trace_end")
+                 "loract_debug_last_cuda_error", "loract_debug_trace_begin", "loract_debug_trace_end",
+                 "loract_debug_wait_expiry", "loract_debug_project")
 
 
 def _debug_lib():
@@ -337,6 +355,25 @@ def debug_gemm(A_terms, B_terms, M: int, N: int, K: int, a_mn: bool, b_mn: bool,
     if out_mode in (OUT_F32, OUT_F64):
         return C0 if splits > 1 else C0[0]
     return C0 if C1 is None else (C0, C1)
+
+
+def debug_wait_expiry(which: int, limit_ns: int, status: torch.Tensor) -> None:
+    """Test hook: a kernel whose bounded wait (0: tensor-core engine, 1: cluster factorisation) runs out after
+    limit_ns and ORs DEV_WAIT_EXPIRED into the uint32 `status` tensor."""
+    l = _debug_lib()
+    l.loract_debug_wait_expiry.restype = ctypes.c_int
+    l.loract_debug_wait_expiry.argtypes = [ctypes.c_int32, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_void_p]
+    _check(l.loract_debug_wait_expiry(which, limit_ns, _ptr(status), _stream(status.device)),
+           "loract_debug_wait_expiry")
+
+
+def debug_project(desc: Desc, U: torch.Tensor, X: torch.Tensor, V: torch.Tensor, ws: torch.Tensor) -> None:
+    """Test / timing hook: V = U^T X exactly as loract_compress runs its last step."""
+    l = _debug_lib()
+    l.loract_debug_project.restype = ctypes.c_int
+    l.loract_debug_project.argtypes = [ctypes.POINTER(Desc)] + [ctypes.c_void_p] * 4 + [ctypes.c_size_t, ctypes.c_void_p]
+    _check(l.loract_debug_project(ctypes.byref(desc), _ptr(U), _ptr(X), _ptr(V), _ptr(ws), ws.numel(),
+                                  _stream(X.device)), "loract_debug_project")
 
 
 def debug_set_pair_mode(on: bool) -> None:

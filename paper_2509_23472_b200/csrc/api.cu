@@ -38,27 +38,7 @@ void count_launch(const char* kernel, cudaStream_t stream) {
   g_trace_names.push_back(std::string(g_trace_label) + " [" + kernel + "]");
 }
 
-namespace {
-
-constexpr size_t kAlign = 256;
-inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
-
-// relative diagonal shifts of the three Cholesky factorisations (fp32 small blocks)
 constexpr int kMaxPowerIters = 8;      // t of Algorithm 1 accepted by loract_compress
-constexpr float kShiftSample = 1e-6f;  // Gram of the sampled rows
-constexpr float kShiftFirst = 3e-6f;   // first Gram of the sketch
-constexpr float kShiftSecond = 1e-7f;  // second Gram (already close to the identity)
-
-struct Carver {
-  unsigned char* base;
-  size_t off = 0;
-  explicit Carver(void* p) : base((unsigned char*)p) {}
-  void* take(size_t bytes) {
-    void* r = base ? base + off : nullptr;
-    off += align_up(bytes);
-    return r;
-  }
-};
 
 loract_status_t check_desc(const loract_desc_t* d) {
   if (!d) return LORACT_ERR_INVALID_ARG;
@@ -74,6 +54,27 @@ loract_status_t check_desc(const loract_desc_t* d) {
   if (d->d % mult || d->ldx % mult) return LORACT_ERR_ALIGNMENT;
   return LORACT_OK;
 }
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// relative diagonal shifts of the three Cholesky factorisations (fp32 small blocks)
+constexpr float kShiftSample = 1e-6f;  // Gram of the sampled rows
+constexpr float kShiftFirst = 3e-6f;   // first Gram of the sketch
+constexpr float kShiftSecond = 1e-7f;  // second Gram (already close to the identity)
+
+struct Carver {
+  unsigned char* base;
+  size_t off = 0;
+  explicit Carver(void* p) : base((unsigned char*)p) {}
+  void* take(size_t bytes) {
+    void* r = base ? base + off : nullptr;
+    off += align_up(bytes);
+    return r;
+  }
+};
+
 inline bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
 inline int elem_bytes(const loract_desc_t* d) { return d->dtype == LORACT_BF16 ? 2 : 4; }
 
@@ -553,7 +554,7 @@ loract_status_t loract_prenorm_backward(const loract_desc_t* desc, const void* U
 size_t loract_rsvd_workspace_bytes(const loract_desc_t* desc, int32_t oversample) {
   if (check_desc(desc) != LORACT_OK || desc->dtype != LORACT_BF16) return 0;
   const int l = desc->rank + oversample;
-  if (oversample < 0 || l % 16 || l > 512 || l > desc->n_tokens || l > desc->d) return 0;
+  if (oversample < 0 || l % 8 || l > 512 || l > desc->n_tokens || l > desc->d) return 0;
   Plan plan = make_plan(desc->n_tokens, desc->d, l, true);
   Carver c(nullptr);
   c.take(256);
@@ -625,6 +626,20 @@ const char* loract_status_string(loract_status_t s) {
   return "unknown status";
 }
 
+loract_status_t loract_status_from_device_word(uint32_t word) {
+  if (word & LORACT_DEV_WAIT_EXPIRED) return LORACT_ERR_TIMEOUT;
+  if (word & (LORACT_DEV_NONFINITE | LORACT_DEV_SAMPLER_SHORT)) return LORACT_ERR_NUMERIC;
+  return LORACT_OK;   // a clamped pivot alone is a warning: the factors are valid
+}
+
+loract_status_t loract_debug_wait_expiry(int32_t which, uint64_t limit_ns, uint32_t* status_word, void* stream) {
+  if (!status_word || limit_ns == 0 || limit_ns > 100000000ull) return LORACT_ERR_INVALID_ARG;   // 100 ms at most
+  cudaStream_t st = (cudaStream_t)stream;
+  if (which == 0) return from_cuda(gemm_tc_wait_probe_launch(status_word, limit_ns, st));
+  if (which == 1) return from_cuda(small_block_cluster_wait_probe_launch(status_word, limit_ns, st));
+  return LORACT_ERR_INVALID_ARG;
+}
+
 uint64_t loract_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 loract_status_t loract_debug_gemm(int32_t M, int32_t N, int32_t K, int32_t a_mn, int32_t b_mn,
@@ -644,6 +659,18 @@ loract_status_t loract_debug_gemm(int32_t M, int32_t N, int32_t K, int32_t a_mn,
     return from_cuda(gemm_tc_launch(g, status_word, (cudaStream_t)stream));
   }
   return from_cuda(gemm_simt_launch(g, (cudaStream_t)stream));
+}
+
+loract_status_t loract_debug_project(const loract_desc_t* desc, const void* U, const void* X, void* V, void* ws,
+                                     size_t ws_bytes, void* stream) {
+  loract_status_t s = check_desc(desc);
+  if (s != LORACT_OK) return s;
+  if (!U || !X || !V || !ws) return LORACT_ERR_INVALID_ARG;
+  CompressWs w;
+  Plan plan;
+  const size_t need = carve_compress(ws, desc, /*with_A=*/false, &w, &plan);
+  if (ws_bytes < need) return LORACT_ERR_WORKSPACE_TOO_SMALL;
+  return from_cuda(project(U, X, desc->ldx, plan, V, w.b, w.status, (cudaStream_t)stream));
 }
 
 void loract_debug_trace_begin(void* stream) {
@@ -677,7 +704,7 @@ loract_status_t loract_debug_small_block(int32_t r, const void* partials, int32_
                                          int64_t partial_stride, int32_t use_f64, float shift_rel, void* scratch,
                                          float* linv_f32, void* linv_hi, void* linv_lo, uint32_t* status_word,
                                          void* stream) {
-  if (r < 16 || r > 512 || r % 16 || !partials || !scratch || n_partials < 1) return LORACT_ERR_INVALID_ARG;
+  if (r < 16 || r > 512 || r % 8 || !partials || !scratch || n_partials < 1) return LORACT_ERR_INVALID_ARG;
   SmallBlockArgs a;
   a.r = r; a.partials = partials; a.partial_type = partial_f64 ? ELEM_F64 : ELEM_F32;
   a.n_partials = n_partials; a.partial_stride = partial_stride; a.use_f64 = use_f64 != 0;

@@ -15,6 +15,9 @@ namespace loract {
 void count_launch(const char* kernel = "", cudaStream_t stream = nullptr);
 void trace_label(const char* label);
 
+// The argument rules every entry point shares (include/loract.h, "Conventions"): LORACT_OK or the error.
+loract_status_t check_desc(const loract_desc_t* d);
+
 #define LORACT_CUDA_TRY(expr)                          \
   do {                                                 \
     cudaError_t _e = (expr);                           \
@@ -101,6 +104,10 @@ bool gemm_tc_supported(const GemmDesc& g);
 cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t stream);
 int gemm_tc_pick_splits(int M, int N, int K, bool a_mn, bool b_mn);
 void gemm_tc_set_pair_mode(int on);   // test hook: 0 keeps every contraction on the one-CTA kernel
+// Test hooks for the give-up path of the bounded waits: a kernel that waits (with the engine's / the cluster
+// kernel's own wait) on a barrier nothing completes, for at most limit_ns, then sets LORACT_DEV_WAIT_EXPIRED.
+cudaError_t gemm_tc_wait_probe_launch(uint32_t* dev_status, uint64_t limit_ns, cudaStream_t stream);
+cudaError_t small_block_cluster_wait_probe_launch(uint32_t* dev_status, uint64_t limit_ns, cudaStream_t stream);
 
 // Plain CUDA-core kernel for any shape and type (fp32 path, small or odd shapes).
 cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t stream);

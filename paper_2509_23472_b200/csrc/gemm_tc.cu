@@ -90,7 +90,8 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 // Bounded wait.  Returns false if the limit expired (or another role already gave up).
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                  uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   // the wall clock is read only once in a while, and first after 1024 failed polls: a read of %globaltimer is
   // slow enough to matter on the hand-offs of the operand ring, which all pass through here
@@ -101,7 +102,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
       if (*abort_flag) return false;
       const uint64_t now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      else if (now - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
   }
 }
@@ -922,6 +923,25 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   if (threadIdx.x == 0 && abort_flag && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_WAIT_EXPIRED);
 }
 
+// ------------------------------------------------------------------ the abort path, exercised on purpose
+// One thread waits, with the engine's own bounded wait, on a barrier that nothing ever arrives on.  The wait
+// must give up after `limit_ns`, and the kernel then does what every role of the engine does: it records
+// LORACT_DEV_WAIT_EXPIRED and returns.  Nothing else runs, so the context stays usable.
+__global__ void wait_expiry_probe_kernel(uint32_t* dev_status, uint64_t limit_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  bool ok = true;
+  if (threadIdx.x == 0) ok = mbar_wait_bounded(&bar, 0, &abort_flag, limit_ns);
+  __syncthreads();
+  if (threadIdx.x == 0 && (!ok || abort_flag) && dev_status) atomicOr(dev_status, LORACT_DEV_WAIT_EXPIRED);
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -1086,6 +1106,12 @@ int g_pair_mode = 1;   // 0: never use the two-CTA kernels (test hook); 1: by sh
 }  // namespace
 
 void gemm_tc_set_pair_mode(int on) { g_pair_mode = on; }
+
+cudaError_t gemm_tc_wait_probe_launch(uint32_t* dev_status, uint64_t limit_ns, cudaStream_t stream) {
+  wait_expiry_probe_kernel<<<1, 32, 0, stream>>>(dev_status, limit_ns);
+  count_launch(__func__, stream);
+  return cudaGetLastError();
+}
 
 bool gemm_tc_supported(const GemmDesc& g) {
   if (g.a_type != ELEM_BF16 || g.b_type != ELEM_BF16) return false;

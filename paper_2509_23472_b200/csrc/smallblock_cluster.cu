@@ -107,7 +107,7 @@ __device__ __forceinline__ uint64_t timer_ns() {
 // Every barrier of this kernel completes exactly once (phase 0).  Called by ONE thread of a warp group;
 // the others block on the named barrier that follows, so that waiting costs no issue slots.  Returns
 // false once the CTA has given up.
-__device__ __forceinline__ bool bar_wait(uint64_t* bar, volatile int* gave_up) {
+__device__ __forceinline__ bool bar_wait(uint64_t* bar, volatile int* gave_up, uint64_t limit_ns = kClusterWaitNs) {
   if (bar_try(bar)) return true;
   if (*gave_up) return false;
   uint64_t t0 = 0;
@@ -118,7 +118,7 @@ __device__ __forceinline__ bool bar_wait(uint64_t* bar, volatile int* gave_up) {
       if (*gave_up) return false;
       const uint64_t now = timer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kClusterWaitNs) { *gave_up = 1; return false; }
+      else if (now - t0 > limit_ns) { *gave_up = 1; return false; }
     }
   }
 }
@@ -801,7 +801,34 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
   cluster_sync_all();
 }
 
+// The give-up path of this file's waits, exercised on purpose: a two-CTA cluster in which CTA 1 waits, with
+// bar_wait, for bytes that CTA 0 never sends.  After `limit_ns` it records LORACT_DEV_WAIT_EXPIRED and both
+// CTAs run to the closing cluster barrier, as the factorisation kernel does.
+__global__ void __cluster_dims__(2, 1, 1) cluster_wait_probe_kernel(uint32_t* dev_status, uint64_t limit_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int gave_up;
+  uint32_t rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+  if (threadIdx.x == 0) {
+    bar_init(&bar, 1);
+    gave_up = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    bar_expect(&bar, 16);   // sixteen bytes that never arrive
+  }
+  cluster_sync_all();
+  if (rank == 1 && threadIdx.x == 0) bar_wait(&bar, &gave_up, limit_ns);
+  __syncthreads();
+  if (threadIdx.x == 0 && gave_up && dev_status) atomicOr(dev_status, LORACT_DEV_WAIT_EXPIRED);
+  cluster_sync_all();
+}
+
 }  // namespace
+
+cudaError_t small_block_cluster_wait_probe_launch(uint32_t* dev_status, uint64_t limit_ns, cudaStream_t stream) {
+  cluster_wait_probe_kernel<<<2, 32, 0, stream>>>(dev_status, limit_ns);
+  count_launch(__func__, stream);
+  return cudaGetLastError();
+}
 
 bool small_block_cluster_supported(const SmallBlockArgs& a) {
   return !a.use_f64 && a.partial_type == ELEM_F32 && a.r <= kMaxBlk * kB && a.r % 4 == 0 &&

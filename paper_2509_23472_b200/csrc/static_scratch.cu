@@ -7,6 +7,8 @@
 // caller-provided workspace for its intermediate T = U^T G; this variant needs none.  Its scratch is a
 // fixed array inside the library image (below), so every GPU that loads the library holds
 // kStaticScratchBytes of device memory until the process exits, and the problem size is limited.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace loract {
@@ -21,19 +23,23 @@ constexpr size_t kStaticHeaderBytes = 256;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
-unsigned char* g_scratch_addr[kMaxDevices] = {};
+// One slot per device, written once.  Two host threads that make their first call at the same moment both
+// look the address up and store the same value, which is harmless; the atomic keeps the store and the loads
+// well defined.  (A cudaDeviceReset in the same process invalidates the slot: callers that reset a device
+// must not use this entry point afterwards.)
+std::atomic<unsigned char*> g_scratch_addr[kMaxDevices];
 
 // Set-up, once per device, with that device current: resolve the device address of the array.
 cudaError_t static_scratch_address(unsigned char** out) {
   int dev = 0;
   LORACT_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  if (!g_scratch_addr[dev]) {
-    unsigned char* p = nullptr;
+  unsigned char* p = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!p) {
     LORACT_CUDA_TRY(cudaGetSymbolAddress((void**)&p, g_static_scratch));
-    g_scratch_addr[dev] = p;
+    g_scratch_addr[dev].store(p, std::memory_order_release);
   }
-  *out = g_scratch_addr[dev];
+  *out = p;
   return cudaSuccess;
 }
 
@@ -45,14 +51,11 @@ using namespace loract;
 extern "C" loract_status_t loract_weight_grad_static(const loract_desc_t* desc, const void* U, const void* V,
                                                      const void* G, int32_t g, int64_t ldg, float* dW,
                                                      int accumulate, void* stream) {
-  if (!desc || !U || !V || !G || !dW) return LORACT_ERR_INVALID_ARG;
-  if (desc->dtype != LORACT_F32 && desc->dtype != LORACT_BF16) return LORACT_ERR_INVALID_ARG;
-  if (desc->reserved != 0 || desc->n_tokens < 1 || desc->d < 1) return LORACT_ERR_INVALID_ARG;
-  if (desc->n_tokens > 0x7fffffffLL || desc->d > 0x7fffffffLL) return LORACT_ERR_INVALID_ARG;
-  if (desc->rank < 16 || desc->rank > 512 || desc->rank % 16) return LORACT_ERR_INVALID_ARG;
+  const loract_status_t ds = check_desc(desc);   // the same descriptor rules as loract_weight_grad
+  if (ds != LORACT_OK) return ds;
+  if (!U || !V || !G || !dW) return LORACT_ERR_INVALID_ARG;
   if (g < 1 || g > 256 || ldg < g) return LORACT_ERR_INVALID_ARG;
-  const int64_t mult = desc->dtype == LORACT_BF16 ? 8 : 4;
-  if (desc->d % mult || ldg % mult) return LORACT_ERR_ALIGNMENT;
+  if (ldg % (desc->dtype == LORACT_BF16 ? 8 : 4)) return LORACT_ERR_ALIGNMENT;
   if (((uintptr_t)U & 15) || ((uintptr_t)V & 15) || ((uintptr_t)G & 15)) return LORACT_ERR_ALIGNMENT;
   const int r = desc->rank;
   // the fixed scratch must hold T and at least one partial sum of T
@@ -87,5 +90,17 @@ extern "C" loract_status_t loract_weight_grad_static(const loract_desc_t* desc, 
     q.out = OUT_F32; q.C0 = dW; q.ldc = g; q.accumulate = accumulate != 0;
     e = gemm_simt_launch(q, st);
   }
+  return e == cudaSuccess ? LORACT_OK : LORACT_ERR_CUDA;
+}
+
+// The status word of the static entry point lives in the library's own array, out of reach of
+// loract_read_device_status; this reader copies it to the host.  Allocates nothing; synchronises `stream`.
+extern "C" loract_status_t loract_weight_grad_static_status(uint32_t* out_host, void* stream) {
+  if (!out_host) return LORACT_ERR_INVALID_ARG;
+  unsigned char* base = nullptr;
+  if (static_scratch_address(&base) != cudaSuccess) return LORACT_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMemcpyAsync(out_host, base, 4, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   return e == cudaSuccess ? LORACT_OK : LORACT_ERR_CUDA;
 }

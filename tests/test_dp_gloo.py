@@ -65,3 +65,26 @@ def test_two_ranks_get_their_own_batches_and_one_whole_job_number():
     assert dp.whole_job_gbs(2, 10 ** 9, 1000.0) == 2.0
     # without a process group the aggregate is the identity
     assert dp.max_over_ranks([3.0, 1.5]) == [3.0, 1.5]
+
+
+def test_bench_starts_its_own_ranks_when_run_without_a_launcher():
+    """`python bench.py --gpus 2` with no WORLD_SIZE in the environment starts two ranks itself (through
+    torch.distributed.run) and reports n_gpus 2.  --plumbing-only keeps it to what runs without a GPU: rank
+    start-up on a gloo group, the barriers, the max over ranks and the whole-job figure."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--plumbing-only"],
+                       capture_output=True, text=True, env=env, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                              # rank 0 alone prints
+    out = json.loads(lines[0])
+    base = synth.get_workload("llama7b_block")
+    assert out["n_gpus"] == 2 and out["plumbing_only"] is True
+    assert out["ms_per_step"] == 2.0                    # the slower rank's time
+    assert out["seeds"] == [base.seed, base.seed + dp.SEED_STRIDE] and out["call_ids"] == [0, 1]
+    assert out["value"] == dp.whole_job_gbs(2, base.n_tokens * base.d * base.elem_bytes, 2.0)

@@ -19,15 +19,16 @@ def dev():
     return torch.device("cuda:0")
 
 
-@pytest.mark.parametrize("name", ["llama7b_block", "llama7b_mlp", "llama13b_s1024_r64", "llama13b_s1024_r512",
-                                  "llama13b_s8192_r64", "llama13b_s8192_r512", "llama13b_s2048_r128",
-                                  "llama13b_s4096_r256"])
+SWEEP = [f"llama13b_s{s}_r{r}" for s in (1024, 2048, 4096, 8192) for r in (64, 128, 256, 512)]
+
+
+@pytest.mark.parametrize("name", ["llama7b_block", "llama7b_mlp"] + SWEEP)
 def test_full_size_configuration(dev, name):
     w = synth.get_workload(name)
     inp = synth.make_inputs(w, device=dev)
     res = check_compress(inp["X"], w.rank, w.seed, G=inp["G"])
-    print(f"{name}: err gpu {res['err']:.5f} oracle {res['ref']['err']:.5f} orth {res['orth']:.1e} "
-          f"wgrad {res['wgrad_rel']:.1e}")
+    print(f"{name}: err gpu {res['err']:.5f} oracle {res['ref']['err']:.5f} projection distance {res['proj']:.2e} "
+          f"orth {res['orth']:.1e} wgrad {res['wgrad_rel']:.1e}")
     del res, inp
     torch.cuda.empty_cache()
 
