@@ -310,6 +310,124 @@ __global__ void __launch_bounds__(256) norm_forward_kernel(const T* __restrict__
   }
 }
 
+// The same unit with 16-byte accesses, one warp per row.  A lane takes the chunks lane, lane + 32, ... of the
+// row (8 bf16 or 4 fp32 values each), so every load and store instruction of a warp covers 512 contiguous
+// bytes.  Rows of up to kKeep chunks per lane (d <= 4096 in bf16, 2048 in fp32) stay in registers, packed as
+// loaded: X is read from memory exactly once and the statistics (mean, then the centred second moment, as
+// in the kernel above) are taken from the registers.  Longer rows are read again for each pass.
+constexpr int kNormKeep = 16;
+
+template <typename T>
+struct NormChunk;
+template <>
+struct NormChunk<__nv_bfloat16> {
+  static constexpr int kVals = 8;
+  static __device__ __forceinline__ void unpack(const uint4& c, float (&v)[8]) {
+    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      v[2 * h] = __uint_as_float(w[h] << 16);
+      v[2 * h + 1] = __uint_as_float(w[h] & 0xffff0000u);
+    }
+  }
+  static __device__ __forceinline__ uint4 pack(const float (&v)[8]) {
+    uint32_t w[4];
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      const __nv_bfloat162 t = __floats2bfloat162_rn(v[2 * h], v[2 * h + 1]);
+      w[h] = *reinterpret_cast<const uint32_t*>(&t);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+  }
+};
+template <>
+struct NormChunk<float> {
+  static constexpr int kVals = 4;
+  static __device__ __forceinline__ void unpack(const uint4& c, float (&v)[4]) {
+    v[0] = __uint_as_float(c.x); v[1] = __uint_as_float(c.y); v[2] = __uint_as_float(c.z); v[3] = __uint_as_float(c.w);
+  }
+  static __device__ __forceinline__ uint4 pack(const float (&v)[4]) {
+    return make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+  }
+};
+
+template <typename T, bool kInRegs>
+__global__ void __launch_bounds__(256) norm_forward_vec_kernel(const T* __restrict__ X, int64_t n, int64_t d,
+                                                               int64_t ldx, const T* __restrict__ gamma,
+                                                               const T* __restrict__ beta, float eps, int kind,
+                                                               T* __restrict__ A, int64_t lda,
+                                                               float* __restrict__ rstd_out,
+                                                               float* __restrict__ mean_out) {
+  using C = NormChunk<T>;
+  constexpr int kV = C::kVals;
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= n) return;
+  const int n_chunks = (int)(d / kV);
+  const uint4* x = reinterpret_cast<const uint4*>(X + row * ldx);
+  const uint4* gm = reinterpret_cast<const uint4*>(gamma);
+  const uint4* bt = reinterpret_cast<const uint4*>(beta);
+  uint4* a = reinterpret_cast<uint4*>(A + row * lda);
+  uint4 keep[kInRegs ? kNormKeep : 1];
+  if (kInRegs) {
+#pragma unroll
+    for (int i = 0; i < kNormKeep; ++i) {
+      const int c = lane + 32 * i;
+      keep[i] = c < n_chunks ? x[c] : make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+  auto chunk = [&](int i, int c) -> uint4 { return kInRegs ? keep[i] : x[c]; };
+  const int per_lane = kInRegs ? kNormKeep : (n_chunks + 31) / 32;
+  float mean = 0.f;
+  if (kind == LORACT_NORM_LAYER) {
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < per_lane; ++i) {
+      const int c = lane + 32 * i;
+      if (c >= n_chunks) break;
+      float v[kV];
+      C::unpack(chunk(i, c), v);
+#pragma unroll
+      for (int q = 0; q < kV; ++q) s += v[q];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    mean = s / (float)d;
+  }
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < per_lane; ++i) {
+    const int c = lane + 32 * i;
+    if (c >= n_chunks) break;
+    float v[kV];
+    C::unpack(chunk(i, c), v);
+#pragma unroll
+    for (int q = 0; q < kV; ++q) { const float t = v[q] - mean; ss += t * t; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float rstd = rsqrtf(ss / (float)d + eps);
+  if (lane == 0) {
+    rstd_out[row] = rstd;
+    if (mean_out) mean_out[row] = mean;
+  }
+#pragma unroll
+  for (int i = 0; i < per_lane; ++i) {
+    const int c = lane + 32 * i;
+    if (c >= n_chunks) break;
+    float v[kV], g[kV], b[kV];
+    C::unpack(chunk(i, c), v);
+    C::unpack(__ldg(gm + c), g);
+    if (beta) C::unpack(__ldg(bt + c), b);
+#pragma unroll
+    for (int q = 0; q < kV; ++q) {
+      v[q] = (v[q] - mean) * rstd * g[q];
+      if (beta) v[q] += b[q];
+    }
+    a[c] = C::pack(v);
+  }
+}
+
 template <typename TA, typename TB>
 cudaError_t launch_simt_typed(const SimtParams& p, bool acc64, cudaStream_t stream) {
   dim3 grid((p.N + kTile - 1) / kTile, (p.M + kTile - 1) / kTile, p.splits);
@@ -407,14 +525,34 @@ cudaError_t norm_forward_launch(const void* X, int64_t n, int64_t d, int64_t ldx
                                 int64_t lda, float* rstd, float* mean, cudaStream_t stream) {
   const int warps = 8;
   const int grid = (int)((n + warps - 1) / warps);
-  if (elem_type == ELEM_BF16)
-    norm_forward_kernel<__nv_bfloat16><<<grid, warps * 32, 0, stream>>>(
-        (const __nv_bfloat16*)X, n, d, ldx, (const __nv_bfloat16*)gamma, (const __nv_bfloat16*)beta,
-        eps, kind, (__nv_bfloat16*)A, lda, rstd, mean);
-  else
-    norm_forward_kernel<float><<<grid, warps * 32, 0, stream>>>(
-        (const float*)X, n, d, ldx, (const float*)gamma, (const float*)beta, eps, kind, (float*)A, lda,
-        rstd, mean);
+  const int vals = elem_type == ELEM_BF16 ? 8 : 4;
+  // 16-byte accesses need every row of X and A, and gamma and beta, on a 16-byte boundary
+  const bool vec = d % vals == 0 && ldx % vals == 0 && lda % vals == 0 && (((uintptr_t)X | (uintptr_t)A |
+                   (uintptr_t)gamma | (uintptr_t)beta) & 15) == 0;
+  const bool in_regs = d <= (int64_t)vals * 32 * kNormKeep;
+  if (elem_type == ELEM_BF16) {
+    typedef __nv_bfloat16 T;
+    if (vec && in_regs)
+      norm_forward_vec_kernel<T, true><<<grid, warps * 32, 0, stream>>>((const T*)X, n, d, ldx, (const T*)gamma,
+                                                                       (const T*)beta, eps, kind, (T*)A, lda, rstd, mean);
+    else if (vec)
+      norm_forward_vec_kernel<T, false><<<grid, warps * 32, 0, stream>>>((const T*)X, n, d, ldx, (const T*)gamma,
+                                                                        (const T*)beta, eps, kind, (T*)A, lda, rstd, mean);
+    else
+      norm_forward_kernel<T><<<grid, warps * 32, 0, stream>>>((const T*)X, n, d, ldx, (const T*)gamma, (const T*)beta,
+                                                              eps, kind, (T*)A, lda, rstd, mean);
+  } else {
+    typedef float T;
+    if (vec && in_regs)
+      norm_forward_vec_kernel<T, true><<<grid, warps * 32, 0, stream>>>((const T*)X, n, d, ldx, (const T*)gamma,
+                                                                       (const T*)beta, eps, kind, (T*)A, lda, rstd, mean);
+    else if (vec)
+      norm_forward_vec_kernel<T, false><<<grid, warps * 32, 0, stream>>>((const T*)X, n, d, ldx, (const T*)gamma,
+                                                                        (const T*)beta, eps, kind, (T*)A, lda, rstd, mean);
+    else
+      norm_forward_kernel<T><<<grid, warps * 32, 0, stream>>>((const T*)X, n, d, ldx, (const T*)gamma, (const T*)beta,
+                                                              eps, kind, (T*)A, lda, rstd, mean);
+  }
   count_launch(__func__, stream);
   return cudaGetLastError();
 }
