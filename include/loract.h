@@ -153,7 +153,7 @@ loract_status_t loract_weight_grad_static_status(uint32_t* out_host, void* strea
 /* Comparator of Section 3.2: randomized SVD at the same rank -- Algorithm 1 with a Gaussian test matrix
  * of rank + oversample columns (Philox + Box-Muller, counter word 1 set to 1) and `power_iters`
  * iterations of Y = X (X^T Q).  Writes the un-truncated pair: Uq (n_tokens x l), B (l x d), l = rank +
- * oversample (a multiple of 8, <= 512).  The cut from l to `rank` columns (the singular value decomposition
+ * oversample (a multiple of 8, <= 640; oversample <= 128).  The cut from l to `rank` columns (the singular value decomposition
  * of the small matrix B) is left to the caller.  bf16 only.  ws must hold loract_rsvd_workspace_bytes. */
 size_t loract_rsvd_workspace_bytes(const loract_desc_t* desc, int32_t oversample);
 loract_status_t loract_rsvd(const loract_desc_t* desc, int32_t oversample, const void* X, void* Uq,

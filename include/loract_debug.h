@@ -61,7 +61,7 @@ int32_t loract_debug_last_cuda_error(void);
  * W = sum of n_partials r x r matrices (fp32 if partial_f64 == 0, else fp64; `partial_stride` elements
  * apart); L L^T = W + shift_rel * mean(diag W) * I; writes L^{-1} (lower triangular, row-major) as fp32
  * (linv_f32), as a bf16 hi/lo pair (linv_hi, linv_lo), any of which may be NULL.  use_f64 selects the
- * arithmetic.  scratch: 2*r*r + 2*256*256 elements of the compute type.  r a multiple of 8, <= 512. */
+ * arithmetic.  scratch: 2*r*r + 2*256*(256 + max(r-256,0) + max(r-512,0)) elements of the compute type.  r a multiple of 8, <= 640. */
 loract_status_t loract_debug_small_block(int32_t r, const void* partials, int32_t partial_f64,
                                          int32_t n_partials, int64_t partial_stride, int32_t use_f64,
                                          float shift_rel, void* scratch, float* linv_f32, void* linv_hi,

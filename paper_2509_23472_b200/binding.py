@@ -410,7 +410,7 @@ def debug_small_block(partials: torch.Tensor, use_f64: bool, shift_rel: float,
     l = _debug_lib()
     dev = partials.device
     n_p, r, _ = partials.shape
-    scratch = torch.empty(2 * r * r + 2 * 256 * 256 + 64 * r, dtype=torch.float64 if use_f64 else torch.float32,
+    scratch = torch.empty(2 * r * r + 2 * 256 * (256 + max(r - 256, 0) + max(r - 512, 0)) + 64 * r, dtype=torch.float64 if use_f64 else torch.float32,
                           device=dev)
     L32 = torch.zeros(r, r, dtype=torch.float32, device=dev)
     Lh = torch.zeros(r, r, dtype=torch.bfloat16, device=dev)

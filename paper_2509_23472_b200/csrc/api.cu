@@ -118,9 +118,12 @@ void carve_basis(Carver& c, const Plan& p, BasisWs* w) {
   if (p.bf16) {
     w->Lh = (__nv_bfloat16*)c.take(l * l * 2);
     w->Ll = (__nv_bfloat16*)c.take(l * l * 2);
-    // r <= 256 needs none (shared-memory kernel); above that the two-level scheme keeps W, X and two 256 x 256
-    // temporaries here
-    w->sb_scratch = c.take((2 * l * l + 2 * 256 * 256) * sizeof(float));
+    // r <= 256 needs none (shared-memory kernel); above that the block scheme keeps W, X and, per level, two
+    // (width - 256) x 256 temporaries here
+    const size_t lvl1 = l > 256 ? l - 256 : 0, lvl2 = l > 512 ? l - 512 : 0;
+    size_t tmp = 2 * 256 * (lvl1 + lvl2);
+    if (tmp < 2 * 256 * 256) tmp = 2 * 256 * 256;
+    w->sb_scratch = c.take((2 * l * l + tmp) * sizeof(float));
     const size_t gs = (size_t)(p.splits_gs > p.splits_w ? p.splits_gs : p.splits_w);
     w->gram_partials = (float*)c.take(gs * l * l * 4);
     w->Yh = (__nv_bfloat16*)c.take(n * l * 2);
@@ -554,7 +557,7 @@ loract_status_t loract_prenorm_backward(const loract_desc_t* desc, const void* U
 size_t loract_rsvd_workspace_bytes(const loract_desc_t* desc, int32_t oversample) {
   if (check_desc(desc) != LORACT_OK || desc->dtype != LORACT_BF16) return 0;
   const int l = desc->rank + oversample;
-  if (oversample < 0 || l % 8 || l > 512 || l > desc->n_tokens || l > desc->d) return 0;
+  if (oversample < 0 || oversample > 128 || l % 8 || l > 640 || l > desc->n_tokens || l > desc->d) return 0;
   Plan plan = make_plan(desc->n_tokens, desc->d, l, true);
   Carver c(nullptr);
   c.take(256);
@@ -704,7 +707,7 @@ loract_status_t loract_debug_small_block(int32_t r, const void* partials, int32_
                                          int64_t partial_stride, int32_t use_f64, float shift_rel, void* scratch,
                                          float* linv_f32, void* linv_hi, void* linv_lo, uint32_t* status_word,
                                          void* stream) {
-  if (r < 16 || r > 512 || r % 8 || !partials || !scratch || n_partials < 1) return LORACT_ERR_INVALID_ARG;
+  if (r < 16 || r > 640 || r % 8 || !partials || !scratch || n_partials < 1) return LORACT_ERR_INVALID_ARG;
   SmallBlockArgs a;
   a.r = r; a.partials = partials; a.partial_type = partial_f64 ? ELEM_F64 : ELEM_F32;
   a.n_partials = n_partials; a.partial_stride = partial_stride; a.use_f64 = use_f64 != 0;

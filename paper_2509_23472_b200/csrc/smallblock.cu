@@ -272,27 +272,40 @@ cudaError_t launch_typed(const SBParams& p, cudaStream_t stream) {
 
 }  // namespace
 
-// 256 < r <= 512 in fp32: the matrix as 2 x 2 blocks, W = [W11 . ; W21 W22], the leading block 256 wide.
+// r > 256 in fp32: the matrix as 2 x 2 blocks, W = [W11 . ; W21 W22], the leading block 256 wide.
 //   L11 = chol(W11), X11 = L11^-1            (shared-memory cluster kernel)
 //   L21 = W21 X11^T,  S = W22 - L21 L21^T    (fp32 CUDA-core products)
-//   L22 = chol(S), X22 = L22^-1              (shared-memory cluster kernel)
+//   L22 = chol(S), X22 = L22^-1              (the same again if S is wider than 256, else the cluster kernel)
 //   X21 = -X22 (L21 X11)                     (fp32 CUDA-core products)
-// scratch: W (r x r) + X (r x r) + two 256 x 256 temporaries, fp32.
-cudaError_t small_block_two_level(const SmallBlockArgs& a, cudaStream_t stream) {
-  const int r = a.r, r1 = 256, r2 = r - r1;
-  float* W = (float*)a.scratch;
-  float* X = a.linv_f32 ? a.linv_f32 : W + (size_t)r * r;
-  float* T1 = W + 2 * (size_t)r * r;
-  float* T2 = T1 + (size_t)r1 * r1;
-  LORACT_CUDA_TRY(reduce_partials_launch((const float*)a.partials, a.n_partials, a.partial_stride, (int64_t)r * r, W,
-                                         nullptr, stream));
-  if (a.linv_f32) LORACT_CUDA_TRY(cudaMemsetAsync(X, 0, (size_t)r * r * 4, stream));
-  LORACT_CUDA_TRY(cudaMemsetAsync(a.linv_hi, 0, (size_t)r * r * 2, stream));   // the block above the diagonal
-  if (a.linv_lo) LORACT_CUDA_TRY(cudaMemsetAsync(a.linv_lo, 0, (size_t)r * r * 2, stream));
-  SmallBlockArgs s1 = a;
-  s1.r = r1; s1.partials = W; s1.n_partials = 1; s1.partial_stride = 0; s1.in_ld = r; s1.out_ld = r;
-  s1.linv_f32 = X; s1.scratch = nullptr;
-  LORACT_CUDA_TRY(small_block_cluster_launch(s1, stream));
+// W (n x n, leading dimension ld) is overwritten by the Schur complements; X (fp32) and the bf16 pair receive the
+// inverse factor at the same place and leading dimension.  T: 2 * 256 * (n - 256) floats for this level's two
+// temporaries, followed by what the levels below need.  The shift and the pivot floor of every level come from
+// the diagonal of the whole matrix's leading block (`scale`): a Schur complement may be nothing but rounding noise.
+struct TwoLevelCtx {
+  float shift_rel;
+  uint32_t* dev_status;
+  int64_t ld;
+  const float* scale_diag;
+  int scale_n;
+  cudaStream_t stream;
+};
+
+cudaError_t factor_blocks(const TwoLevelCtx& c, float* W, float* X, __nv_bfloat16* hi, __nv_bfloat16* lo, int n,
+                          float* T, bool top) {
+  const int64_t ld = c.ld;
+  if (n <= 256) {
+    SmallBlockArgs s;
+    s.r = n; s.partials = W; s.partial_type = ELEM_F32; s.n_partials = 1; s.partial_stride = 0;
+    s.use_f64 = false; s.shift_rel = c.shift_rel; s.in_ld = ld; s.out_ld = ld;
+    s.linv_f32 = X; s.linv_hi = hi; s.linv_lo = lo; s.dev_status = c.dev_status;
+    if (!top) { s.scale_diag = c.scale_diag; s.scale_n = c.scale_n; s.scale_ld = ld; }
+    return small_block_cluster_launch(s, c.stream);
+  }
+  const int r1 = 256, r2 = n - r1;
+  float* T1 = T;
+  float* T2 = T1 + (size_t)r2 * r1;
+  float* Tnext = T2 + (size_t)r2 * r1;
+  LORACT_CUDA_TRY(factor_blocks(c, W, X, hi, lo, r1, Tnext, top));
   auto simt = [&](int M, int N, int K, const float* A, int64_t lda, const float* B, int64_t ldb, bool b_mn, float* C,
                   int64_t ldc, float alpha, bool accumulate) {
     GemmDesc g;
@@ -300,33 +313,45 @@ cudaError_t small_block_two_level(const SmallBlockArgs& a, cudaStream_t stream) 
     g.a_type = g.b_type = ELEM_F32;
     g.terms[0] = {A, B};
     g.out = OUT_F32; g.C0 = C; g.ldc = ldc; g.alpha = alpha; g.accumulate = accumulate;
-    return gemm_f32_small_launch(g, stream);
+    return gemm_f32_small_launch(g, c.stream);
   };
-  const float* W21 = W + (size_t)r1 * r;
-  float* W22 = W + (size_t)r1 * r + r1;
+  const float* W21 = W + (size_t)r1 * ld;
+  float* W22 = W + (size_t)r1 * ld + r1;
+  float* X22 = X + (size_t)r1 * ld + r1;
+  float* X21 = X + (size_t)r1 * ld;
   // L21 = W21 X11^T : C[m][n] = sum_k W21[m][k] X11[n][k]
-  LORACT_CUDA_TRY(simt(r2, r1, r1, W21, r, X, r, false, T1, r1, 1.f, false));
+  LORACT_CUDA_TRY(simt(r2, r1, r1, W21, ld, X, ld, false, T1, r1, 1.f, false));
   // S = W22 - L21 L21^T, in place
-  LORACT_CUDA_TRY(simt(r2, r2, r1, T1, r1, T1, r1, false, W22, r, -1.f, true));
-  SmallBlockArgs s2 = s1;
-  s2.r = r2; s2.partials = W22; s2.linv_f32 = X + (size_t)r1 * r + r1;
-  s2.linv_hi = a.linv_hi + (size_t)r1 * r + r1;
-  s2.linv_lo = a.linv_lo ? a.linv_lo + (size_t)r1 * r + r1 : nullptr;
-  // shift and pivot floor on the scale of W: S may be nothing but rounding noise of W22 - L21 L21^T, and a floor
-  // taken from its own diagonal would then let that noise through as pivots
-  s2.scale_diag = W; s2.scale_n = r1; s2.scale_ld = r;
-  LORACT_CUDA_TRY(small_block_cluster_launch(s2, stream));
+  LORACT_CUDA_TRY(simt(r2, r2, r1, T1, r1, T1, r1, false, W22, ld, -1.f, true));
+  LORACT_CUDA_TRY(factor_blocks(c, W22, X22, hi + (size_t)r1 * ld + r1, lo ? lo + (size_t)r1 * ld + r1 : nullptr, r2,
+                                Tnext, false));
   // X21 = -X22 (L21 X11): T2[m][n] = sum_k L21[m][k] X11[k][n];  X21[m][n] = -sum_k X22[m][k] T2[k][n]
-  LORACT_CUDA_TRY(simt(r2, r1, r1, T1, r1, X, r, true, T2, r1, 1.f, false));
-  float* X21 = X + (size_t)r1 * r;
-  LORACT_CUDA_TRY(simt(r2, r1, r2, X + (size_t)r1 * r + r1, r, T2, r1, true, X21, r, -1.f, false));
-  return split_block_launch(X21, r2, r1, r, a.linv_hi + (size_t)r1 * r, a.linv_lo ? a.linv_lo + (size_t)r1 * r : nullptr,
-                            stream);
+  LORACT_CUDA_TRY(simt(r2, r1, r1, T1, r1, X, ld, true, T2, r1, 1.f, false));
+  LORACT_CUDA_TRY(simt(r2, r1, r2, X22, ld, T2, r1, true, X21, ld, -1.f, false));
+  return split_block_launch(X21, r2, r1, ld, hi + (size_t)r1 * ld, lo ? lo + (size_t)r1 * ld : nullptr, c.stream);
+}
+
+// scratch: W (r x r) + X (r x r) + the temporaries of every level, fp32.
+cudaError_t small_block_two_level(const SmallBlockArgs& a, cudaStream_t stream) {
+  const int r = a.r;
+  float* W = (float*)a.scratch;
+  float* X = a.linv_f32 ? a.linv_f32 : W + (size_t)r * r;
+  float* T = W + 2 * (size_t)r * r;
+  LORACT_CUDA_TRY(reduce_partials_launch((const float*)a.partials, a.n_partials, a.partial_stride, (int64_t)r * r, W,
+                                         nullptr, stream));
+  // blocks above the diagonal are never written below: X is read as a whole by the products of the next level up
+  LORACT_CUDA_TRY(cudaMemsetAsync(X, 0, (size_t)r * r * 4, stream));
+  LORACT_CUDA_TRY(cudaMemsetAsync(a.linv_hi, 0, (size_t)r * r * 2, stream));
+  if (a.linv_lo) LORACT_CUDA_TRY(cudaMemsetAsync(a.linv_lo, 0, (size_t)r * r * 2, stream));
+  TwoLevelCtx c;
+  c.shift_rel = a.shift_rel; c.dev_status = a.dev_status; c.ld = r; c.scale_diag = W; c.scale_n = 256;
+  c.stream = stream;
+  return factor_blocks(c, W, X, a.linv_hi, a.linv_lo, r, T, true);
 }
 
 cudaError_t small_block_launch(const SmallBlockArgs& a, cudaStream_t stream) {
   if (small_block_cluster_supported(a)) return small_block_cluster_launch(a, stream);
-  if (!a.use_f64 && a.partial_type == ELEM_F32 && a.r > 256 && a.r <= 512 && a.r % 8 == 0 && !a.linv_full &&
+  if (!a.use_f64 && a.partial_type == ELEM_F32 && a.r > 256 && a.r <= 768 && a.r % 8 == 0 && !a.linv_full &&
       a.linv_hi && a.in_ld == 0 && a.out_ld == 0 && (((uintptr_t)a.partials & 15) == 0) &&
       (a.partial_stride % 4 == 0))
     return small_block_two_level(a, stream);

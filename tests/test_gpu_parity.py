@@ -211,10 +211,10 @@ def test_rsvd_comparator(dev):
     assert e_l <= gpu_err(X64, Q0, B0) + 2e-3
 
 
-@pytest.mark.parametrize("r", [128, 256])
+@pytest.mark.parametrize("r", [128, 256, 512])
 def test_rsvd_comparator_oversampled_ranks(dev, r):
-    # l = r + 8 at the ranks of the sweep: 136 (one accumulator tile, ragged) and 264 (two-level small block)
-    w = synth.scaled(synth.llama13b_sweep_point(1024, r), n_tokens=3072, d=1024, rank=r, signal_rank=512)
+    # l = r + 8 at the ranks of the sweep: 136 (one accumulator tile, ragged), 264 and 520 (block small-block scheme)
+    w = synth.scaled(synth.llama13b_sweep_point(1024, r), n_tokens=3072, d=1024, rank=r, signal_rank=768 if r == 512 else 512)
     X = synth.make_inputs(w, device=dev)["X"]
     Q, Bm = B.rsvd(X, r, oversample=8, power_iters=1, seed=4)
     assert Q.shape == (3072, r + 8)

@@ -33,7 +33,7 @@ def spd(r: int, cond: float, seed: int) -> np.ndarray:
                                               (96, 1, 1e4), (128, 5, 1e5), (160, 2, 1e3), (192, 1, 1e3),
                                               (208, 3, 1e4), (224, 1, 1e2), (240, 2, 1e5), (256, 16, 1e5),
                                               (256, 1, 1.5), (272, 2, 1e3), (320, 1, 1e4), (384, 3, 1e5),
-                                              (496, 2, 1e3), (512, 4, 1e4)])
+                                              (496, 2, 1e3), (512, 4, 1e4), (520, 1, 1e3), (640, 2, 1e4)])
 def test_inverse_cholesky_factor(dev, r, n_partials, cond):
     W = spd(r, cond, seed=r + n_partials)
     rng = np.random.default_rng(7)
