@@ -16,6 +16,10 @@ What follows the paper, and where:
   * ``norm_forward`` / ``compress_prenorm`` / ``prenorm_backward``
                        Section 3.3, the pre-norm unit and its three gradient
                        equations
+  * ``activation_forward`` / ``activation_backward``
+                       Section 3.1, the gradient equation for an element-wise
+                       Z = f(X) whose saved activation A = X is compressed:
+                       grad_X = grad_Z * f'(A~)
   * ``truncated_svd``  Section 3.2 (the Eckart-Young optimum, yardstick)
   * ``rsvd``           Section 3.2: the same steps as Algorithm 1 with the
                        sampled rows replaced by a Gaussian test matrix
@@ -238,6 +242,42 @@ def prenorm_backward_rms(A_tilde, gamma, rstd, grad_A):
     gXbar = _f64(grad_A) * gamma[None, :]
     inner = np.mean(gXbar * Xbar, axis=1)
     return _f64(rstd)[:, None] * (gXbar - Xbar * inner[:, None])
+
+
+# --------------------------------------------------------------------------
+# Element-wise consumers (Section 3.1: the derivative of Z = f(X) is taken at A~)
+# --------------------------------------------------------------------------
+def _std_normal_cdf(a):
+    from math import erf, sqrt
+    return 0.5 * (1.0 + np.vectorize(erf)(a / sqrt(2.0)))
+
+
+def activation_forward(A, kind: str = "silu"):
+    """Z = f(A) element-wise.  "silu": a / (1 + exp(-a));  "gelu": a * Phi(a), Phi the standard normal
+    distribution function (the exact form, not the tanh approximation)."""
+    A = _f64(A)
+    if kind == "silu":
+        return A / (1.0 + np.exp(-A))
+    if kind == "gelu":
+        return A * _std_normal_cdf(A)
+    raise ValueError(kind)
+
+
+def activation_backward(A_tilde, grad_Z, kind: str = "silu"):
+    """grad_X = grad_Z * f'(A~), the gradient equation of Section 3.1 for an element-wise f.
+
+    silu: f'(a) = s (1 + a (1 - s)), s = 1 / (1 + exp(-a));
+    gelu: f'(a) = Phi(a) + a phi(a), phi the standard normal density.
+    """
+    a = _f64(A_tilde)
+    if kind == "silu":
+        s = 1.0 / (1.0 + np.exp(-a))
+        d = s * (1.0 + a * (1.0 - s))
+    elif kind == "gelu":
+        d = _std_normal_cdf(a) + a * np.exp(-0.5 * a * a) / np.sqrt(2.0 * np.pi)
+    else:
+        raise ValueError(kind)
+    return _f64(grad_Z) * d
 
 
 # --------------------------------------------------------------------------

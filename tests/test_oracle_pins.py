@@ -334,3 +334,28 @@ def test_sampled_versus_gaussian_test_matrix_report_only():
     opt = orc.rel_fro_error(A, *orc.truncated_svd(A, k))
     print(f"sampled {lo:.3e}  gaussian {rs:.3e}  optimum {opt:.3e}")
     assert opt <= lo and opt <= rs
+
+
+# ------------------------------------------------------------------ element-wise consumers (Section 3.1)
+@pytest.mark.parametrize("kind", ["silu", "gelu"])
+def test_activation_backward_is_the_derivative_of_the_forward(kind):
+    """Pins activation_backward to something other than its own formula: central differences of
+    activation_forward, and values that are known in closed form."""
+    rng = np.random.default_rng(5)
+    a = rng.uniform(-6.0, 6.0, size=(7, 11))
+    g = rng.standard_normal((7, 11))
+    h = 1e-5
+    fd = (orc.activation_forward(a + h, kind) - orc.activation_forward(a - h, kind)) / (2 * h)
+    assert np.allclose(orc.activation_backward(a, g, kind), g * fd, rtol=1e-7, atol=1e-9)
+    one = np.ones(1)
+    # f'(0) = 1/2 for both; f' -> 1 far to the right and -> 0 far to the left
+    assert abs(orc.activation_backward(np.zeros(1), one, kind)[0] - 0.5) < 1e-15
+    assert abs(orc.activation_backward(np.array([40.0]), one, kind)[0] - 1.0) < 1e-12
+    assert abs(orc.activation_backward(np.array([-40.0]), one, kind)[0]) < 1e-12
+    # forward: silu(1) = 1 / (1 + 1/e), gelu(1) = Phi(1) = 0.841344746...
+    want = 1.0 / (1.0 + np.exp(-1.0)) if kind == "silu" else 0.8413447460685429
+    assert abs(orc.activation_forward(np.ones(1), kind)[0] - want) < 1e-14
+    # silu'(a) + silu'(-a) = 1 and gelu'(a) + gelu'(-a) = 1 (odd part of f is a / 2)
+    assert np.allclose(orc.activation_backward(a, one, kind) + orc.activation_backward(-a, one, kind), 1.0, atol=1e-12)
+    # linear in grad_Z
+    assert np.allclose(orc.activation_backward(a, 3.0 * g, kind), 3.0 * orc.activation_backward(a, g, kind))
