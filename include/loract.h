@@ -48,6 +48,7 @@ typedef enum {
 
 typedef enum { LORACT_F32 = 0, LORACT_BF16 = 1 } loract_dtype_t;
 typedef enum { LORACT_NORM_RMS = 0, LORACT_NORM_LAYER = 1 } loract_norm_t;
+typedef enum { LORACT_ACT_SILU = 0, LORACT_ACT_GELU = 1 } loract_act_t;
 
 /* Bits of the device status word (see loract_read_device_status). */
 #define LORACT_DEV_PIVOT_CLAMPED 0x1u  /* a Cholesky pivot was not positive and was clamped       */
@@ -125,6 +126,17 @@ size_t loract_prenorm_backward_workspace_bytes(const loract_desc_t* desc);
 loract_status_t loract_prenorm_backward(const loract_desc_t* desc, const void* U, const void* V,
                                         const void* gamma, const float* rstd, const void* grad_A,
                                         void* grad_X, void* ws, size_t ws_bytes, void* stream);
+
+/* Section 3.1, the gradient equation grad_X = grad_Z * dZ/dX taken at the reconstructed activation, for an
+ * element-wise Z = f(X) whose saved input A = X was compressed to (U, V):  grad_X = grad_Z * f'(A~), A~ = U V.
+ *   LORACT_ACT_SILU : f(a) = a / (1 + exp(-a)),  f'(a) = s (1 + a (1 - s)), s = 1 / (1 + exp(-a))
+ *   LORACT_ACT_GELU : f(a) = a Phi(a) (exact form), f'(a) = Phi(a) + a phi(a)
+ * grad_Z: device, n_tokens x d, row stride ldx.  grad_X: device, n_tokens x d, row stride ldx, written.  A~ is
+ * never stored: its tiles exist only in tensor memory, inside the kernel that writes grad_X (grad_Z is read
+ * once, grad_X written once, the factors read once).  bf16 only (LORACT_ERR_UNSUPPORTED for fp32).  Needs no
+ * workspace. */
+loract_status_t loract_activation_backward(const loract_desc_t* desc, const void* U, const void* V,
+                                           const void* grad_Z, int32_t kind, void* grad_X, void* stream);
 
 /* The same result as loract_weight_grad, for callers that cannot allocate device memory and so cannot
  * provide `ws`.  (The paper has no counterpart: this is a property of the library, not of the method.)

@@ -22,7 +22,7 @@ DEV_PIVOT_CLAMPED, DEV_WAIT_EXPIRED, DEV_SAMPLER_SHORT, DEV_NONFINITE = 1, 2, 4,
 EXPORTS = (
     "loract_workspace_bytes", "loract_sample_indices", "loract_compress", "loract_reconstruct",
     "loract_weight_grad", "loract_weight_grad_static", "loract_weight_grad_static_status", "loract_compress_prenorm",
-    "loract_prenorm_backward_workspace_bytes", "loract_prenorm_backward", "loract_rsvd_workspace_bytes", "loract_rsvd",
+    "loract_prenorm_backward_workspace_bytes", "loract_prenorm_backward", "loract_activation_backward", "loract_rsvd_workspace_bytes", "loract_rsvd",
     "loract_read_device_status", "loract_status_from_device_word", "loract_status_string",
     "loract_kernel_launch_count",
 )
@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
         l.loract_prenorm_backward_workspace_bytes.argtypes = [dp]
         l.loract_prenorm_backward.restype = ctypes.c_int
         l.loract_prenorm_backward.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        l.loract_activation_backward.restype = ctypes.c_int
+        l.loract_activation_backward.argtypes = [dp, vp, vp, vp, i32, vp, vp]
         l.loract_rsvd_workspace_bytes.restype = sz
         l.loract_rsvd_workspace_bytes.argtypes = [dp, i32]
         l.loract_rsvd.restype = ctypes.c_int
@@ -274,10 +276,28 @@ def prenorm_backward(U: torch.Tensor, V: torch.Tensor, gamma: torch.Tensor, rstd
     if need == 0:
         raise LoractError(1, "loract_prenorm_backward_workspace_bytes")
     ws = ws if ws is not None else torch.empty(need, dtype=torch.uint8, device=U.device)
-    grad_X = torch.empty_like(grad_A)
+    grad_X = torch.empty_strided((n, d), (grad_A.stride(0), 1), dtype=grad_A.dtype, device=grad_A.device)
     _check(lib().loract_prenorm_backward(ctypes.byref(desc), _ptr(U), _ptr(V), _ptr(gamma), _ptr(rstd), _ptr(grad_A),
                                          _ptr(grad_X), _ptr(ws), ws.numel(), _stream(U.device)),
            "loract_prenorm_backward")
+    return grad_X
+
+
+ACT_SILU, ACT_GELU = 0, 1
+
+
+def activation_backward(U: torch.Tensor, V: torch.Tensor, grad_Z: torch.Tensor, kind: int = ACT_SILU) -> torch.Tensor:
+    """grad_X = grad_Z * f'(U V) for an element-wise activation whose input was compressed (Section 3.1)."""
+    for t, what in ((U, "U"), (V, "V"), (grad_Z, "grad_Z")):
+        _cuda(t, what)
+    n, r = U.shape
+    d = V.shape[1]
+    if grad_Z.shape != (n, d) or grad_Z.stride(1) != 1:
+        raise ValueError("grad_Z must be a row-major (n_tokens x d) tensor")
+    desc = Desc(n, d, grad_Z.stride(0), r, 0, _dtype_code(U), 0, 0, 0)
+    grad_X = torch.empty_strided((n, d), (grad_Z.stride(0), 1), dtype=grad_Z.dtype, device=grad_Z.device)
+    _check(lib().loract_activation_backward(ctypes.byref(desc), _ptr(U), _ptr(V), _ptr(grad_Z), kind, _ptr(grad_X),
+                                            _stream(U.device)), "loract_activation_backward")
     return grad_X
 
 

@@ -554,6 +554,27 @@ loract_status_t loract_prenorm_backward(const loract_desc_t* desc, const void* U
   return from_cuda(e);
 }
 
+loract_status_t loract_activation_backward(const loract_desc_t* desc, const void* U, const void* V,
+                                           const void* grad_Z, int32_t kind, void* grad_X, void* stream) {
+  loract_status_t s = check_desc(desc);
+  if (s != LORACT_OK) return s;
+  if (desc->dtype != LORACT_BF16) return LORACT_ERR_UNSUPPORTED;
+  if (kind != LORACT_ACT_SILU && kind != LORACT_ACT_GELU) return LORACT_ERR_INVALID_ARG;
+  if (!U || !V || !grad_Z || !grad_X) return LORACT_ERR_INVALID_ARG;
+  if (misaligned(U) || misaligned(V) || misaligned(grad_Z) || misaligned(grad_X)) return LORACT_ERR_ALIGNMENT;
+  // grad_X = grad_Z * f'(A~), A~ = U V tile by tile in tensor memory only: the epilogue of the reconstruct
+  // contraction takes the derivative and multiplies
+  GemmDesc g;
+  g.M = (int)desc->n_tokens; g.N = (int)desc->d; g.K = desc->rank; g.b_mn = true;
+  g.lda = desc->rank; g.ldb = desc->d;
+  g.terms[0] = {U, V};
+  g.out = OUT_ACT_BWD; g.C0 = grad_X; g.ldc = desc->ldx;
+  g.ep_E = grad_Z; g.ep_ld = desc->ldx; g.ep_kind = kind;
+  trace_label("activation backward: grad_X");
+  if (!gemm_tc_supported(g)) return LORACT_ERR_UNSUPPORTED;
+  return from_cuda(gemm_tc_launch(g, nullptr, (cudaStream_t)stream));
+}
+
 size_t loract_rsvd_workspace_bytes(const loract_desc_t* desc, int32_t oversample) {
   if (check_desc(desc) != LORACT_OK || desc->dtype != LORACT_BF16) return 0;
   const int l = desc->rank + oversample;

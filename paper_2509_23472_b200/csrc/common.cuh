@@ -63,7 +63,10 @@ enum OutMode : int {
   OUT_F64 = 3,    // C0: double (SIMT path only)
   // C0: bf16, C0[m][n] = row_a[m] * col[n] * E[m][n] - row_b[m] / col[n] * acc[m][n]  (tensor-core path only):
   // the input gradient of the RMS pre-norm unit from a reconstructed tile that is never stored
-  OUT_RMS_BWD = 4
+  OUT_RMS_BWD = 4,
+  // C0: bf16, C0[m][n] = E[m][n] * f'(acc[m][n]), f = SiLU (ep_kind 0) or GELU (ep_kind 1)  (tensor-core path
+  // only): the input gradient of an element-wise activation from a reconstructed tile that is never stored
+  OUT_ACT_BWD = 5
 };
 
 enum ElemType : int { ELEM_F32 = 0, ELEM_BF16 = 1, ELEM_F64 = 2 };
@@ -96,6 +99,7 @@ struct GemmDesc {
   const float* ep_row_a = nullptr;
   const float* ep_row_b = nullptr;
   const void* ep_col = nullptr;
+  int ep_kind = 0;         // OUT_ACT_BWD: which activation
 };
 
 // tcgen05 engine: bf16 operands, fp32 accumulation in tensor memory.  Returns cudaErrorNotSupported

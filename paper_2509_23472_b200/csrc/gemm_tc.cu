@@ -56,6 +56,7 @@ struct TcParams {
   const float* ep_row_a;
   const float* ep_row_b;
   const void* ep_col;
+  int ep_kind;        // OUT_ACT_BWD: 0 SiLU, 1 GELU
   uint32_t* dev_status;
   int tma_store;      // 1: the epilogue stages 32-row boxes in shared memory and writes them with TMA stores
   int st_m_tiles;     // streaming kernel: 256-row tiles along M
@@ -158,6 +159,16 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
+// f'(a) of the element-wise consumers (OUT_ACT_BWD).  SiLU: s (1 + a (1 - s)), s the logistic function;
+// GELU (exact form): Phi(a) + a phi(a).  The result is multiplied by the upstream gradient and rounded to bf16.
+__device__ __forceinline__ float act_derivative(float a, int kind) {
+  if (kind == 0) {
+    const float s = 1.f / (1.f + __expf(-a));
+    return s * (1.f + a * (1.f - s));
+  }
+  return 0.5f * (1.f + erff(a * 0.70710678118f)) + a * 0.39894228040f * __expf(-0.5f * a * a);
+}
+
 // ---- staged epilogue.  A thread owns one accumulator row, so a direct store instruction of a warp touches 32
 // different rows, 16 bytes each: every 128-byte line of the output is written in eight pieces by eight
 // instructions.  Instead each epilogue warp puts its 32 rows x 128 bytes into shared memory in the layout of a
@@ -236,6 +247,7 @@ __device__ __forceinline__ void tc_store_tile_staged(const TcParams& p, const Tm
   }
   const bool split_out = p.out == OUT_SPLIT;
   const bool rms = p.out == OUT_RMS_BWD;
+  const bool act = p.out == OUT_ACT_BWD;
   const bool live = m < p.M;                                 // rows past M are clipped by the store
   float ra = 0.f, rb = 0.f;
   if (rms && live) { ra = p.ep_row_a[m]; rb = p.ep_row_b[m]; }
@@ -274,6 +286,33 @@ __device__ __forceinline__ void tc_store_tile_staged(const TcParams& p, const Tm
               if (nn < p.N) {
                 const float c = __bfloat162float(col[8 * q + h]);
                 const float r = ra * c * __bfloat162float(e[8 * q + h]) - rb * __uint_as_float(v[8 * q + h]) / c;
+                const uint32_t bits = (uint32_t)__bfloat16_as_ushort(__float2bfloat16(r));
+                ow[h >> 1] |= (h & 1) ? (bits << 16) : bits;
+              }
+            }
+          }
+          stage_write16(box_hi, lane, 4 * half + q, make_uint4(ow[0], ow[1], ow[2], ow[3]));
+        }
+      } else if (act) {
+        const bool cols_ok = n + 32 <= p.N;
+        const __nv_bfloat16* e = (const __nv_bfloat16*)p.ep_E + (int64_t)m * p.ep_ld + n;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t ow[4] = {0u, 0u, 0u, 0u};
+          if (live && cols_ok) {
+            const uint4 ev = reinterpret_cast<const uint4*>(e)[q];
+            const uint32_t ew[4] = {ev.x, ev.y, ev.z, ev.w};
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              const float e0 = __uint_as_float(ew[h] << 16), e1 = __uint_as_float(ew[h] & 0xffff0000u);
+              const float a0 = __uint_as_float(v[8 * q + 2 * h]), a1 = __uint_as_float(v[8 * q + 2 * h + 1]);
+              ow[h] = pack_bf16x2(e0 * act_derivative(a0, p.ep_kind), e1 * act_derivative(a1, p.ep_kind));
+            }
+          } else if (live) {
+            for (int h = 0; h < 8; ++h) {
+              const int nn = n + 8 * q + h;
+              if (nn < p.N) {
+                const float r = __bfloat162float(e[8 * q + h]) * act_derivative(__uint_as_float(v[8 * q + h]), p.ep_kind);
                 const uint32_t bits = (uint32_t)__bfloat16_as_ushort(__float2bfloat16(r));
                 ow[h >> 1] |= (h & 1) ? (bits << 16) : bits;
               }
@@ -377,6 +416,12 @@ __device__ __forceinline__ void tc_store_tile(const TcParams& p, const TmapPack&
             dst[q] = __float2bfloat16(ra * c * __bfloat162float(e[q]) - rb * __uint_as_float(v[q]) / c);
           }
         }
+      } else if (p.out == OUT_ACT_BWD) {
+        // grad_X = grad_Z * f'(reconstructed A): the tile of the reconstructed activation exists only here
+        __nv_bfloat16* dst = (__nv_bfloat16*)p.C0 + (int64_t)m * p.ldc + n;
+        const __nv_bfloat16* e = (const __nv_bfloat16*)p.ep_E + (int64_t)m * p.ep_ld + n;
+        for (int q = 0; q < valid; ++q)
+          dst[q] = __float2bfloat16(__bfloat162float(e[q]) * act_derivative(__uint_as_float(v[q]), p.ep_kind));
       } else {
         __nv_bfloat16* dst_hi = (__nv_bfloat16*)p.C0 + (int64_t)m * p.ldc + n;
         __nv_bfloat16* dst_lo = (p.out == OUT_SPLIT) ? (__nv_bfloat16*)p.C1 + (int64_t)m * p.ldc + n : nullptr;
@@ -1115,7 +1160,9 @@ cudaError_t gemm_tc_wait_probe_launch(uint32_t* dev_status, uint64_t limit_ns, c
 
 bool gemm_tc_supported(const GemmDesc& g) {
   if (g.a_type != ELEM_BF16 || g.b_type != ELEM_BF16) return false;
-  if (!(g.out == OUT_F32 || g.out == OUT_BF16 || g.out == OUT_SPLIT || g.out == OUT_RMS_BWD)) return false;
+  if (!(g.out == OUT_F32 || g.out == OUT_BF16 || g.out == OUT_SPLIT || g.out == OUT_RMS_BWD || g.out == OUT_ACT_BWD))
+    return false;
+  if (g.out == OUT_ACT_BWD && (!g.ep_E || g.splits > 1 || g.ep_kind < 0 || g.ep_kind > 1)) return false;
   if (g.out == OUT_RMS_BWD && (!g.ep_E || !g.ep_row_a || !g.ep_row_b || !g.ep_col || g.splits > 1)) return false;
   if (g.M < 1 || g.N < 1 || g.K < 1 || g.n_terms < 1 || g.n_terms > 3) return false;
   if (g.lda % 8 || g.ldb % 8) return false;
@@ -1155,6 +1202,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   while ((int)p.tmem_cols < p.bn) p.tmem_cols *= 2;
   p.accumulate = g.accumulate ? 1 : 0;
   p.ep_E = g.ep_E; p.ep_ld = g.ep_ld; p.ep_row_a = g.ep_row_a; p.ep_row_b = g.ep_row_b; p.ep_col = g.ep_col;
+  p.ep_kind = g.ep_kind;
   p.dev_status = dev_status;
   p.st_m_tiles = 0; p.st_units = 0; p.tma_store = 0;
 
@@ -1177,6 +1225,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
     if (g.out == OUT_SPLIT && ((uintptr_t)g.C1 & 15)) return false;
     if (splits > 1 && g.split_stride != (int64_t)g.M * g.ldc) return false;
     if (g.out == OUT_RMS_BWD && (((uintptr_t)g.ep_E & 15) || ((uintptr_t)g.ep_col & 15) || g.ep_ld % 8)) return false;
+    if (g.out == OUT_ACT_BWD && (((uintptr_t)g.ep_E & 15) || g.ep_ld % 8)) return false;
     return true;
   };
   auto make_out_maps = [&]() -> cudaError_t {

@@ -319,3 +319,34 @@ def test_prenorm_backward_matches_the_three_gradient_equations(dev, n, d, r):
     err_A = np.linalg.norm(A_tilde - to64(A)) / np.linalg.norm(to64(A))
     rel_exact = np.linalg.norm(to64(gX) - exact) / np.linalg.norm(exact)
     assert rel_exact <= 2.0 * err_A + 1e-2, (rel_exact, err_A)
+
+
+# ------------------------------------------------------------------ element-wise consumer (Section 3.1)
+@pytest.mark.parametrize("kind,name", [(B.ACT_SILU, "silu"), (B.ACT_GELU, "gelu")])
+@pytest.mark.parametrize("n,d,r", [(1024, 512, 64), (1000, 776, 96), (4096, 2048, 256)])
+def test_activation_backward_matches_the_gradient_equation(dev, kind, name, n, d, r):
+    """grad_X = grad_Z * f'(A~) with A~ = U V never stored: the device against the oracle's equation on the same
+    stored factors (this isolates the consumer), and against the exact gradient at the uncompressed input."""
+    w = synth.scaled(synth.WORKLOADS["llama7b_block"], n_tokens=n, d=d, rank=r, signal_rank=min(2 * r, d // 2))
+    X = synth.make_inputs(w, device=dev)["X"]
+    X = (X.float() * (2.0 / float(X.float().std()))).to(X.dtype)      # entries of a few units: f' is not flat there
+    U, V, _ = B.compress(X, r, seed=w.seed)
+    g = torch.Generator(device=dev)
+    g.manual_seed(91)
+    gZ = torch.randn(n, d, generator=g, device=dev).to(X.dtype)
+    gX = B.activation_backward(U, V, gZ, kind)
+    torch.cuda.synchronize()
+    assert gX.shape == (n, d) and gX.dtype == X.dtype
+    A_tilde = to64(U) @ to64(V)
+    want = orc.activation_backward(A_tilde, to64(gZ), name)
+    rel = np.linalg.norm(to64(gX) - want) / np.linalg.norm(want)
+    assert rel <= 1e-2, rel                     # bf16 output: 2^-9 per entry
+    exact = orc.activation_backward(to64(X), to64(gZ), name)
+    err_A = np.linalg.norm(A_tilde - to64(X)) / np.linalg.norm(to64(X))
+    rel_exact = np.linalg.norm(to64(gX) - exact) / np.linalg.norm(exact)
+    assert rel_exact <= 2.0 * err_A + 1e-2, (rel_exact, err_A)   # |f''| <= 1/2: the compression error, not more
+    # a row stride larger than d, and nothing written past d
+    wide_in = torch.zeros(n, d + 64, dtype=X.dtype, device=dev)
+    wide_in[:, :d] = gZ
+    out = B.activation_backward(U, V, wide_in[:, :d], kind)
+    assert out.stride(0) == d + 64 and torch.equal(out, gX)
