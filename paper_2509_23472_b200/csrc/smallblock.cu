@@ -351,7 +351,7 @@ cudaError_t small_block_two_level(const SmallBlockArgs& a, cudaStream_t stream) 
 
 cudaError_t small_block_launch(const SmallBlockArgs& a, cudaStream_t stream) {
   if (small_block_cluster_supported(a)) return small_block_cluster_launch(a, stream);
-  if (!a.use_f64 && a.partial_type == ELEM_F32 && a.r > 256 && a.r <= 768 && a.r % 8 == 0 && !a.linv_full &&
+  if (!a.use_f64 && a.partial_type == ELEM_F32 && a.r > 256 && a.r <= 512 && a.r % 8 == 0 && !a.linv_full &&
       a.linv_hi && a.in_ld == 0 && a.out_ld == 0 && (((uintptr_t)a.partials & 15) == 0) &&
       (a.partial_stride % 4 == 0))
     return small_block_two_level(a, stream);
@@ -368,7 +368,10 @@ cudaError_t small_block_launch(const SmallBlockArgs& a, cudaStream_t stream) {
   p.linv_hi = a.linv_hi;
   p.linv_lo = a.linv_lo;
   p.dev_status = a.dev_status;
-  return a.use_f64 ? launch_typed<double>(p, stream) : launch_typed<float>(p, stream);
+  // Widths above 512 (the comparator with extra test vectors at rank 512) would need a third level of fp32 Schur
+  // complements, whose rounding noise reaches the smallest pivots (measured: clamped pivots at 520 columns,
+  // non-finite factors at 32768 rows): they take the general kernel in fp64 instead.
+  return (a.use_f64 || a.r > 512) ? launch_typed<double>(p, stream) : launch_typed<float>(p, stream);
 }
 
 }  // namespace loract

@@ -23,10 +23,13 @@ def tol_projection(err_oracle: float, dtype_key: str) -> float:
     preconditioned test matrix to the storage type and keeps the sketch to 16 bits, which tilts only the
     trailing directions of range(Y), those whose singular values are at the level of the projection error
     itself; tilting a direction of weight s by an angle t moves the projection by s * t, so this part scales
-    with the error level.  The bar is 2^-8 + err / 4 for bf16 and 2e-5 + err / 100 for fp32."""
+    with the error level.  Measured on all five configurations, the sixteen sweep points and the reduced shapes:
+    1.6e-3 to 3.2e-3 for bf16 whatever the error level (0.002 to 0.84), i.e. the storage rounding alone (the
+    largest values at 64 to 400 rows), and 5e-7 for fp32.  The bar is 2^-8 + err / 100 for bf16 and
+    5e-6 + err / 100 for fp32."""
     if dtype_key == "bf16":
-        return 2.0 ** -8 + 0.25 * err_oracle
-    return 2e-5 + 0.01 * err_oracle
+        return 2.0 ** -8 + 0.01 * err_oracle
+    return 5e-6 + 0.01 * err_oracle
 
 
 def to64(t: torch.Tensor) -> np.ndarray:
@@ -95,6 +98,8 @@ def check_compress(X, rank, seed, call_id=0, G=None, dtype_key="bf16", ws=None, 
     res = {"U": U, "V": V, "idx": idx, "err": e_gpu, "ref": ref, "orth": d, "ws": ws}
     if full_rank:
         res["proj"] = projection_distance(X64, U, V, ref["U"], ref["V"])
+        print(f"[parity] {tuple(X.shape)} r={rank} {dtype_key}: err gpu {e_gpu:.5f} oracle {ref['err']:.5f} "
+              f"projection distance {res['proj']:.2e} (bar {tol_projection(ref['err'], dtype_key):.2e})")
         assert res["proj"] <= tol_projection(ref["err"], dtype_key), (res["proj"], ref["err"])
     if G is not None:
         dW = B.weight_grad(U, V, G)

@@ -90,7 +90,7 @@ def test_row_stride_larger_than_d_and_determinism(dev):
 def test_all_rows_sampled_is_exact_up_to_storage_rounding(dev):
     w = synth.scaled(synth.WORKLOADS["llama7b_block"], n_tokens=64, d=512, rank=64, signal_rank=128)
     X = synth.make_inputs(w, device=dev)["X"]
-    res = check_compress(X, 64, seed=1)
+    res = check_compress(X, 64, seed=1, full_rank=False)     # r = N: the projection is the identity
     assert sorted(res["idx"].cpu().tolist()) == list(range(64))
     assert res["err"] <= 6e-3      # only the bf16 rounding of U and V is left
 
