@@ -214,6 +214,9 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="loract", choices=["loract", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
+                    help="repeat the block of --steps steps until the timed region has run this long (0: one block; "
+                         "for runs under a profiler)")
     ap.add_argument("--plumbing-only", action="store_true",
                     help="rank start-up, barriers and the max over ranks only, on a gloo group, no GPU work")
     ap.add_argument("--kernel-only", nargs="?", const="pass1", default=None,
@@ -319,14 +322,14 @@ def main():
     launches0 = B.kernel_launch_count()
     torch.cuda.synchronize()
     # The timed region: blocks of exactly `steps` steps, each step between its own pair of events, repeated
-    # until the region has run for MIN_TIMED_SECONDS, so that the clock record has samples under load.
+    # until the region has run for --min-seconds (default 1 s), so that the clock record has samples under load.
     times = []
     repeats = 0
     t_wall = time.perf_counter()
     while True:
         times += timed(lambda i: step(Xs[i % n_copies], Gs[i % n_copies]), args.steps)
         repeats += 1
-        enough = time.perf_counter() - t_wall >= MIN_TIMED_SECONDS or repeats >= 4000
+        enough = time.perf_counter() - t_wall >= args.min_seconds or repeats >= 4000
         if dist is not None:   # every rank runs the same number of blocks: rank 0 decides
             flag = torch.tensor([1 if enough else 0], device=dev)
             dist.broadcast(flag, 0)
