@@ -69,7 +69,12 @@ typedef struct {
 } loract_desc_t;
 
 /* Bytes of scratch that loract_compress / loract_compress_prenorm / loract_weight_grad need for this
- * descriptor (the maximum over the three).  Returns 0 if the descriptor is invalid. */
+ * descriptor (the maximum over the three).  Returns 0 if the descriptor is invalid.
+ * Size: the sketch and the once-orthonormalised basis as bf16 pairs (8 * n_tokens * rank bytes), the split-K
+ * partial sums of V and of the Gram matrices, the sampled rows and the test matrix (4 * rank * d bytes), and,
+ * for loract_compress_prenorm without A_out, the normalised input itself.  At n_tokens = 16384, d = 4096,
+ * rank = 256 in bf16 that is about 90 MB, 0.67 of X; it is transient (nothing in it is read after the call
+ * returns its results) and can be shared by every layer's call that does not overlap another on the GPU. */
 size_t loract_workspace_bytes(const loract_desc_t* desc);
 
 /* Algorithm 1, line 1: the `rank` distinct row indices, uniform without replacement.  The sample is the
