@@ -86,7 +86,7 @@ struct BasisWs {
   float* v_partials;
   void* sb_scratch;
   // fp32 path
-  float *Linv32, *Y32, *Q32;
+  float *Linv32, *Y32, *Q32, *part32;
   double* gram64;
   int splits_gram_sample, splits_gram, splits_v;
 };
@@ -98,6 +98,11 @@ struct Plan {
   int splits_gs, splits_w, splits_v;
 };
 
+inline int simt_splits(int64_t k) {
+  int64_t s = k / 128;
+  return s < 1 ? 1 : (s > 8 ? 8 : (int)s);
+}
+
 Plan make_plan(int64_t n, int64_t d, int l, bool bf16) {
   Plan p;
   p.n = n; p.d = d; p.l = l; p.bf16 = bf16;
@@ -106,7 +111,11 @@ Plan make_plan(int64_t n, int64_t d, int l, bool bf16) {
     p.splits_w = gemm_tc_pick_splits(l, l, (int)n, true, true);
     p.splits_v = gemm_tc_pick_splits(l, (int)d, (int)n, true, true);
   } else {
-    p.splits_gs = p.splits_w = p.splits_v = 1;
+    // CUDA-core path: the generic kernel walks K sixteen elements at a time, so a long contraction with few output
+    // tiles is split over K (partial sums, added in a fixed order afterwards)
+    p.splits_gs = simt_splits(d);
+    p.splits_w = simt_splits(n);
+    p.splits_v = simt_splits(n);
   }
   return p;
 }
@@ -134,9 +143,13 @@ void carve_basis(Carver& c, const Plan& p, BasisWs* w) {
   } else {
     w->Linv32 = (float*)c.take(l * l * 4);
     w->sb_scratch = c.take((l * l + (l + 31) / 32 * 1024) * sizeof(double));
-    w->gram64 = (double*)c.take(l * l * 8);
+    const size_t gs = (size_t)(p.splits_gs > p.splits_w ? p.splits_gs : p.splits_w);
+    w->gram64 = (double*)c.take(gs * l * l * 8);
     w->Y32 = (float*)c.take(n * l * 4);
     w->Q32 = (float*)c.take(n * l * 4);
+    // partial sums of pass 1 (n x l per split over d) and of pass 2 (l x d per split over the tokens)
+    const size_t p1 = (size_t)simt_splits((int64_t)d) * n * l, p2 = (size_t)p.splits_v * l * d;
+    w->part32 = (float*)c.take((p1 > p2 ? p1 : p2) * 4);
   }
 }
 
@@ -158,8 +171,18 @@ cudaError_t gram_rows(const void* S, int l, int64_t d, bool bf16, const BasisWs&
     g.split_stride = (int64_t)l * l;
   } else {
     g.out = OUT_F64; g.C0 = w.gram64; g.acc64 = true;
+    g.splits = w.splits_gram_sample; g.split_stride = (int64_t)l * l;
   }
   return run_gemm(g, status, stream);
+}
+
+// fp32 contraction on the CUDA-core kernel, split over K into `splits` partial sums that are then added in a
+// fixed order into `out` (M x N, leading dimension N).
+cudaError_t simt_split_f32(GemmDesc g, int splits, float* partials, float* out, cudaStream_t stream) {
+  if (splits <= 1) { g.out = OUT_F32; g.C0 = out; return gemm_simt_launch(g, stream); }
+  g.out = OUT_F32; g.C0 = partials; g.splits = splits; g.split_stride = (int64_t)g.M * g.ldc;
+  LORACT_CUDA_TRY(gemm_simt_launch(g, stream));
+  return reduce_partials_launch(partials, splits, g.split_stride, g.split_stride, out, nullptr, stream);
 }
 
 constexpr int kReduceFirst = 8;    // partial count from which a separate, all-SM reduction pays
@@ -183,7 +206,7 @@ cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs&
     a.use_f64 = false; a.shift_rel = shift;
     a.linv_hi = w.Lh; a.linv_lo = w.Ll;
   } else {
-    a.partials = w.gram64; a.partial_type = ELEM_F64; a.n_partials = 1; a.partial_stride = 0;
+    a.partials = w.gram64; a.partial_type = ELEM_F64; a.n_partials = n_partials; a.partial_stride = (int64_t)l * l;
     a.use_f64 = true; a.shift_rel = shift * 1e-8f;
     a.linv_f32 = w.Linv32;
   }
@@ -223,9 +246,13 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
     g.M = n; g.N = l; g.K = (int)p.d; g.lda = ldx; g.ldb = p.d; g.a_type = g.b_type = el;
     g.terms[0] = {X, Omega};
     g.ldc = l;
-    if (p.bf16) { g.out = OUT_SPLIT; g.C0 = w.Yh; g.C1 = w.Yl; } else { g.out = OUT_F32; g.C0 = w.Y32; }
     trace_label("pass 1: Y = X Omega^T");
-    LORACT_CUDA_TRY(run_gemm(g, status, stream));
+    if (p.bf16) {
+      g.out = OUT_SPLIT; g.C0 = w.Yh; g.C1 = w.Yl;
+      LORACT_CUDA_TRY(run_gemm(g, status, stream));
+    } else {
+      LORACT_CUDA_TRY(simt_split_f32(g, simt_splits(p.d), w.part32, w.Y32, stream));
+    }
   }
   for (int round = 0; round < 2; ++round) {
     const void* Yh = p.bf16 ? (const void*)(round ? w.Qh : w.Yh) : (const void*)(round ? w.Q32 : w.Y32);
@@ -242,6 +269,7 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
       } else {
         g.terms[0] = {Yh, Yh};
         g.out = OUT_F64; g.C0 = w.gram64; g.acc64 = true;
+        g.splits = w.splits_gram; g.split_stride = (int64_t)l * l;
       }
       trace_label(round ? "Gram 2" : "Gram 1");
       LORACT_CUDA_TRY(run_gemm(g, status, stream));
@@ -276,7 +304,7 @@ cudaError_t project(const void* U, const void* X, int64_t ldx, const Plan& p, vo
   g.terms[0] = {U, X};
   g.ldc = p.d;
   trace_label("pass 2: V = U^T X");
-  if (!p.bf16) { g.out = OUT_F32; g.C0 = V; return run_gemm(g, status, stream); }
+  if (!p.bf16) return simt_split_f32(g, w.splits_v, w.part32, (float*)V, stream);
   if (w.splits_v <= 1) { g.out = OUT_BF16; g.C0 = V; return run_gemm(g, status, stream); }
   g.out = OUT_F32; g.C0 = w.v_partials; g.splits = w.splits_v; g.split_stride = (int64_t)p.l * p.d;
   LORACT_CUDA_TRY(run_gemm(g, status, stream));
@@ -349,7 +377,7 @@ size_t carve_wgrad(void* ws, const loract_desc_t* desc, int g, WgradWs* out) {
   c.take(256);
   WgradWs w;
   w.splits = desc->dtype == LORACT_BF16 ? gemm_tc_pick_splits(desc->rank, g, (int)desc->n_tokens, true, true)
-                                        : (desc->n_tokens >= 4096 ? 16 : 1);
+                                        : 2 * simt_splits(desc->n_tokens);
   w.partials = (float*)c.take((size_t)w.splits * desc->rank * g * 4);
   w.T = (float*)c.take((size_t)desc->rank * g * 4);
   w.g8 = (g + 7) / 8 * 8;

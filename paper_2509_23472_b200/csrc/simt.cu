@@ -49,25 +49,41 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(SimtParams p) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = (TAcc)0;
 
+  // Each thread loads 4 elements of each operand tile; the faster-varying thread index follows the contiguous
+  // dimension of the stored operand.  The next tile is fetched into registers before the current one is
+  // multiplied, so the global-memory latency of a tile hides behind the arithmetic of its predecessor.
   for (int term = 0; term < p.n_terms; ++term) {
     const TA* A = (const TA*)p.A[term];
     const TB* B = (const TB*)p.B[term];
-    for (int k0 = k_begin; k0 < k_end; k0 += kTileK) {
-      // each thread loads 4 elements of each tile; the faster-varying thread index follows the
-      // contiguous dimension of the stored operand
-      for (int e = tid; e < kTile * kTileK; e += 256) {
+    float ra[4], rb[4];
+    auto fetch = [&](int k0) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int e = tid + 256 * u;
         int mm, kk;
         if (p.sak == 1) { kk = e % kTileK; mm = e / kTileK; } else { mm = e % kTile; kk = e / kTile; }
         const int m = m0 + mm, k = k0 + kk;
-        As[kk][mm] = (m < p.M && k < k_end) ? load_as_float(A + m * p.sam + k * p.sak) : 0.f;
+        ra[u] = (m < p.M && k < k_end) ? load_as_float(A + m * p.sam + k * p.sak) : 0.f;
+        int nn, kb;
+        if (p.sbk == 1) { kb = e % kTileK; nn = e / kTileK; } else { nn = e % kTile; kb = e / kTile; }
+        const int n = n0 + nn, k2 = k0 + kb;
+        rb[u] = (n < p.N && k2 < k_end) ? load_as_float(B + k2 * p.sbk + n * p.sbn) : 0.f;
       }
-      for (int e = tid; e < kTile * kTileK; e += 256) {
-        int nn, kk;
-        if (p.sbk == 1) { kk = e % kTileK; nn = e / kTileK; } else { nn = e % kTile; kk = e / kTile; }
-        const int n = n0 + nn, k = k0 + kk;
-        Bs[kk][nn] = (n < p.N && k < k_end) ? load_as_float(B + k * p.sbk + n * p.sbn) : 0.f;
+    };
+    if (k_begin < k_end) fetch(k_begin);
+    for (int k0 = k_begin; k0 < k_end; k0 += kTileK) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int e = tid + 256 * u;
+        int mm, kk;
+        if (p.sak == 1) { kk = e % kTileK; mm = e / kTileK; } else { mm = e % kTile; kk = e / kTile; }
+        As[kk][mm] = ra[u];
+        int nn, kb;
+        if (p.sbk == 1) { kb = e % kTileK; nn = e / kTileK; } else { nn = e % kTile; kb = e / kTile; }
+        Bs[kb][nn] = rb[u];
       }
       __syncthreads();
+      if (k0 + kTileK < k_end) fetch(k0 + kTileK);
 #pragma unroll
       for (int kk = 0; kk < kTileK; ++kk) {
         float a[4], b[4];
