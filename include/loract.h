@@ -143,6 +143,38 @@ loract_status_t loract_prenorm_backward(const loract_desc_t* desc, const void* U
 loract_status_t loract_activation_backward(const loract_desc_t* desc, const void* U, const void* V,
                                            const void* grad_Z, int32_t kind, void* grad_X, void* stream);
 
+/* Algorithm 1 (t = 0) on ONE matrix X whose token rows are sharded over several GPUs (sequence or context
+ * parallelism), as one joint factorisation: the same U V = P_Y X as loract_compress on the whole X.  Every shard
+ * runs the stages below on its own rows [row0, row0 + n_tokens) (desc->n_tokens is the shard's row count, desc->
+ * seed / call_id are the same on every shard); between stages the caller adds the small matrices over all shards
+ * (an all-reduce with NCCL; what arrives lands in local memory before the next stage reads it) -- the library
+ * itself does no communication.  bf16 only; every shard needs at least `rank` rows.
+ *   1. loract_joint_sample_rows : line 1.  The `rank` sampled rows of the whole matrix (indices in [0, n_global),
+ *      the same on every shard); S (rank x d) receives those that live on this shard, zeros elsewhere.
+ *      -> add S over the shards (one non-zero contribution per row: exact).
+ *   2. loract_joint_sketch      : line 2.  Y_local = X_local Omega^T with the test matrix Omega made from S_sum (the
+ *      same bits on every shard), and W_partial (rank x rank fp32) = Y_local^T Y_local.  -> add W_partial.
+ *   3. loract_joint_orthonormalise, round 0 : line 7, first half.  Y_local <- Y_local L^-T with L L^T = W_sum;
+ *      W_next_partial = the new Y_local^T Y_local.  -> add W_next_partial.
+ *      round 1 : second half.  U_local (n_tokens x rank) = Y_local L^-T with the factor of the second sum.
+ *   4. loract_joint_project     : line 8.  V_partial (rank x d fp32) = U_local^T X_local.  -> add V_partial.
+ *   5. loract_joint_finish      : V (rank x d, bf16) = V_sum rounded once.
+ * The sketch and the once-orthonormalised sketch stay in `ws` between the stages: the same `ws` (at least
+ * loract_joint_workspace_bytes(desc) bytes) must be passed to stages 1 to 4 of one factorisation.  The device
+ * status word at the start of `ws` is cleared by stage 1 and collects every later stage's conditions. */
+size_t loract_joint_workspace_bytes(const loract_desc_t* desc);
+loract_status_t loract_joint_sample_rows(const loract_desc_t* desc, int64_t n_global, int64_t row0,
+                                         const void* X_local, void* S, int32_t* idx_out, void* ws, size_t ws_bytes,
+                                         void* stream);
+loract_status_t loract_joint_sketch(const loract_desc_t* desc, const void* X_local, const void* S_sum,
+                                    float* W_partial, void* ws, size_t ws_bytes, void* stream);
+loract_status_t loract_joint_orthonormalise(const loract_desc_t* desc, int32_t round, const float* W_sum,
+                                            float* W_next_partial, void* U_local, void* ws, size_t ws_bytes,
+                                            void* stream);
+loract_status_t loract_joint_project(const loract_desc_t* desc, const void* U_local, const void* X_local,
+                                     float* V_partial, void* ws, size_t ws_bytes, void* stream);
+loract_status_t loract_joint_finish(const loract_desc_t* desc, const float* V_sum, void* V, void* stream);
+
 /* The same result as loract_weight_grad, for callers that cannot allocate device memory and so cannot
  * provide `ws`.  (The paper has no counterpart: this is a property of the library, not of the method.)
  * Typical callers: a backward hook running while the framework's caching allocator is locked or out of

@@ -22,7 +22,9 @@ DEV_PIVOT_CLAMPED, DEV_WAIT_EXPIRED, DEV_SAMPLER_SHORT, DEV_NONFINITE = 1, 2, 4,
 EXPORTS = (
     "loract_workspace_bytes", "loract_sample_indices", "loract_compress", "loract_reconstruct",
     "loract_weight_grad", "loract_weight_grad_static", "loract_weight_grad_static_status", "loract_compress_prenorm",
-    "loract_prenorm_backward_workspace_bytes", "loract_prenorm_backward", "loract_activation_backward", "loract_rsvd_workspace_bytes", "loract_rsvd",
+    "loract_prenorm_backward_workspace_bytes", "loract_prenorm_backward", "loract_activation_backward",
+    "loract_joint_workspace_bytes", "loract_joint_sample_rows", "loract_joint_sketch", "loract_joint_orthonormalise",
+    "loract_joint_project", "loract_joint_finish", "loract_rsvd_workspace_bytes", "loract_rsvd",
     "loract_read_device_status", "loract_status_from_device_word", "loract_status_string",
     "loract_kernel_launch_count",
 )
@@ -81,6 +83,18 @@ def lib() -> ctypes.CDLL:
         l.loract_prenorm_backward.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         l.loract_activation_backward.restype = ctypes.c_int
         l.loract_activation_backward.argtypes = [dp, vp, vp, vp, i32, vp, vp]
+        l.loract_joint_workspace_bytes.restype = sz
+        l.loract_joint_workspace_bytes.argtypes = [dp]
+        l.loract_joint_sample_rows.restype = ctypes.c_int
+        l.loract_joint_sample_rows.argtypes = [dp, i64, i64, vp, vp, vp, vp, sz, vp]
+        l.loract_joint_sketch.restype = ctypes.c_int
+        l.loract_joint_sketch.argtypes = [dp, vp, vp, vp, vp, sz, vp]
+        l.loract_joint_orthonormalise.restype = ctypes.c_int
+        l.loract_joint_orthonormalise.argtypes = [dp, i32, vp, vp, vp, vp, sz, vp]
+        l.loract_joint_project.restype = ctypes.c_int
+        l.loract_joint_project.argtypes = [dp, vp, vp, vp, vp, sz, vp]
+        l.loract_joint_finish.restype = ctypes.c_int
+        l.loract_joint_finish.argtypes = [dp, vp, vp, vp]
         l.loract_rsvd_workspace_bytes.restype = sz
         l.loract_rsvd_workspace_bytes.argtypes = [dp, i32]
         l.loract_rsvd.restype = ctypes.c_int

@@ -388,6 +388,71 @@ size_t carve_wgrad(void* ws, const loract_desc_t* desc, int g, WgradWs* out) {
   return c.off;
 }
 
+// ------------------------------------------------------------------ joint compression of a token-sharded X
+// Every shard runs the same stages on its rows; between stages the caller adds the small matrices the stages
+// hand out over all shards (the sampled rows, the r x r Gram matrices, V).  State between stages (the test matrix,
+// the sketch, the once-orthonormalised sketch, L^-1) stays in the shard's workspace.
+struct JointWs {
+  uint32_t* status;
+  int32_t* idx;
+  void* Omega;
+  BasisWs b;
+};
+
+size_t carve_joint(void* ws, const loract_desc_t* desc, JointWs* out, Plan* plan) {
+  *plan = make_plan(desc->n_tokens, desc->d, desc->rank, true);
+  Carver c(ws);
+  JointWs w;
+  w.status = (uint32_t*)c.take(256);
+  w.idx = (int32_t*)c.take((size_t)desc->rank * 4);
+  w.Omega = c.take((size_t)desc->rank * desc->d * 2);
+  carve_basis(c, *plan, &w.b);
+  if (out) *out = w;
+  return c.off;
+}
+
+// W (l x l fp32, summed over this shard's split-K partials) = Y^T Y for a tall bf16 pair Y = Yh + Yl (n x l).
+cudaError_t gram_tall_sum(const void* Yh, const void* Yl, int n, int l, const BasisWs& w, float* W, uint32_t* status,
+                          cudaStream_t stream) {
+  GemmDesc g;
+  g.M = l; g.N = l; g.K = n; g.a_mn = true; g.b_mn = true; g.lda = l; g.ldb = l;
+  g.n_terms = 3;
+  g.terms[0] = {Yh, Yh}; g.terms[1] = {Yh, Yl}; g.terms[2] = {Yl, Yh};
+  g.out = OUT_F32; g.ldc = l;
+  if (w.splits_gram <= 1) { g.C0 = W; return run_gemm(g, status, stream); }
+  g.C0 = w.gram_partials; g.splits = w.splits_gram; g.split_stride = (int64_t)l * l;
+  LORACT_CUDA_TRY(run_gemm(g, status, stream));
+  return reduce_partials_launch(w.gram_partials, w.splits_gram, g.split_stride, g.split_stride, W, nullptr, stream);
+}
+
+// L^-1 (bf16 pair in w.Lh / w.Ll) from one summed l x l Gram matrix.
+cudaError_t factor_matrix(const float* W, int l, float shift, const BasisWs& w, uint32_t* status, cudaStream_t stream) {
+  SmallBlockArgs a;
+  a.r = l; a.scratch = w.sb_scratch; a.dev_status = status;
+  a.partials = W; a.partial_type = ELEM_F32; a.n_partials = 1; a.partial_stride = (int64_t)l * l;
+  a.use_f64 = false; a.shift_rel = shift;
+  a.linv_hi = w.Lh; a.linv_lo = w.Ll;
+  return small_block_launch(a, stream);
+}
+
+// C = Y L^-T for a tall bf16 pair Y (n x l): as a bf16 pair (Ch, Cl) or, with Cl == nullptr, rounded once to bf16.
+cudaError_t apply_linv(const void* Yh, const void* Yl, int n, int l, const BasisWs& w, void* Ch, void* Cl,
+                       uint32_t* status, cudaStream_t stream) {
+  GemmDesc g;
+  g.M = n; g.N = l; g.K = l; g.lda = l; g.ldb = l; g.ldc = l;
+  g.n_terms = 3;
+  g.terms[0] = {Yh, w.Lh}; g.terms[1] = {Yh, w.Ll}; g.terms[2] = {Yl, w.Lh};
+  if (Cl) { g.out = OUT_SPLIT; g.C0 = Ch; g.C1 = Cl; } else { g.out = OUT_BF16; g.C0 = Ch; }
+  return run_gemm(g, status, stream);
+}
+
+loract_status_t check_joint(const loract_desc_t* desc) {
+  loract_status_t s = check_desc(desc);
+  if (s != LORACT_OK) return s;
+  if (desc->dtype != LORACT_BF16 || desc->power_iters != 0) return LORACT_ERR_UNSUPPORTED;
+  return LORACT_OK;
+}
+
 std::atomic<int> g_last_cuda_error{0};
 loract_status_t from_cuda(cudaError_t e) {
   if (e == cudaSuccess) return LORACT_OK;
@@ -601,6 +666,122 @@ loract_status_t loract_activation_backward(const loract_desc_t* desc, const void
   trace_label("activation backward: grad_X");
   if (!gemm_tc_supported(g)) return LORACT_ERR_UNSUPPORTED;
   return from_cuda(gemm_tc_launch(g, nullptr, (cudaStream_t)stream));
+}
+
+size_t loract_joint_workspace_bytes(const loract_desc_t* desc) {
+  if (check_joint(desc) != LORACT_OK) return 0;
+  Plan plan;
+  return carve_joint(nullptr, desc, nullptr, &plan);
+}
+
+loract_status_t loract_joint_sample_rows(const loract_desc_t* desc, int64_t n_global, int64_t row0, const void* X_local,
+                                         void* S, int32_t* idx_out, void* ws, size_t ws_bytes, void* stream) {
+  loract_status_t s = check_joint(desc);
+  if (s != LORACT_OK) return s;
+  if (!X_local || !S || !ws) return LORACT_ERR_INVALID_ARG;
+  if (n_global < desc->n_tokens || n_global > 0x7fffffffLL || row0 < 0 || row0 + desc->n_tokens > n_global ||
+      desc->rank > n_global)
+    return LORACT_ERR_INVALID_ARG;
+  if (misaligned(X_local) || misaligned(S) || ((uintptr_t)ws & 255)) return LORACT_ERR_ALIGNMENT;
+  JointWs w;
+  Plan plan;
+  if (ws_bytes < carve_joint(ws, desc, &w, &plan)) return LORACT_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  trace_label("joint: sample");
+  cudaError_t e = sample_indices_launch(desc->seed, desc->call_id, (uint32_t)n_global, desc->rank, w.idx, w.status, st,
+                                        idx_out, true);
+  trace_label("joint: gather own rows");
+  if (e == cudaSuccess)
+    e = gather_rows_window_launch(X_local, desc->ldx, w.idx, desc->rank, desc->d, 2, row0, desc->n_tokens, S, st);
+  return from_cuda(e);
+}
+
+loract_status_t loract_joint_sketch(const loract_desc_t* desc, const void* X_local, const void* S_sum, float* W_partial,
+                                    void* ws, size_t ws_bytes, void* stream) {
+  loract_status_t s = check_joint(desc);
+  if (s != LORACT_OK) return s;
+  if (!X_local || !S_sum || !W_partial || !ws) return LORACT_ERR_INVALID_ARG;
+  if (misaligned(X_local) || misaligned(S_sum) || misaligned(W_partial) || ((uintptr_t)ws & 255))
+    return LORACT_ERR_ALIGNMENT;
+  JointWs w;
+  Plan plan;
+  if (ws_bytes < carve_joint(ws, desc, &w, &plan)) return LORACT_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int r = desc->rank, n = (int)desc->n_tokens;
+  // the test matrix from the complete sampled rows: the same bits on every shard
+  cudaError_t e = precondition_rows(S_sum, r, desc->d, true, w.Omega, w.b, w.status, st);
+  if (e == cudaSuccess) {  // this shard's rows of the sketch, Y = X_local Omega^T
+    GemmDesc g;
+    g.M = n; g.N = r; g.K = (int)desc->d; g.lda = desc->ldx; g.ldb = desc->d;
+    g.terms[0] = {X_local, w.Omega};
+    g.ldc = r; g.out = OUT_SPLIT; g.C0 = w.b.Yh; g.C1 = w.b.Yl;
+    trace_label("joint: pass 1");
+    e = run_gemm(g, w.status, st);
+  }
+  trace_label("joint: Gram 1 of the shard");
+  if (e == cudaSuccess) e = gram_tall_sum(w.b.Yh, w.b.Yl, n, r, w.b, W_partial, w.status, st);
+  return from_cuda(e);
+}
+
+loract_status_t loract_joint_orthonormalise(const loract_desc_t* desc, int32_t round, const float* W_sum,
+                                            float* W_next_partial, void* U_local, void* ws, size_t ws_bytes,
+                                            void* stream) {
+  loract_status_t s = check_joint(desc);
+  if (s != LORACT_OK) return s;
+  if (round != 0 && round != 1) return LORACT_ERR_INVALID_ARG;
+  if (!W_sum || !ws || (round == 0 && !W_next_partial) || (round == 1 && !U_local)) return LORACT_ERR_INVALID_ARG;
+  if (misaligned(W_sum) || (round == 0 && misaligned(W_next_partial)) || (round == 1 && misaligned(U_local)) ||
+      ((uintptr_t)ws & 255))
+    return LORACT_ERR_ALIGNMENT;
+  JointWs w;
+  Plan plan;
+  if (ws_bytes < carve_joint(ws, desc, &w, &plan)) return LORACT_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int r = desc->rank, n = (int)desc->n_tokens;
+  trace_label(round ? "joint: small block 3" : "joint: small block 2");
+  cudaError_t e = factor_matrix(W_sum, r, round ? kShiftSecond : kShiftFirst, w.b, w.status, st);
+  trace_label(round ? "joint: apply L^-T 2" : "joint: apply L^-T 1");
+  if (round == 0) {
+    if (e == cudaSuccess) e = apply_linv(w.b.Yh, w.b.Yl, n, r, w.b, w.b.Qh, w.b.Ql, w.status, st);
+    trace_label("joint: Gram 2 of the shard");
+    if (e == cudaSuccess) e = gram_tall_sum(w.b.Qh, w.b.Ql, n, r, w.b, W_next_partial, w.status, st);
+  } else {
+    if (e == cudaSuccess) e = apply_linv(w.b.Qh, w.b.Ql, n, r, w.b, U_local, nullptr, w.status, st);
+  }
+  return from_cuda(e);
+}
+
+loract_status_t loract_joint_project(const loract_desc_t* desc, const void* U_local, const void* X_local,
+                                     float* V_partial, void* ws, size_t ws_bytes, void* stream) {
+  loract_status_t s = check_joint(desc);
+  if (s != LORACT_OK) return s;
+  if (!U_local || !X_local || !V_partial || !ws) return LORACT_ERR_INVALID_ARG;
+  if (misaligned(U_local) || misaligned(X_local) || misaligned(V_partial) || ((uintptr_t)ws & 255))
+    return LORACT_ERR_ALIGNMENT;
+  JointWs w;
+  Plan plan;
+  if (ws_bytes < carve_joint(ws, desc, &w, &plan)) return LORACT_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  GemmDesc g;
+  g.M = plan.l; g.N = (int)plan.d; g.K = (int)plan.n; g.a_mn = true; g.b_mn = true; g.lda = plan.l; g.ldb = desc->ldx;
+  g.terms[0] = {U_local, X_local};
+  g.ldc = plan.d; g.out = OUT_F32;
+  trace_label("joint: pass 2 of the shard");
+  if (w.b.splits_v <= 1) { g.C0 = V_partial; return from_cuda(run_gemm(g, w.status, st)); }
+  g.C0 = w.b.v_partials; g.splits = w.b.splits_v; g.split_stride = (int64_t)plan.l * plan.d;
+  cudaError_t e = run_gemm(g, w.status, st);
+  if (e == cudaSuccess)
+    e = reduce_partials_launch(w.b.v_partials, w.b.splits_v, g.split_stride, g.split_stride, V_partial, nullptr, st);
+  return from_cuda(e);
+}
+
+loract_status_t loract_joint_finish(const loract_desc_t* desc, const float* V_sum, void* V, void* stream) {
+  loract_status_t s = check_joint(desc);
+  if (s != LORACT_OK) return s;
+  if (!V_sum || !V) return LORACT_ERR_INVALID_ARG;
+  if (misaligned(V_sum) || misaligned(V)) return LORACT_ERR_ALIGNMENT;
+  const int64_t count = (int64_t)desc->rank * desc->d;
+  return from_cuda(reduce_partials_launch(V_sum, 1, 0, count, nullptr, (__nv_bfloat16*)V, (cudaStream_t)stream));
 }
 
 size_t loract_rsvd_workspace_bytes(const loract_desc_t* desc, int32_t oversample) {

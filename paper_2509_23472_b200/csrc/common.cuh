@@ -127,6 +127,10 @@ cudaError_t sample_indices_launch(uint64_t seed, uint64_t call_id, uint32_t n_ro
 // dst (rank x d, stride d) = src[idx, :] (stride ld); 16-byte loads.  elem_bytes 2 or 4.
 cudaError_t gather_rows_launch(const void* src, int64_t ld, const int32_t* idx, int rank, int64_t d,
                                int elem_bytes, void* dst, cudaStream_t stream);
+// The same for one shard of a token-sharded matrix (src = rows [row0, row0 + n_local) of the whole matrix, idx in
+// whole-matrix row numbers): rows that live on another shard are written as zeros.
+cudaError_t gather_rows_window_launch(const void* src, int64_t ld, const int32_t* idx, int rank, int64_t d,
+                                      int elem_bytes, int64_t row0, int64_t n_local, void* dst, cudaStream_t stream);
 // Gaussian test matrix for the RSVD comparator: dst (l x d bf16, row-major) with
 // dst[c][j] = z(j * l + c), z the Philox + Box-Muller stream (counter word 1 = 1).
 cudaError_t gaussian_rows_launch(uint64_t seed, uint64_t call_id, int l, int64_t d,

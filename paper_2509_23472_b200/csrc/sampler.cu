@@ -108,6 +108,22 @@ __global__ void gather_rows_kernel(const uint4* __restrict__ src, int64_t ld_vec
     dst[(int64_t)row * d_vec + v] = __ldg(src + srow * ld_vec + v);
 }
 
+// The same for one shard of a token-sharded matrix: `src` holds the rows [row0, row0 + n_local) of the whole
+// matrix, idx are row numbers of the whole matrix; a sampled row that lives on another shard is written as
+// zeros, so that the sum of all shards' results is the gathered matrix.
+__global__ void gather_rows_window_kernel(const uint4* __restrict__ src, int64_t ld_vec,
+                                          const int32_t* __restrict__ idx, int64_t d_vec, int64_t row0,
+                                          int64_t n_local, uint4* __restrict__ dst) {
+  const int row = blockIdx.y;
+  pdl_wait();
+  pdl_launch_dependents();
+  const int64_t srow = (int64_t)idx[row] - row0;
+  const bool mine = srow >= 0 && srow < n_local;
+  for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < d_vec;
+       v += (int64_t)gridDim.x * blockDim.x)
+    dst[(int64_t)row * d_vec + v] = mine ? __ldg(src + srow * ld_vec + v) : make_uint4(0u, 0u, 0u, 0u);
+}
+
 // dst[c][j] = z(j * l + c): element e of the normal stream is z_(e mod 4) of Philox block e div 4,
 // u = (w0 + 1) / 2^32, v = w1 / 2^32, z0 = sqrt(-2 ln u) cos(2 pi v), z1 = ... sin(2 pi v).
 __global__ void gaussian_rows_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_t call_lo,
@@ -161,6 +177,19 @@ cudaError_t gather_rows_launch(const void* src, int64_t ld, const int32_t* idx, 
   if (gx > 64) gx = 64;
   LORACT_CUDA_TRY(launch_pdl(gather_rows_kernel, dim3(gx, rank), dim3(threads), 0, stream, (const uint4*)src, ld_vec,
                              idx, d_vec, (uint4*)dst));
+  count_launch(__func__, stream);
+  return cudaGetLastError();
+}
+
+cudaError_t gather_rows_window_launch(const void* src, int64_t ld, const int32_t* idx, int rank, int64_t d,
+                                      int elem_bytes, int64_t row0, int64_t n_local, void* dst, cudaStream_t stream) {
+  const int64_t per_vec = 16 / elem_bytes;
+  const int64_t d_vec = d / per_vec, ld_vec = ld / per_vec;
+  const int threads = 256;
+  int gx = (int)((d_vec + threads - 1) / threads);
+  if (gx > 64) gx = 64;
+  LORACT_CUDA_TRY(launch_pdl(gather_rows_window_kernel, dim3(gx, rank), dim3(threads), 0, stream, (const uint4*)src,
+                             ld_vec, idx, d_vec, row0, n_local, (uint4*)dst));
   count_launch(__func__, stream);
   return cudaGetLastError();
 }

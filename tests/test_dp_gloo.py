@@ -88,3 +88,61 @@ def test_bench_starts_its_own_ranks_when_run_without_a_launcher():
     assert out["ms_per_step"] == 2.0                    # the slower rank's time
     assert out["seeds"] == [base.seed, base.seed + dp.SEED_STRIDE] and out["call_ids"] == [0, 1]
     assert out["value"] == dp.whole_job_gbs(2, base.n_tokens * base.d * base.elem_bytes, 2.0)
+
+
+class _FakeShard:
+    """Stands in for joint.JointShard on a CPU process group: every stage hands out a matrix that depends on the
+    rank and records what sum it was given, so that the order of the stages and the reductions can be checked."""
+
+    def __init__(self, rank):
+        self.rank, self.seen = rank, []
+        self.U, self.idx = torch.full((2, 2), float(rank)), torch.arange(2)
+
+    def sample_rows(self):
+        return torch.full((2, 3), 1.0 + self.rank)
+
+    def sketch(self, S_sum):
+        self.seen.append(("S", S_sum.clone()))
+        return torch.full((2, 2), 10.0 * (1 + self.rank))
+
+    def orthonormalise(self, round_, W_sum):
+        self.seen.append((f"W{round_}", W_sum.clone()))
+        return torch.full((2, 2), 100.0 * (1 + self.rank)) if round_ == 0 else self.U
+
+    def project(self):
+        return torch.full((2, 3), 1000.0 * (1 + self.rank))
+
+    def finish(self, V_sum):
+        self.seen.append(("V", V_sum.clone()))
+        return V_sum
+
+
+def _joint_worker(rank: int, world: int, port: int, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        from paper_2509_23472_b200 import joint
+        shard = _FakeShard(rank)
+
+        def add(parts):
+            t = parts[0].clone()
+            dist.all_reduce(t, op=dist.ReduceOp.SUM)
+            return t
+        joint.run_stages([shard], add)
+        out[rank] = [(k, float(v.flatten()[0])) for k, v in shard.seen]
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_joint_compression_stages_reduce_the_right_matrix_at_the_right_time():
+    """The stage sequence of the token-sharded compression on two gloo ranks: each stage must be handed the SUM
+    over the ranks of what the previous stage produced, in the order rows, Gram 1, Gram 2, V."""
+    world = 2
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_joint_worker, args=(world, _free_port(), out), nprocs=world, join=True)
+        res = {k: list(v) for k, v in out.items()}
+    want = [("S", 3.0), ("W0", 30.0), ("W1", 300.0), ("V", 3000.0)]
+    assert res[0] == want and res[1] == want
