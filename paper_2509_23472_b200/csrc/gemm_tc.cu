@@ -61,6 +61,8 @@ struct TcParams {
   int tma_store;      // 1: the epilogue stages 32-row boxes in shared memory and writes them with TMA stores
   int st_m_tiles;     // streaming kernel: 256-row tiles along M
   int st_units;       // streaming kernel: tiles in all (column tile major, then M)
+  int st_stages;      // streaming kernel: stages of the A ring (<= kStreamStages)
+  int store_bufs;     // staging boxes per epilogue warp (1 or 2)
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -141,6 +143,14 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t v[32]) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tc_ld64(uint32_t taddr, uint32_t v[64]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31]), "=r"(v[32]), "=r"(v[33]), "=r"(v[34]), "=r"(v[35]), "=r"(v[36]), "=r"(v[37]), "=r"(v[38]), "=r"(v[39]), "=r"(v[40]), "=r"(v[41]), "=r"(v[42]), "=r"(v[43]), "=r"(v[44]), "=r"(v[45]), "=r"(v[46]), "=r"(v[47]), "=r"(v[48]), "=r"(v[49]), "=r"(v[50]), "=r"(v[51]), "=r"(v[52]), "=r"(v[53]), "=r"(v[54]), "=r"(v[55]), "=r"(v[56]), "=r"(v[57]), "=r"(v[58]), "=r"(v[59]), "=r"(v[60]), "=r"(v[61]), "=r"(v[62]), "=r"(v[63])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle.  K-major: rows of 128 bytes, groups of 8 rows
@@ -184,6 +194,7 @@ constexpr uint32_t kStoreWarpBytes = kStoreBufs * kStoreBoxBytes;
 struct StoreStage {
   unsigned char* base;   // this warp's boxes (1024-byte aligned); nullptr: direct stores only
   uint32_t cnt;          // boxes sent so far
+  uint32_t bufs;         // boxes this warp cycles through (1 or 2)
 };
 
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int x, int y) {
@@ -198,13 +209,16 @@ __device__ __forceinline__ void bulk_wait_read() {
 // Boxes cnt .. cnt + kNeed - 1 may be written once the stores that last used them have read shared memory.
 template <int kNeed>
 __device__ __forceinline__ void stage_acquire(const StoreStage& st, int lane) {
-  if (st.cnt + kNeed > kStoreBufs) {
-    if (lane == 0) bulk_wait_read<kStoreBufs - kNeed>();
+  if (st.cnt + kNeed > st.bufs) {
+    if (lane == 0) {
+      if (st.bufs > (uint32_t)kNeed) bulk_wait_read<kStoreBufs - kNeed>();
+      else bulk_wait_read<0>();
+    }
     __syncwarp();
   }
 }
 __device__ __forceinline__ unsigned char* stage_box(const StoreStage& st, uint32_t k) {
-  return st.base + ((st.cnt + k) % kStoreBufs) * kStoreBoxBytes;
+  return st.base + ((st.cnt + k) % st.bufs) * kStoreBoxBytes;
 }
 __device__ __forceinline__ void stage_write16(unsigned char* box, int lane, int chunk, uint4 v) {
   *reinterpret_cast<uint4*>(box + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = v;
@@ -255,11 +269,12 @@ __device__ __forceinline__ void tc_store_tile_staged(const TcParams& p, const Tm
     if (split_out) stage_acquire<2>(st, lane); else stage_acquire<1>(st, lane);
     unsigned char* box_hi = stage_box(st, 0);
     unsigned char* box_lo = stage_box(st, 1);
+    uint32_t v64[64];
+    tc_ld64(taddr + (uint32_t)c0, v64);
+    tc_wait_ld();
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
-      uint32_t v[32];
-      tc_ld32(taddr + (uint32_t)(c0 + 32 * half), v);
-      tc_wait_ld();
+      const uint32_t* v = v64 + 32 * half;
       const int n = n0 + c0 + 32 * half;
       if (rms) {
         const bool cols_ok = n + 32 <= p.N;                  // a partial group is clipped anyway; read nothing past N
@@ -469,6 +484,7 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const TmapPack& m
     StoreStage st;
     st.base = ring + (uint32_t)(warp - 2) * kStoreWarpBytes;
     st.cnt = 0;
+    st.bufs = kStoreBufs;
     tc_store_tile(p, maps, tmem_base, warp, lane, m0, n0, split, st);
     stage_drain(st, lane);
   } else if (ok && n_iter == 0 && m < p.M && p.out == OUT_F32 && warp < 6) {
@@ -762,11 +778,17 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
 //     only A is streamed through a ring of 128 x 64 stages;
 //   * the accumulator is double buffered in tensor memory (2 x bn columns): the tensor cores work on tile
 //     i + 1 while the eight epilogue warps read and store tile i.
+// Tiles are 256 columns wide whenever the output mode allows it: with 128 columns one instruction keeps the
+// tensor pipe busy for 64 cycles, less than the issuing thread needs per instruction (about 100 cycles with
+// the fence and the commit of a K block), and the kernel ran issue-bound at about 0.6 of the 256-wide rate.
+// Beyond four K blocks the resident B (16 KB per K block and CTA) leaves room for a shorter A ring and one
+// staging box per epilogue warp only; the epilogue has the slack (it is about half the tensor time there).
 // Barriers.  a_full / a_empty: the ring, as in the pair kernel.  b_full (leader): both halves of B have
 // landed; b_empty (each CTA, by commit): every MMA that reads the resident B is done, it may be replaced.
 // acc_full[j] (each CTA, by commit): buffer j holds a finished tile; acc_empty[j] (leader, one arrival
 // per CTA, sent by the first epilogue warp once all eight have arrived on the CTA's own epi_done[j]): buffer j has been read in both CTAs.  No load uses cluster multicast.
 constexpr int kStreamStages = 6;
+constexpr int kStreamSmemMax = 226 * 1024;                 // dynamic shared memory the streaming kernel may ask for
 
 // An arrival on a barrier of the peer CTA.  Relaxed: it announces that tensor-memory reads have completed
 // (tcgen05.wait::ld has returned), no memory written by this thread has to become visible with it, and a
@@ -877,8 +899,8 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
         }
         const int m0 = mt * 2 * kBM + (int)cta_rank * kBM;
         for (int kb = 0; kb < p.kb_total; ++kb, ++it) {
-          const int s = it % kStreamStages;
-          ok = mbar_wait_bounded(&a_empty[s], (uint32_t)(((it / kStreamStages) & 1) ^ 1), &abort_flag);
+          const int s = it % p.st_stages;
+          ok = mbar_wait_bounded(&a_empty[s], (uint32_t)(((it / p.st_stages) & 1) ^ 1), &abort_flag);
           if (!ok) break;
           if (leader) mbar_arrive_expect_tx(&a_full[s], 2u * kABytes);
           tma_load_2d_pair(ring + (size_t)s * kABytes, &maps.a[0], map_to_rank(smem_u32(&a_full[s]), 0u), kb * kBK, m0);
@@ -907,8 +929,8 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(j * p.bn);
         for (int kb = 0; kb < p.kb_total; ++kb, ++it) {
-          const int s = it % kStreamStages;
-          ok = mbar_wait_bounded(&a_full[s], (uint32_t)((it / kStreamStages) & 1), &abort_flag);
+          const int s = it % p.st_stages;
+          ok = mbar_wait_bounded(&a_full[s], (uint32_t)((it / p.st_stages) & 1), &abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint64_t a_desc = make_smem_desc(smem_u32(ring + (size_t)s * kABytes), false);
@@ -927,7 +949,8 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   } else {
     bool ok = true;
     StoreStage st;
-    st.base = ring + (size_t)kStreamStages * kABytes + (uint32_t)(warp - 2) * kStoreWarpBytes;
+    st.bufs = (uint32_t)p.store_bufs;
+    st.base = ring + (size_t)p.st_stages * kABytes + (uint32_t)(warp - 2) * st.bufs * kStoreBoxBytes;
     st.cnt = 0;
     for (int u = u_begin, ui = 0; u < u_end; ++u, ++ui) {
       const int j = ui & 1;
@@ -1108,7 +1131,7 @@ cudaError_t launch_stream(const TmapPack& maps, TcParams p, size_t smem, cudaStr
   const bool cached = dev >= 0 && dev < 64 && configured[dev];
   int pairs = cached ? max_pairs[dev] : 0;
   if (!cached) {
-    const int smem_max = 8 * 8192 + kStreamStages * (int)kABytes + kEpiWarps * (int)kStoreWarpBytes + 1024;
+    const int smem_max = kStreamSmemMax;
     LORACT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
     cudaLaunchConfig_t q = {};
     q.gridDim = dim3(2); q.blockDim = dim3(kThreads); q.dynamicSmemBytes = smem_max;
@@ -1204,7 +1227,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   p.ep_E = g.ep_E; p.ep_ld = g.ep_ld; p.ep_row_a = g.ep_row_a; p.ep_row_b = g.ep_row_b; p.ep_col = g.ep_col;
   p.ep_kind = g.ep_kind;
   p.dev_status = dev_status;
-  p.st_m_tiles = 0; p.st_units = 0; p.tma_store = 0;
+  p.st_m_tiles = 0; p.st_units = 0; p.tma_store = 0; p.st_stages = kStreamStages; p.store_bufs = kStoreBufs;
 
   TmapPack maps;
   for (int t = 0; t < g.n_terms; ++t) {
@@ -1241,16 +1264,27 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   if (g_pair_mode == 1 && g.M >= 2 * kBM && !g.a_mn && g.b_mn && g.n_terms == 1 && splits == 1 && p.kb_total <= 8 &&
       g.N >= 256) {
     TcParams sp = p;
-    sp.bn = p.kb_total <= 4 ? 256 : 128;
+    // 256 columns per tile (the tensor pipe is issue-bound on narrower instructions).  The resident B takes
+    // 16 KB per K block and CTA; beyond four K blocks the A ring and the staging boxes shrink to make room
+    // (one box per warp cannot serve the two-box split output, which keeps 128 columns).
+    sp.bn = (p.kb_total <= 4 || g.out != OUT_SPLIT) ? 256 : 128;
     sp.b_bytes = (uint32_t)(sp.bn / 2 / 64) * 8192u;
     sp.tmem_cols = 2u * (uint32_t)sp.bn;
+    sp.st_stages = kStreamStages;
+    sp.store_bufs = kStoreBufs;
+    if (sp.bn == 256 && p.kb_total > 4) {
+      sp.store_bufs = 1;
+      const int room = kStreamSmemMax - 1024 - p.kb_total * (int)sp.b_bytes - kEpiWarps * (int)kStoreBoxBytes;
+      sp.st_stages = std::min(kStreamStages, room / (int)kABytes);
+    }
     sp.st_m_tiles = (g.M + 2 * kBM - 1) / (2 * kBM);
     const long long units = (long long)sp.st_m_tiles * ((g.N + sp.bn - 1) / sp.bn);
     if (units >= 148 && units < (1ll << 30)) {
       sp.st_units = (int)units;
       sp.tma_store = staged_ok(sp.bn) ? 1 : 0;
       if (sp.tma_store) LORACT_CUDA_TRY(make_out_maps());
-      const size_t ssmem = (size_t)sp.kb_total * sp.b_bytes + (size_t)kStreamStages * kABytes + kEpiWarps * kStoreWarpBytes + 1024;
+      const size_t ssmem = (size_t)sp.kb_total * sp.b_bytes + (size_t)sp.st_stages * kABytes +
+                           (size_t)kEpiWarps * sp.store_bufs * kStoreBoxBytes + 1024;
       return launch_stream(maps, sp, ssmem, stream);
     }
   }

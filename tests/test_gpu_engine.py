@@ -91,7 +91,8 @@ def test_both_forms_agree_bit_for_bit_on_a_gram_product(dev):
 @pytest.mark.parametrize("M,N,K,out_mode", [
     (8192, 4096, 256, "bf16"),     # 32 x 16 tiles of 256 x 256, four K blocks: two or three column tiles per pair
     (7000, 1288, 96, "f32"),       # ragged rows, ragged last column tile, K not a multiple of 64
-    (4100, 2560, 512, "bf16"),     # eight K blocks: 128-wide column tiles
+    (4100, 2560, 512, "bf16"),     # eight K blocks: B takes 128 KB, so a four-stage ring and one staging box per warp
+    (3000, 1032, 384, "f32"),      # six K blocks, fp32 boxes, ragged rows and columns
     (40000, 256, 48, "f32"),       # one column tile, many row tiles
 ])
 def test_persistent_form_for_short_contractions_with_a_large_output(dev, M, N, K, out_mode):

@@ -297,7 +297,7 @@ def test_private_outlier_tokens_need_one_power_iteration(dev):
 
 
 # ------------------------------------------------------------------ pre-norm unit, backward (Section 3.3)
-@pytest.mark.parametrize("n,d,r", [(1024, 512, 64), (1000, 768, 96), (4096, 1024, 256)])
+@pytest.mark.parametrize("n,d,r", [(1024, 512, 64), (1000, 768, 96), (4096, 1024, 256), (2048, 1024, 512)])
 def test_prenorm_backward_matches_the_three_gradient_equations(dev, n, d, r):
     w = synth.scaled(synth.WORKLOADS["llama7b_block"], n_tokens=n, d=d, rank=r, signal_rank=min(2 * r, d // 2))
     w = synth.Workload(**{**w.__dict__, "prenorm": "rms"})
@@ -323,7 +323,7 @@ def test_prenorm_backward_matches_the_three_gradient_equations(dev, n, d, r):
 
 # ------------------------------------------------------------------ element-wise consumer (Section 3.1)
 @pytest.mark.parametrize("kind,name", [(B.ACT_SILU, "silu"), (B.ACT_GELU, "gelu")])
-@pytest.mark.parametrize("n,d,r", [(1024, 512, 64), (1000, 776, 96), (4096, 2048, 256)])
+@pytest.mark.parametrize("n,d,r", [(1024, 512, 64), (1000, 776, 96), (4096, 2048, 256), (2048, 1024, 512)])
 def test_activation_backward_matches_the_gradient_equation(dev, kind, name, n, d, r):
     """grad_X = grad_Z * f'(A~) with A~ = U V never stored: the device against the oracle's equation on the same
     stored factors (this isolates the consumer), and against the exact gradient at the uncompressed input."""
