@@ -116,7 +116,9 @@ cudaError_t small_block_cluster_wait_probe_launch(uint32_t* dev_status, uint64_t
 // Plain CUDA-core kernel for any shape and type (fp32 path, small or odd shapes).
 cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t stream);
 // fp32 x fp32 -> fp32 for matrices of a few hundred rows and columns (32 x 32 tiles, one per CTA).
-cudaError_t gemm_f32_small_launch(const GemmDesc& g, cudaStream_t stream);
+// `second`: an independent product carried by the same launch (both may read what earlier launches wrote;
+// neither may read the other's output).
+cudaError_t gemm_f32_small_launch(const GemmDesc& g, cudaStream_t stream, const GemmDesc* second = nullptr);
 
 // ---------------------------------------------------------------- sampler and gather
 // idx_copy (optional) receives the same indices; clear_status: the kernel sets the status word instead of OR-ing

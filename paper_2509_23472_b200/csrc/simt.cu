@@ -167,14 +167,19 @@ __global__ void reduce_split3_kernel(const float* __restrict__ partials, int n_p
 // fp32 product for the r x r blocks of the two-level small-block scheme: C = alpha * A B (+ C), all of a few
 // hundred rows and columns.  32 x 32 output tiles on 64 threads (4 x 4 outputs each, operands read from
 // shared memory along the contraction index with 16-byte loads), so that a 256 x 256 product spreads over
-// 64 SMs; the K loop is double-buffered through registers.
+// 64 SMs; the K loop is double-buffered through registers.  One launch carries up to two independent products
+// (grid.z picks one): the two-level scheme has a pair of them at one point of its chain.
 constexpr int kT32 = 32, kT32Ld = 36;
 
-__global__ void __launch_bounds__(64) gemm_f32_tile32_kernel(SimtParams p) {
+__global__ void __launch_bounds__(64) gemm_f32_tile32_kernel(SimtParams p0, SimtParams p1) {
   __shared__ __align__(16) float As[kT32 * kT32Ld];   // [m][k]
   __shared__ __align__(16) float Bs[kT32 * kT32Ld];   // [n][k]
+  const SimtParams& p = blockIdx.z ? p1 : p0;
   const int tid = threadIdx.x;
   const int m0 = blockIdx.y * kT32, n0 = blockIdx.x * kT32;
+  pdl_wait();
+  pdl_launch_dependents();
+  if (m0 >= p.M || n0 >= p.N) return;
   const int tm = tid >> 3, tn = tid & 7;               // outputs (4 tm + i, tn + 8 j)
   const float* A = (const float*)p.A[0];
   const float* B = (const float*)p.B[0];
@@ -499,20 +504,27 @@ cudaError_t reduce_split3_launch(const float* partials, int n_partials, int64_t 
   return cudaGetLastError();
 }
 
-cudaError_t gemm_f32_small_launch(const GemmDesc& g, cudaStream_t stream) {
-  if (g.a_type != ELEM_F32 || g.b_type != ELEM_F32 || g.out != OUT_F32 || g.n_terms != 1 || g.splits > 1)
-    return cudaErrorNotSupported;
-  SimtParams p = {};
-  p.M = g.M; p.N = g.N; p.K = g.K;
-  if (g.a_mn) { p.sam = 1; p.sak = g.lda; } else { p.sam = g.lda; p.sak = 1; }
-  if (g.b_mn) { p.sbn = 1; p.sbk = g.ldb; } else { p.sbn = g.ldb; p.sbk = 1; }
-  p.n_terms = 1;
-  p.A[0] = g.terms[0].A; p.B[0] = g.terms[0].B;
-  p.out = g.out; p.C0 = g.C0; p.ldc = g.ldc; p.splits = 1;
-  p.accumulate = g.accumulate ? 1 : 0;
-  p.alpha = g.alpha;
-  dim3 grid((g.N + kT32 - 1) / kT32, (g.M + kT32 - 1) / kT32);
-  gemm_f32_tile32_kernel<<<grid, 64, 0, stream>>>(p);
+cudaError_t gemm_f32_small_launch(const GemmDesc& g, cudaStream_t stream, const GemmDesc* second) {
+  auto fill = [](const GemmDesc& g, SimtParams& p) {
+    if (g.a_type != ELEM_F32 || g.b_type != ELEM_F32 || g.out != OUT_F32 || g.n_terms != 1 || g.splits > 1)
+      return false;
+    p = SimtParams{};
+    p.M = g.M; p.N = g.N; p.K = g.K;
+    if (g.a_mn) { p.sam = 1; p.sak = g.lda; } else { p.sam = g.lda; p.sak = 1; }
+    if (g.b_mn) { p.sbn = 1; p.sbk = g.ldb; } else { p.sbn = g.ldb; p.sbk = 1; }
+    p.n_terms = 1;
+    p.A[0] = g.terms[0].A; p.B[0] = g.terms[0].B;
+    p.out = g.out; p.C0 = g.C0; p.ldc = g.ldc; p.splits = 1;
+    p.accumulate = g.accumulate ? 1 : 0;
+    p.alpha = g.alpha;
+    return true;
+  };
+  SimtParams p0, p1;
+  if (!fill(g, p0) || (second && !fill(*second, p1))) return cudaErrorNotSupported;
+  if (!second) p1 = p0;
+  const int M = second ? std::max(g.M, second->M) : g.M, N = second ? std::max(g.N, second->N) : g.N;
+  dim3 grid((N + kT32 - 1) / kT32, (M + kT32 - 1) / kT32, second ? 2 : 1);
+  LORACT_CUDA_TRY(launch_pdl(gemm_f32_tile32_kernel, grid, dim3(64), 0, stream, p0, p1));
   count_launch(__func__, stream);
   return cudaGetLastError();
 }

@@ -306,28 +306,32 @@ cudaError_t factor_blocks(const TwoLevelCtx& c, float* W, float* X, __nv_bfloat1
   float* T2 = T1 + (size_t)r2 * r1;
   float* Tnext = T2 + (size_t)r2 * r1;
   LORACT_CUDA_TRY(factor_blocks(c, W, X, hi, lo, r1, Tnext, top));
-  auto simt = [&](int M, int N, int K, const float* A, int64_t lda, const float* B, int64_t ldb, bool b_mn, float* C,
-                  int64_t ldc, float alpha, bool accumulate) {
+  auto product = [&](int M, int N, int K, const float* A, int64_t lda, const float* B, int64_t ldb, bool b_mn,
+                     float* C, int64_t ldc, float alpha, bool accumulate) {
     GemmDesc g;
     g.M = M; g.N = N; g.K = K; g.lda = lda; g.ldb = ldb; g.b_mn = b_mn;
     g.a_type = g.b_type = ELEM_F32;
     g.terms[0] = {A, B};
     g.out = OUT_F32; g.C0 = C; g.ldc = ldc; g.alpha = alpha; g.accumulate = accumulate;
-    return gemm_f32_small_launch(g, c.stream);
+    return g;
   };
   const float* W21 = W + (size_t)r1 * ld;
   float* W22 = W + (size_t)r1 * ld + r1;
   float* X22 = X + (size_t)r1 * ld + r1;
   float* X21 = X + (size_t)r1 * ld;
   // L21 = W21 X11^T : C[m][n] = sum_k W21[m][k] X11[n][k]
-  LORACT_CUDA_TRY(simt(r2, r1, r1, W21, ld, X, ld, false, T1, r1, 1.f, false));
-  // S = W22 - L21 L21^T, in place
-  LORACT_CUDA_TRY(simt(r2, r2, r1, T1, r1, T1, r1, false, W22, ld, -1.f, true));
+  LORACT_CUDA_TRY(gemm_f32_small_launch(product(r2, r1, r1, W21, ld, X, ld, false, T1, r1, 1.f, false), c.stream));
+  // One launch, two products that both read L21: S = W22 - L21 L21^T (in place) and
+  // T2 = L21 X11, T2[m][n] = sum_k L21[m][k] X11[k][n], which the last product below needs.
+  {
+    const GemmDesc schur = product(r2, r2, r1, T1, r1, T1, r1, false, W22, ld, -1.f, true);
+    const GemmDesc l21x11 = product(r2, r1, r1, T1, r1, X, ld, true, T2, r1, 1.f, false);
+    LORACT_CUDA_TRY(gemm_f32_small_launch(schur, c.stream, &l21x11));
+  }
   LORACT_CUDA_TRY(factor_blocks(c, W22, X22, hi + (size_t)r1 * ld + r1, lo ? lo + (size_t)r1 * ld + r1 : nullptr, r2,
                                 Tnext, false));
-  // X21 = -X22 (L21 X11): T2[m][n] = sum_k L21[m][k] X11[k][n];  X21[m][n] = -sum_k X22[m][k] T2[k][n]
-  LORACT_CUDA_TRY(simt(r2, r1, r1, T1, r1, X, ld, true, T2, r1, 1.f, false));
-  LORACT_CUDA_TRY(simt(r2, r1, r2, X22, ld, T2, r1, true, X21, ld, -1.f, false));
+  // X21 = -X22 T2 : X21[m][n] = -sum_k X22[m][k] T2[k][n]
+  LORACT_CUDA_TRY(gemm_f32_small_launch(product(r2, r1, r2, X22, ld, T2, r1, true, X21, ld, -1.f, false), c.stream));
   return split_block_launch(X21, r2, r1, ld, hi + (size_t)r1 * ld, lo ? lo + (size_t)r1 * ld : nullptr, c.stream);
 }
 
