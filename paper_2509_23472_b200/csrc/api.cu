@@ -185,6 +185,7 @@ cudaError_t simt_split_f32(GemmDesc g, int splits, float* partials, float* out, 
   return reduce_partials_launch(partials, splits, g.split_stride, g.split_stride, out, nullptr, stream);
 }
 
+constexpr double kL2KeepBytes = 48.0 * 1024 * 1024;   // of X, asked to stay in L2 between the two passes (about 20 MB do)
 constexpr int kReduceFirst = 8;    // partial count from which a separate, all-SM reduction pays
 cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs& w, uint32_t* status,
                    cudaStream_t stream) {
@@ -249,6 +250,13 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
     trace_label("pass 1: Y = X Omega^T");
     if (p.bf16) {
       g.out = OUT_SPLIT; g.C0 = w.Yh; g.C1 = w.Yl;
+      // The projection reads X again a few hundred microseconds from now: the last columns this pass streams are
+      // asked to stay in L2 (as many bytes of X as kL2KeepBytes).
+      const double x_bytes = (double)n * (double)p.d * 2.0;
+      if (x_bytes > 0) {
+        const double frac = kL2KeepBytes >= x_bytes ? 1.0 : kL2KeepBytes / x_bytes;
+        g.a_keep_from_k = (int64_t)((1.0 - frac) * (double)p.d);
+      }
       LORACT_CUDA_TRY(run_gemm(g, status, stream));
     } else {
       LORACT_CUDA_TRY(simt_split_f32(g, simt_splits(p.d), w.part32, w.Y32, stream));

@@ -100,6 +100,9 @@ struct GemmDesc {
   const float* ep_row_b = nullptr;
   const void* ep_col = nullptr;
   int ep_kind = 0;         // OUT_ACT_BWD: which activation
+  // Two-CTA kernel, K-major A: loads of A from this K element on ask L2 to evict them last (a later kernel
+  // reads the same bytes again); negative: no hint.
+  int64_t a_keep_from_k = -1;
 };
 
 // tcgen05 engine: bf16 operands, fp32 accumulation in tensor memory.  Returns cudaErrorNotSupported

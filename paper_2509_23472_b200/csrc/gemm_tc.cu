@@ -63,6 +63,7 @@ struct TcParams {
   int st_units;       // streaming kernel: tiles in all (column tile major, then M)
   int st_stages;      // streaming kernel: stages of the A ring (<= kStreamStages)
   int store_bufs;     // staging boxes per epilogue warp (1 or 2)
+  int a_keep_from_kb; // two-CTA kernel: K block from which the loads of A carry an evict-last hint (kb_total: none)
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -218,7 +219,7 @@ __device__ __forceinline__ void stage_acquire(const StoreStage& st, int lane) {
   }
 }
 __device__ __forceinline__ unsigned char* stage_box(const StoreStage& st, uint32_t k) {
-  return st.base + ((st.cnt + k) % st.bufs) * kStoreBoxBytes;
+  return st.base + (st.bufs == 1 ? 0u : ((st.cnt + k) & 1u)) * kStoreBoxBytes;
 }
 __device__ __forceinline__ void stage_write16(unsigned char* box, int lane, int chunk, uint4 v) {
   *reinterpret_cast<uint4*>(box + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = v;
@@ -625,6 +626,20 @@ __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorM
       ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(bar_cluster_addr), "r"(x), "r"(y)
       : "memory");
 }
+// The same load with an L2 eviction-priority hint (a policy made by createpolicy).
+__device__ __forceinline__ void tma_load_2d_pair_hint(void* smem_dst, const CUtensorMap* map, uint32_t bar_cluster_addr,
+                                                      int x, int y, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(smem_u32(smem_dst)), "l"((uint64_t)map), "r"(bar_cluster_addr), "r"(x), "r"(y), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
 __device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
   asm volatile(
       "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -692,12 +707,14 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
       const int nb0 = n0 + (int)cta_rank * half_n;           // this CTA's half of the B tile
       // stage, parity, term and K block are carried along (no division in the loop)
       int s = (warp == 0 ? 0 : 1) % kPairStages;
+      const uint64_t keep_policy = l2_policy_evict_last();
       uint32_t parity = 1u;
       int term = 0, kb = (warp == 0 ? 0 : 1);
       while (kb >= kb_count && kb_count > 0) { kb -= kb_count; ++term; }
       for (int it = (warp == 0 ? 0 : 1); it < n_iter; it += 2) {
         if (!mbar_wait_bounded(&empty_bar[s], parity, &abort_flag)) break;
         const int k0 = (kb_begin + kb) * kBK;
+        const int kb_now = kb;
         unsigned char* a_dst = tiles + (size_t)s * stage_bytes;
         unsigned char* b_dst = a_dst + kABytes;
         // the leader expects the bytes of both CTAs on its barrier
@@ -709,6 +726,8 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
         if (A_MN) {
           tma_load_2d_pair(a_dst, &maps.a[term_now], bar, m0, k0);
           tma_load_2d_pair(a_dst + 8192, &maps.a[term_now], bar, m0 + 64, k0);
+        } else if (kb_begin + kb_now >= p.a_keep_from_kb) {
+          tma_load_2d_pair_hint(a_dst, &maps.a[term_now], bar, k0, m0, keep_policy);
         } else {
           tma_load_2d_pair(a_dst, &maps.a[term_now], bar, k0, m0);
         }
@@ -732,15 +751,16 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
       bool ok = true;
       int s = 0;
       uint32_t parity = 0u;
-      const uint32_t tiles_u32 = smem_u32(tiles);
+      // descriptors address shared memory in 16-byte units: one addition per stage instead of building them anew
+      const uint64_t a_desc0 = make_smem_desc(smem_u32(tiles), A_MN);
+      const uint64_t b_desc0 = make_smem_desc(smem_u32(tiles) + kABytes, B_MN);
+      const uint32_t stage_units = stage_bytes >> 4;
       for (int it = 0; it < n_iter && ok; ++it) {
         ok = mbar_wait_bounded(&full_bar[s], parity, &abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t a_addr = tiles_u32 + (uint32_t)s * stage_bytes;
-        const uint32_t b_addr = a_addr + kABytes;
-        const uint64_t a_desc = make_smem_desc(a_addr, A_MN);
-        const uint64_t b_desc = make_smem_desc(b_addr, B_MN);
+        const uint64_t a_desc = a_desc0 + (uint64_t)((uint32_t)s * stage_units);
+        const uint64_t b_desc = b_desc0 + (uint64_t)((uint32_t)s * stage_units);
 #pragma unroll
         for (int k = 0; k < kBK / 16; ++k) {
           const uint64_t a_k = a_desc + (uint64_t)((A_MN ? 2048u : 32u) >> 4) * k;
@@ -880,7 +900,9 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   if (warp == 0) {
     if (lane == 0) {
       const uint32_t bar_b = map_to_rank(smem_u32(&b_full), 0u);
-      int it = 0, nb = 0, cur_nt = -1;
+      int nb = 0, cur_nt = -1;
+      int s = 0;                 // ring stage and its phase, carried along (no division in the loop)
+      uint32_t ph = 0u;
       bool ok = true;
       for (int u = u_begin; u < u_end && ok; ++u) {
         const int nt = u / p.st_m_tiles, mt = u - nt * p.st_m_tiles;
@@ -898,12 +920,12 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
           cur_nt = nt;
         }
         const int m0 = mt * 2 * kBM + (int)cta_rank * kBM;
-        for (int kb = 0; kb < p.kb_total; ++kb, ++it) {
-          const int s = it % p.st_stages;
-          ok = mbar_wait_bounded(&a_empty[s], (uint32_t)(((it / p.st_stages) & 1) ^ 1), &abort_flag);
+        for (int kb = 0; kb < p.kb_total; ++kb) {
+          ok = mbar_wait_bounded(&a_empty[s], ph ^ 1u, &abort_flag);
           if (!ok) break;
           if (leader) mbar_arrive_expect_tx(&a_full[s], 2u * kABytes);
           tma_load_2d_pair(ring + (size_t)s * kABytes, &maps.a[0], map_to_rank(smem_u32(&a_full[s]), 0u), kb * kBK, m0);
+          if (++s == p.st_stages) { s = 0; ph ^= 1u; }
         }
       }
     }
@@ -912,7 +934,12 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
       // instruction descriptor: fp32 accumulator, bf16 A (K-major) and B (MN-major), N >> 3, M = 256 >> 4
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(p.bn >> 3) << 17) |
                              ((uint32_t)((2 * kBM) >> 4) << 24);
-      int it = 0, nb = 0, cur_nt = -1;
+      // descriptors address shared memory in 16-byte units: a ring stage is kABytes, a K block of B b_kb_bytes
+      const uint64_t a_desc0 = make_smem_desc(smem_u32(ring), false);
+      const uint64_t b_desc0 = make_smem_desc(smem_u32(b_res), true);
+      int nb = 0, cur_nt = -1;
+      int s = 0;                 // ring stage and its phase, carried along (a division here costs 9 % of the kernel)
+      uint32_t ph = 0u;
       bool ok = true;
       for (int u = u_begin, ui = 0; u < u_end && ok; ++u, ++ui) {
         const int j = ui & 1;
@@ -928,18 +955,18 @@ gemm_tc_stream_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
         }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(j * p.bn);
-        for (int kb = 0; kb < p.kb_total; ++kb, ++it) {
-          const int s = it % p.st_stages;
-          ok = mbar_wait_bounded(&a_full[s], (uint32_t)((it / p.st_stages) & 1), &abort_flag);
+        for (int kb = 0; kb < p.kb_total; ++kb) {
+          ok = mbar_wait_bounded(&a_full[s], ph, &abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint64_t a_desc = make_smem_desc(smem_u32(ring + (size_t)s * kABytes), false);
-          const uint64_t b_desc = make_smem_desc(smem_u32(b_res + (size_t)kb * b_kb_bytes), true);
+          const uint64_t a_desc = a_desc0 + (uint64_t)((uint32_t)s * (kABytes >> 4));
+          const uint64_t b_desc = b_desc0 + (uint64_t)((uint32_t)kb * (b_kb_bytes >> 4));
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k)
             tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(32u >> 4) * k, b_desc + (uint64_t)(2048u >> 4) * k, idesc,
                              (kb > 0 || k > 0) ? 1u : 0u);
           tc_commit_pair(&a_empty[s]);
+          if (++s == p.st_stages) { s = 0; ph ^= 1u; }
         }
         if (!ok) break;
         tc_commit_pair(&acc_full[j]);
@@ -1228,6 +1255,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   p.ep_kind = g.ep_kind;
   p.dev_status = dev_status;
   p.st_m_tiles = 0; p.st_units = 0; p.tma_store = 0; p.st_stages = kStreamStages; p.store_bufs = kStoreBufs;
+  p.a_keep_from_kb = g.a_keep_from_k >= 0 ? (int)(g.a_keep_from_k / kBK) : p.kb_total;
 
   TmapPack maps;
   for (int t = 0; t < g.n_terms; ++t) {
