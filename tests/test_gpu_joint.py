@@ -56,6 +56,31 @@ def test_sharded_factorisation_is_the_factorisation_of_the_whole_matrix(dev, nam
     print(f"joint {sizes}: err {e_gpu:.5f} oracle {e_ref:.5f} projection distance {proj:.2e}")
 
 
+def test_gathered_rows_are_byte_identical_and_a_window_zeroes_the_rest(dev):
+    # The gather on its own: with the window covering the whole matrix the staged entry returns exactly
+    # X[idx, :] (the bytes, not values within a tolerance); with a window of some rows, the sampled rows outside
+    # it come back as zeros, so that the sum over the shards is X[idx, :] again.
+    n, d, r = 3000, 776, 96
+    g = torch.Generator(device=dev)
+    g.manual_seed(11)
+    X = torch.randn(n, d, generator=g, device=dev).bfloat16()           # the staged entry points take bf16
+    idx_o = orc.sample_indices(n, r, seed=9, call_id=2)
+    whole = joint.JointShard(X, n, 0, r, seed=9, call_id=2)
+    S = whole.sample_rows()
+    torch.cuda.synchronize()
+    assert np.array_equal(whole.idx.cpu().numpy().astype(np.int64), idx_o)
+    expect = X[torch.as_tensor(idx_o, device=dev)]
+    assert torch.equal(S.view(torch.uint8), expect.contiguous().view(torch.uint8))
+    row0, n_local = 1000, 1200
+    part = joint.JointShard(X[row0:row0 + n_local].contiguous(), n, row0, r, seed=9, call_id=2)
+    Sp = part.sample_rows()
+    torch.cuda.synchronize()
+    inside = torch.as_tensor((idx_o >= row0) & (idx_o < row0 + n_local), device=dev)
+    assert 0 < int(inside.sum()) < r                                    # the case has rows on both sides
+    assert torch.equal(Sp[inside].view(torch.uint8), expect[inside].contiguous().view(torch.uint8))
+    assert not bool(Sp[~inside].view(torch.uint8).any())
+
+
 def test_joint_rejects_bad_arguments_before_launching(dev):
     X = torch.zeros(512, 256, dtype=torch.bfloat16, device=dev)
     before = B.kernel_launch_count()
