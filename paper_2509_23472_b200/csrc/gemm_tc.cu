@@ -14,6 +14,7 @@
 #include <cuda.h>
 
 #include <map>
+#include <atomic>
 #include <mutex>
 #include <tuple>
 
@@ -1107,13 +1108,13 @@ int pick_bn(int N) {
 
 template <bool A_MN, bool B_MN>
 cudaError_t launch_variant(const TmapPack& maps, const TcParams& p, dim3 grid, size_t smem, cudaStream_t stream) {
-  static bool configured[64] = {};
+  static std::atomic<bool> configured[64];   // zero-initialised; set once the attribute is in place on a device
   int dev = 0;
   LORACT_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64 || !configured[dev]) {
+  if (dev < 0 || dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
     LORACT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          kStages * (kABytes + 32768) + 1024));
-    if (dev >= 0 && dev < 64) configured[dev] = true;
+    if (dev >= 0 && dev < 64) configured[dev].store(true, std::memory_order_release);
   }
   LORACT_CUDA_TRY(launch_pdl(gemm_tc_kernel<A_MN, B_MN>, grid, dim3(kThreads), smem, stream, maps, p));
   count_launch(__func__, stream);
@@ -1122,13 +1123,13 @@ cudaError_t launch_variant(const TmapPack& maps, const TcParams& p, dim3 grid, s
 
 template <bool A_MN, bool B_MN>
 cudaError_t launch_pair_variant(const TmapPack& maps, const TcParams& p, dim3 grid, size_t smem, cudaStream_t stream) {
-  static bool configured[64] = {};
+  static std::atomic<bool> configured[64];   // zero-initialised; set once the attribute is in place on a device
   int dev = 0;
   LORACT_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64 || !configured[dev]) {
+  if (dev < 0 || dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
     LORACT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_pair_kernel<A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          kPairStages * (kABytes + 16384) + 1024));
-    if (dev >= 0 && dev < 64) configured[dev] = true;
+    if (dev >= 0 && dev < 64) configured[dev].store(true, std::memory_order_release);
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
@@ -1151,12 +1152,12 @@ cudaError_t launch_pair_variant(const TmapPack& maps, const TcParams& p, dim3 gr
 
 // Pairs the streaming kernel is launched with: as many as can be resident at once (one CTA per SM).
 cudaError_t launch_stream(const TmapPack& maps, TcParams p, size_t smem, cudaStream_t stream) {
-  static bool configured[64] = {};
-  static int max_pairs[64] = {};
+  static std::atomic<bool> configured[64];   // zero-initialised; set once the attribute is in place on a device
+  static std::atomic<int> max_pairs[64];
   int dev = 0;
   LORACT_CUDA_TRY(cudaGetDevice(&dev));
-  const bool cached = dev >= 0 && dev < 64 && configured[dev];
-  int pairs = cached ? max_pairs[dev] : 0;
+  const bool cached = dev >= 0 && dev < 64 && configured[dev].load(std::memory_order_acquire);
+  int pairs = cached ? max_pairs[dev].load(std::memory_order_relaxed) : 0;
   if (!cached) {
     const int smem_max = kStreamSmemMax;
     LORACT_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
@@ -1174,7 +1175,10 @@ cudaError_t launch_stream(const TmapPack& maps, TcParams p, size_t smem, cudaStr
       n = prop.multiProcessorCount / 2;
     }
     pairs = n < 1 ? 1 : n;
-    if (dev >= 0 && dev < 64) { max_pairs[dev] = pairs; configured[dev] = true; }
+    if (dev >= 0 && dev < 64) {
+      max_pairs[dev].store(pairs, std::memory_order_relaxed);
+      configured[dev].store(true, std::memory_order_release);
+    }
   }
   if (pairs > p.st_units) pairs = p.st_units;
   cudaLaunchConfig_t cfg = {};

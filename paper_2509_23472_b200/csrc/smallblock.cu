@@ -10,6 +10,8 @@
 // cluster split the rows of every panel and synchronise with the hardware cluster barrier.
 #include <cooperative_groups.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 namespace cg = cooperative_groups;
@@ -257,13 +259,13 @@ small_block_kernel(SBParams p) {
 template <typename T>
 cudaError_t launch_typed(const SBParams& p, cudaStream_t stream) {
   const size_t smem = ((size_t)p.r * kNB + kNB * (kNB + 1) + kNB * kNB) * sizeof(T);
-  static bool configured[64] = {};  // per device and instantiation
+  static std::atomic<bool> configured[64];  // per device and instantiation, zero-initialised
   int dev = 0;
   LORACT_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64 || !configured[dev]) {
+  if (dev < 0 || dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
     LORACT_CUDA_TRY(cudaFuncSetAttribute(small_block_kernel<T>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    if (dev >= 0 && dev < 64) configured[dev] = true;
+    if (dev >= 0 && dev < 64) configured[dev].store(true, std::memory_order_release);
   }
   small_block_kernel<T><<<kCluster, kSBThreads, smem, stream>>>(p);
   count_launch(__func__, stream);

@@ -23,6 +23,8 @@
 // Every wait is bounded (a wall-clock limit for barriers, an iteration limit for flag words); on expiry the
 // CTA records LORACT_DEV_WAIT_EXPIRED, stops waiting and runs to its end (results are then invalid but
 // every access stays in bounds).
+#include <atomic>
+
 #include "common.cuh"
 
 namespace loract {
@@ -852,13 +854,13 @@ cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t str
   p.scale_n = a.scale_n;
   p.scale_ld = a.scale_ld;
   const size_t smem = (size_t)(kMaxTri + kXSlots) * kSlot * sizeof(float) + (size_t)(2 * kB * kLcolLd) * sizeof(float);
-  static bool configured[64] = {};
+  static std::atomic<bool> configured[64];
   int dev = 0;
   LORACT_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64 || !configured[dev]) {
+  if (dev < 0 || dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
     LORACT_CUDA_TRY(cudaFuncSetAttribute(small_block_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem));
-    if (dev >= 0 && dev < 64) configured[dev] = true;
+    if (dev >= 0 && dev < 64) configured[dev].store(true, std::memory_order_release);
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(kCl, 1, 1);
