@@ -61,7 +61,7 @@ typedef struct {
   int64_t d;             /* columns of X (the paper's n)                                     */
   int64_t ldx;           /* row stride of X in elements, >= d                                */
   int32_t rank;          /* r (the paper's k)                                                */
-  int32_t power_iters;   /* t of Algorithm 1 (lines 3 to 6), 0 <= t <= 8; the paper's runs use 0   */
+  int32_t power_iters;   /* t of Algorithm 1 (its loop), 0 <= t <= 8;     the paper's runs use 0   */
   int32_t dtype;         /* loract_dtype_t of X, U, V, X_out, A_out, G, gamma, beta          */
   int32_t reserved;      /* must be 0                                                        */
   uint64_t seed;         /* Philox key                                                       */
@@ -77,7 +77,7 @@ typedef struct {
  * returns its results) and can be shared by every layer's call that does not overlap another on the GPU. */
 size_t loract_workspace_bytes(const loract_desc_t* desc);
 
-/* Algorithm 1, line 1: the `rank` distinct row indices, uniform without replacement.  The sample is the
+/* Algorithm 1, sampling step: the `rank` distinct row indices, uniform without replacement.  The sample is the
  * first `rank` distinct values of the stream c_i = (w_i * n_tokens) >> 32, w_i = word (i mod 4) of the
  * Philox4x32-10 block with key (seed lo, seed hi) and counter (i div 4, 0, call_id lo, call_id hi),
  * in stream order.  idx_dev: device, `rank` int32, written.  ws: device scratch, >= 256 bytes. */
@@ -149,15 +149,15 @@ loract_status_t loract_activation_backward(const loract_desc_t* desc, const void
  * seed / call_id are the same on every shard); between stages the caller adds the small matrices over all shards
  * (an all-reduce with NCCL; what arrives lands in local memory before the next stage reads it) -- the library
  * itself does no communication.  bf16 only; every shard needs at least `rank` rows.
- *   1. loract_joint_sample_rows : line 1.  The `rank` sampled rows of the whole matrix (indices in [0, n_global),
+ *   1. loract_joint_sample_rows : the sampling step.  The `rank` sampled rows of the whole matrix (indices in [0, n_global),
  *      the same on every shard); S (rank x d) receives those that live on this shard, zeros elsewhere.
  *      -> add S over the shards (one non-zero contribution per row: exact).
- *   2. loract_joint_sketch      : line 2.  Y_local = X_local Omega^T with the test matrix Omega made from S_sum (the
+ *   2. loract_joint_sketch      : the sketch.  Y_local = X_local Omega^T with the test matrix Omega made from S_sum (the
  *      same bits on every shard), and W_partial (rank x rank fp32) = Y_local^T Y_local.  -> add W_partial.
- *   3. loract_joint_orthonormalise, round 0 : line 7, first half.  Y_local <- Y_local L^-T with L L^T = W_sum;
+ *   3. loract_joint_orthonormalise, round 0 : the QR step, first half.  Y_local <- Y_local L^-T with L L^T = W_sum;
  *      W_next_partial = the new Y_local^T Y_local.  -> add W_next_partial.
  *      round 1 : second half.  U_local (n_tokens x rank) = Y_local L^-T with the factor of the second sum.
- *   4. loract_joint_project     : line 8.  V_partial (rank x d fp32) = U_local^T X_local.  -> add V_partial.
+ *   4. loract_joint_project     : the projection.  V_partial (rank x d fp32) = U_local^T X_local.  -> add V_partial.
  *   5. loract_joint_finish      : V (rank x d, bf16) = V_sum rounded once.
  * The sketch and the once-orthonormalised sketch stay in `ws` between the stages: the same `ws` (at least
  * loract_joint_workspace_bytes(desc) bytes) must be passed to stages 1 to 4 of one factorisation.  The device

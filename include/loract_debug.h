@@ -12,7 +12,7 @@
 extern "C" {
 #endif
 
-/* The contraction behind Algorithm 1 lines 2 and 8 and behind Reconstruct:
+/* The contraction behind the sketch and the projection of Algorithm 1 and behind Reconstruct:
  * C (M x N) = sum_{t < n_terms} A_t B_t, contraction length K, fp32 accumulation.
  * a_mn = 0: A_t stored [M][K] (row stride lda); a_mn = 1: stored [K][M].  b_mn = 0: B_t stored [N][K]
  * (row stride ldb); b_mn = 1: stored [K][N].  a_type / b_type: 0 fp32, 1 bf16.  A and B point to
@@ -27,7 +27,7 @@ loract_status_t loract_debug_gemm(int32_t M, int32_t N, int32_t K, int32_t a_mn,
                                   void* C0, void* C1, int64_t ldc, int32_t splits, int64_t split_stride,
                                   int32_t acc64, int32_t engine, uint32_t* status_word, void* stream);
 
-/* Line 8 of Algorithm 1 alone, exactly as loract_compress runs it (same kernels, same launch shapes):
+/* The projection step of Algorithm 1 alone, exactly as loract_compress runs it (same kernels, same launch shapes):
  * V (rank x d) = U^T X from a stored U (n_tokens x rank).  ws as for loract_compress.  For timing that step in
  * isolation. */
 loract_status_t loract_debug_project(const loract_desc_t* desc, const void* U, const void* X, void* V, void* ws,
@@ -57,7 +57,7 @@ loract_status_t loract_debug_wait_expiry(int32_t which, uint64_t limit_ns, uint3
 /* The cudaError_t behind the most recent LORACT_ERR_CUDA returned by any entry point (0 if none yet). */
 int32_t loract_debug_last_cuda_error(void);
 
-/* The small-block step of the orthonormalisation (Algorithm 1 line 7 done through Gram matrices):
+/* The small-block step of the orthonormalisation (the QR step of Algorithm 1 done through Gram matrices):
  * W = sum of n_partials r x r matrices (fp32 if partial_f64 == 0, else fp64; `partial_stride` elements
  * apart); L L^T = W + shift_rel * mean(diag W) * I; writes L^{-1} (lower triangular, row-major) as fp32
  * (linv_f32), as a bf16 hi/lo pair (linv_hi, linv_lo), any of which may be NULL.  use_f64 selects the

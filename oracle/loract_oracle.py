@@ -91,7 +91,7 @@ def candidate(i: int, n_rows: int, seed: int, call_id: int) -> int:
 
 
 def sample_indices(n_rows: int, k: int, seed: int, call_id: int = 0) -> np.ndarray:
-    """Algorithm 1, line 1: k distinct row indices, uniform without replacement.
+    """Algorithm 1, sampling step: k distinct row indices, uniform without replacement.
 
     Defined as the first k distinct values of the candidate stream, kept in
     stream order.
@@ -140,16 +140,17 @@ def _f64(a):
 
 
 def range_finder(A, Omega_T, t: int = 0):
-    """Lines 2-7 of Algorithm 1 for a given test matrix (rows of Omega_T are the test vectors).
+    """Algorithm 1 from the sketch to the orthonormal basis, for a given test matrix (rows of Omega_T are the
+    test vectors).
 
     Y = A Omega;  t times { Y = QR;  Y = A (A^T Q) };  Y = QR;  returns Q (m x k).
     """
     A = _f64(A)
-    Y = A @ _f64(Omega_T).T                      # line 2
-    for _ in range(int(t)):                      # lines 3-6
+    Y = A @ _f64(Omega_T).T                      # the sketch
+    for _ in range(int(t)):                      # the power-iteration loop
         Q, _ = np.linalg.qr(Y, mode="reduced")
         Y = A @ (A.T @ Q)
-    Q, _ = np.linalg.qr(Y, mode="reduced")       # line 7
+    Q, _ = np.linalg.qr(Y, mode="reduced")       # QR of the sketch
     return Q
 
 
@@ -158,11 +159,11 @@ def decompose(A, k: int, t: int = 0, seed: int = 0, call_id: int = 0, idx=None):
     A = _f64(A)
     m, _ = A.shape
     if idx is None:
-        idx = sample_indices(m, k, seed, call_id)    # line 1
+        idx = sample_indices(m, k, seed, call_id)    # the sampling step
     idx = np.asarray(idx, dtype=np.int64)
-    A_k = A[idx, :]                                  # line 1: the sampled rows
-    Q = range_finder(A, A_k, t)                      # lines 2-7
-    U = Q                                            # line 8
+    A_k = A[idx, :]                                  # the sampled rows
+    Q = range_finder(A, A_k, t)                      # sketch, loop, QR
+    U = Q                                            # the factor pair
     V = Q.T @ A
     return U, V, idx
 

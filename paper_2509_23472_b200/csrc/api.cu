@@ -235,7 +235,7 @@ cudaError_t precondition_rows(const void* T, int l, int64_t d, bool bf16, void* 
   return run_gemm(g, status, stream);
 }
 
-// Lines 2 and 7 of Algorithm 1 for a test matrix Omega (l x d, rows are the test vectors):
+// The sketch and the orthonormalisation of Algorithm 1 for a test matrix Omega (l x d, rows are the test vectors):
 // Y = X Omega^T, then two rounds of { W = Y^T Y = L L^T ; Y <- Y L^{-T} }.  U (n x l) receives Q.
 cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* Omega, void* U,
                         const BasisWs& w, uint32_t* status, cudaStream_t stream) {
@@ -303,7 +303,7 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
   return cudaSuccess;
 }
 
-// Line 8 of Algorithm 1: V = U^T X  (l x d), from the stored U.
+// The projection step of Algorithm 1: V = U^T X  (l x d), from the stored U.
 cudaError_t project(const void* U, const void* X, int64_t ldx, const Plan& p, void* V, const BasisWs& w,
                     uint32_t* status, cudaStream_t stream) {
   GemmDesc g;
@@ -351,14 +351,15 @@ cudaError_t compress_core(const loract_desc_t* desc, const void* X, int64_t ldx,
                           int32_t* idx_out, const CompressWs& w, const Plan& plan, cudaStream_t stream) {
   const bool bf16 = plan.bf16;
   const int r = desc->rank;
-  // line 1: sample rows, gather them.  The sampler is the first kernel of the call: it clears the status word
+  // the sampling step: sample rows, gather them.  The sampler is the first kernel of the call: it clears the status word
   // and writes the caller's copy of the indices itself.
   trace_label("sample");
   LORACT_CUDA_TRY(sample_indices_launch(desc->seed, desc->call_id, (uint32_t)desc->n_tokens, r, w.idx,
                                         w.status, stream, idx_out, true));
   trace_label("gather");
   LORACT_CUDA_TRY(gather_rows_launch(X, ldx, w.idx, r, desc->d, elem_bytes(desc), w.S, stream));
-  // Lines 2 to 7.  The test matrix (the sampled rows A_k at first, Q^T X in the power iterations of lines
+  // From the sketch to the orthonormal basis.  The test matrix (the sampled rows A_k at first, Q^T X in the power
+  // iterations of the loop
   // 3 to 6) is preconditioned before every product with X: with T T^T = L L^T, Omega = L^{-1} T has the row
   // space of T, so range(X Omega^T) = range(X T^T), but its rows are close to orthonormal, which keeps the
   // spectrum of the sketch from being squared (and, in the iterations, raised to the fourth power).
@@ -366,10 +367,10 @@ cudaError_t compress_core(const loract_desc_t* desc, const void* X, int64_t ldx,
     LORACT_CUDA_TRY(precondition_rows(w.S, r, desc->d, bf16, w.Omega, w.b, w.status, stream));
     // Y = X Omega^T, Y = QR (Q written to U)
     LORACT_CUDA_TRY(range_basis(X, ldx, plan, w.Omega, U, w.b, w.status, stream));
-    // lines 4 and 5 of the loop: the next test matrix is (X^T Q)^T = Q^T X, kept where A_k was
+    // inside the power-iteration loop: the next test matrix is (X^T Q)^T = Q^T X, kept where A_k was
     if (it < desc->power_iters) LORACT_CUDA_TRY(project(U, X, ldx, plan, w.S, w.b, w.status, stream));
   }
-  // line 8: V = U^T X
+  // the projection: V = U^T X
   return project(U, X, ldx, plan, V, w.b, w.status, stream);
 }
 

@@ -1,4 +1,4 @@
-// Tensor-core engine for the dense contractions of the path (Algorithm 1 lines 2 and 8, the Gram
+// Tensor-core engine for the dense contractions of the path (the sketch and the projection of Algorithm 1, the Gram
 // matrices of the orthonormalisation, the application of the triangular factors, Reconstruct).
 //
 // One kernel, written for sm_100a: TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) fills a

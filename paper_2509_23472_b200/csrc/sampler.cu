@@ -1,4 +1,4 @@
-// Row sampling (Algorithm 1, line 1), the row gather, and the Gaussian test matrix of the RSVD
+// Row sampling (the first step of Algorithm 1), the row gather, and the Gaussian test matrix of the RSVD
 // comparator.  The generator is Philox4x32-10 (Salmon et al., SC'11), written out here from the
 // published round function; it shares no code with the CPU oracle.
 #include "common.cuh"

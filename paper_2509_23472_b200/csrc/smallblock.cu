@@ -1,7 +1,7 @@
 // Orthonormalisation of the small (r x r) blocks of the decomposition: Cholesky factor of a Gram
 // matrix and the inverse of that factor, in one thread-block-cluster kernel.
 //
-// Algorithm 1 orthonormalises the tall sketch Y (line 7: Y = QR).  Here that is done through Gram
+// Algorithm 1 orthonormalises the tall sketch Y (its QR step, Y = QR).  Here that is done through Gram
 // matrices: with W = Y^T Y = L L^T, Q = Y L^{-T} has orthonormal columns.  The only serial work is on
 // the r x r matrix W, r <= 512, and this kernel does it: left-looking blocked Cholesky with panels of
 // 32 columns (the 32 x 32 diagonal block is factored by one warp in registers with shuffles, the

@@ -1,5 +1,5 @@
 // Small-block factorisation for r <= 256, fp32: Cholesky factor of an r x r Gram matrix and the inverse
-// of that factor (the serial part of the orthonormalisation, Algorithm 1 line 7 done through Gram
+// of that factor (the serial part of the orthonormalisation, the QR step of Algorithm 1 done through Gram
 // matrices), as one thread-block-cluster kernel whose working set never leaves shared memory.
 //
 // The matrix is cut into 32 x 32 blocks.  Eight CTAs form a cluster:

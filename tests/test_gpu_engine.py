@@ -1,4 +1,4 @@
-"""GPU tests of the tensor-core contraction behind Algorithm 1 lines 2 and 8, the Gram products and
+"""GPU tests of the tensor-core contraction behind the sketch and the projection of Algorithm 1, the Gram products and
 Reconstruct: C = sum_t A_t B_t with bf16 operands and fp32 accumulation, for every operand major, with
 ragged shapes, split-K partials and the bf16 hi/lo output -- in both forms of the kernel (one CTA per
 128-row tile, and a pair of CTAs per 256-row tile).  The reference is the definition, evaluated in float64

@@ -241,7 +241,7 @@ def test_rsvd_comparator_at_the_largest_test_matrix(dev):
     assert abs(e_gpu - e_orc) <= TOL_ERR["bf16"]
 
 
-# ------------------------------------------------------------------ power iterations (Algorithm 1, lines 3 to 6)
+# ------------------------------------------------------------------ power iterations (the loop of Algorithm 1)
 @pytest.mark.parametrize("t", [1, 2])
 def test_power_iterations_match_the_oracle_and_help_on_a_flat_spectrum(dev, t):
     # a slowly decaying spectrum with strong noise: the regime in which the loop of Algorithm 1 pays

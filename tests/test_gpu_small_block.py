@@ -1,4 +1,4 @@
-"""GPU tests of the small-block step of the orthonormalisation (Algorithm 1 line 7 through Gram matrices):
+"""GPU tests of the small-block step of the orthonormalisation (the QR step of Algorithm 1 through Gram matrices):
 from W = sum of partials, the inverse of the Cholesky factor of W + shift * mean(diag W) * I.
 
 Checked against the definition in float64 (numpy's Cholesky and inverse): the device's L^{-1} must be lower
