@@ -346,7 +346,8 @@ def read_device_status(ws: torch.Tensor) -> int:
 OUT_F32, OUT_BF16, OUT_SPLIT, OUT_F64 = 0, 1, 2, 3
 DEBUG_EXPORTS = ("loract_debug_gemm", "loract_debug_small_block", "loract_debug_set_pair_mode",
                  "loract_debug_last_cuda_error", "loract_debug_trace_begin", "loract_debug_trace_end",
-                 "loract_debug_wait_expiry", "loract_debug_project")
+                 "loract_debug_wait_expiry", "loract_debug_project", "loract_debug_gemm_halved",
+                 "loract_debug_reduce_sym")
 
 
 def _debug_lib():
@@ -356,6 +357,11 @@ def _debug_lib():
         l.loract_debug_gemm.restype = ctypes.c_int
         l.loract_debug_gemm.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(vp), i64, ctypes.POINTER(vp), i64,
                                         i32, i32, i32, i32, vp, vp, i64, i32, i64, i32, i32, vp, vp]
+        l.loract_debug_gemm_halved.restype = ctypes.c_int
+        l.loract_debug_gemm_halved.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(vp), i64, ctypes.POINTER(vp),
+                                               i64, i32, i32, i32, i32, i32, vp, vp, i64, i32, i64, i32, i32, vp, vp]
+        l.loract_debug_reduce_sym.restype = ctypes.c_int
+        l.loract_debug_reduce_sym.argtypes = [vp, i32, i64, i32, vp, vp]
         l.loract_debug_small_block.restype = ctypes.c_int
         l.loract_debug_small_block.argtypes = [i32, vp, i32, i32, i64, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp]
         l._debug_ready = True
@@ -364,9 +370,10 @@ def _debug_lib():
 
 def debug_gemm(A_terms, B_terms, M: int, N: int, K: int, a_mn: bool, b_mn: bool, out_mode: int = OUT_F32,
                engine: int = 1, splits: int = 1, acc64: bool = False, status: Optional[torch.Tensor] = None,
-               out: Optional[Tuple[torch.Tensor, Optional[torch.Tensor]]] = None):
+               out: Optional[Tuple[torch.Tensor, Optional[torch.Tensor]]] = None, halve_at_term: int = 0):
     """C = sum_t A_t B_t through one of the two contraction kernels.  Operands are 2-D row-major tensors
-    stored [M][K] / [K][M] (a_mn) and [N][K] / [K][N] (b_mn).  Returns C (or (hi, lo), or the partials)."""
+    stored [M][K] / [K][M] (a_mn) and [N][K] / [K][N] (b_mn).  Returns C (or (hi, lo), or the partials).
+    halve_at_term = h > 0: the sum of the terms before h is halved before term h is added."""
     l = _debug_lib()
     dev = A_terms[0].device
     nt = len(A_terms)
@@ -383,12 +390,23 @@ def debug_gemm(A_terms, B_terms, M: int, N: int, K: int, a_mn: bool, b_mn: bool,
         C0 = torch.zeros(M, N, dtype=torch.bfloat16, device=dev); C1 = None
     else:
         C0 = torch.zeros(M, N, dtype=torch.bfloat16, device=dev); C1 = torch.zeros_like(C0)
-    _check(l.loract_debug_gemm(M, N, K, int(a_mn), int(b_mn), PA, A_terms[0].stride(0), PB, B_terms[0].stride(0),
-                               tcode(A_terms[0]), tcode(B_terms[0]), nt, out_mode, _ptr(C0), _ptr(C1), N, splits,
-                               M * N, int(acc64), engine, _ptr(status), _stream(dev)), "loract_debug_gemm")
+    _check(l.loract_debug_gemm_halved(M, N, K, int(a_mn), int(b_mn), PA, A_terms[0].stride(0), PB,
+                                      B_terms[0].stride(0), tcode(A_terms[0]), tcode(B_terms[0]), nt, halve_at_term,
+                                      out_mode, _ptr(C0), _ptr(C1), N, splits, M * N, int(acc64), engine,
+                                      _ptr(status), _stream(dev)), "loract_debug_gemm")
     if out_mode in (OUT_F32, OUT_F64):
         return C0 if splits > 1 else C0[0]
     return C0 if C1 is None else (C0, C1)
+
+
+def debug_reduce_sym(partials: torch.Tensor) -> torch.Tensor:
+    """Test hook: S + S^T for S the sum of the (n_partials, r, r) fp32 tensor over its first index."""
+    l = _debug_lib()
+    n, r, _ = partials.shape
+    out = torch.empty(r, r, dtype=torch.float32, device=partials.device)
+    _check(l.loract_debug_reduce_sym(_ptr(partials), n, r * r, r, _ptr(out), _stream(partials.device)),
+           "loract_debug_reduce_sym")
+    return out
 
 
 def debug_wait_expiry(which: int, limit_ns: int, status: torch.Tensor) -> None:

@@ -187,8 +187,10 @@ cudaError_t simt_split_f32(GemmDesc g, int splits, float* partials, float* out, 
 
 constexpr double kL2KeepBytes = 48.0 * 1024 * 1024;   // of X, asked to stay in L2 between the two passes (about 20 MB do)
 constexpr int kReduceFirst = 8;    // partial count from which a separate, all-SM reduction pays
+// `sym`: the partials hold D = Yh^T Yh / 2 + Yh^T Yl (the two-term form of the tall Gram products); the matrix to
+// factor is D + D^T.
 cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs& w, uint32_t* status,
-                   cudaStream_t stream) {
+                   cudaStream_t stream, bool sym = false) {
   SmallBlockArgs a;
   a.r = l;
   a.scratch = w.sb_scratch;
@@ -196,7 +198,12 @@ cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs&
   if (bf16) {
     a.partials = w.gram_partials; a.partial_type = ELEM_F32; a.n_partials = n_partials;
     a.partial_stride = (int64_t)l * l;
-    if (l <= 256 && n_partials >= kReduceFirst) {
+    if (sym) {
+      // in place, into the first partial: a CTA of that kernel reads the two tiles it owns from every partial
+      // before it writes them, and no other CTA touches them (the scratch area is the factorisation's own)
+      LORACT_CUDA_TRY(reduce_sym_launch(w.gram_partials, n_partials, a.partial_stride, l, w.gram_partials, stream));
+      a.n_partials = 1;
+    } else if (l <= 256 && n_partials >= kReduceFirst) {
       // The factorisation runs on eight SMs; summing many partials there is a read of several MB through
       // eight SMs' worth of bandwidth.  All SMs sum them first (same order of additions, so the same bits).
       float* W = (float*)w.sb_scratch;
@@ -271,8 +278,11 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
       g.a_type = g.b_type = el;
       g.ldc = l;
       if (p.bf16) {
-        g.n_terms = 3;
-        g.terms[0] = {Yh, Yh}; g.terms[1] = {Yh, Yl}; g.terms[2] = {Yl, Yh};
+        // D = Yh^T Yh / 2 + Yh^T Yl: the sum of the partials, added to its transpose before the factorisation,
+        // is Yh^T Yh + Yh^T Yl + Yl^T Yh (the product of the two low parts is below fp32 rounding)
+        g.n_terms = 2;
+        g.terms[0] = {Yh, Yh}; g.terms[1] = {Yh, Yl};
+        g.halve_at_term = 1;
         g.out = OUT_F32; g.C0 = w.gram_partials; g.splits = w.splits_gram; g.split_stride = (int64_t)l * l;
       } else {
         g.terms[0] = {Yh, Yh};
@@ -283,7 +293,7 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
       LORACT_CUDA_TRY(run_gemm(g, status, stream));
     }
     trace_label(round ? "small block 3" : "small block 2");
-    LORACT_CUDA_TRY(factor(l, p.bf16, w.splits_gram, round ? kShiftSecond : kShiftFirst, w, status, stream));
+    LORACT_CUDA_TRY(factor(l, p.bf16, w.splits_gram, round ? kShiftSecond : kShiftFirst, w, status, stream, p.bf16));
     {  // Y <- Y L^{-T}:  C[m][j] = sum_k Y[m][k] Linv[j][k]
       GemmDesc g;
       g.M = n; g.N = l; g.K = l; g.lda = l; g.ldb = l; g.a_type = g.b_type = el;
@@ -425,13 +435,15 @@ cudaError_t gram_tall_sum(const void* Yh, const void* Yl, int n, int l, const Ba
                           cudaStream_t stream) {
   GemmDesc g;
   g.M = l; g.N = l; g.K = n; g.a_mn = true; g.b_mn = true; g.lda = l; g.ldb = l;
-  g.n_terms = 3;
-  g.terms[0] = {Yh, Yh}; g.terms[1] = {Yh, Yl}; g.terms[2] = {Yl, Yh};
+  // two terms, the first halved: the partials sum to D with D + D^T = Yh^T Yh + Yh^T Yl + Yl^T Yh
+  g.n_terms = 2;
+  g.terms[0] = {Yh, Yh}; g.terms[1] = {Yh, Yl};
+  g.halve_at_term = 1;
   g.out = OUT_F32; g.ldc = l;
-  if (w.splits_gram <= 1) { g.C0 = W; return run_gemm(g, status, stream); }
-  g.C0 = w.gram_partials; g.splits = w.splits_gram; g.split_stride = (int64_t)l * l;
+  const int splits = w.splits_gram < 1 ? 1 : w.splits_gram;
+  g.C0 = w.gram_partials; g.splits = splits; g.split_stride = (int64_t)l * l;
   LORACT_CUDA_TRY(run_gemm(g, status, stream));
-  return reduce_partials_launch(w.gram_partials, w.splits_gram, g.split_stride, g.split_stride, W, nullptr, stream);
+  return reduce_sym_launch(w.gram_partials, splits, g.split_stride, l, W, stream);
 }
 
 // L^-1 (bf16 pair in w.Lh / w.Ll) from one summed l x l Gram matrix.
@@ -889,13 +901,31 @@ loract_status_t loract_debug_gemm(int32_t M, int32_t N, int32_t K, int32_t a_mn,
                                   int32_t a_type, int32_t b_type, int32_t n_terms, int32_t out_mode, void* C0,
                                   void* C1, int64_t ldc, int32_t splits, int64_t split_stride, int32_t acc64,
                                   int32_t engine, uint32_t* status_word, void* stream) {
+  return loract_debug_gemm_halved(M, N, K, a_mn, b_mn, A, lda, B, ldb, a_type, b_type, n_terms, 0, out_mode, C0, C1,
+                                  ldc, splits, split_stride, acc64, engine, status_word, stream);
+}
+
+loract_status_t loract_debug_reduce_sym(const float* partials, int32_t n_partials, int64_t stride, int32_t r,
+                                        float* out, void* stream) {
+  if (!partials || !out || n_partials < 1 || r < 1) return LORACT_ERR_INVALID_ARG;
+  return from_cuda(reduce_sym_launch(partials, n_partials, stride, r, out, (cudaStream_t)stream));
+}
+
+loract_status_t loract_debug_gemm_halved(int32_t M, int32_t N, int32_t K, int32_t a_mn, int32_t b_mn,
+                                         const void* const* A, int64_t lda, const void* const* B, int64_t ldb,
+                                         int32_t a_type, int32_t b_type, int32_t n_terms, int32_t halve_at_term,
+                                         int32_t out_mode, void* C0, void* C1, int64_t ldc, int32_t splits,
+                                         int64_t split_stride, int32_t acc64, int32_t engine, uint32_t* status_word,
+                                         void* stream) {
   if (!A || !B || !C0 || n_terms < 1 || n_terms > 3 || M < 1 || N < 1 || K < 1) return LORACT_ERR_INVALID_ARG;
+  if (halve_at_term < 0 || halve_at_term >= n_terms) return LORACT_ERR_INVALID_ARG;
   GemmDesc g;
   g.M = M; g.N = N; g.K = K; g.a_mn = a_mn != 0; g.b_mn = b_mn != 0; g.lda = lda; g.ldb = ldb;
   g.a_type = a_type; g.b_type = b_type; g.n_terms = n_terms;
   for (int t = 0; t < n_terms; ++t) g.terms[t] = {A[t], B[t]};
   g.out = out_mode; g.C0 = C0; g.C1 = C1; g.ldc = ldc; g.splits = splits < 1 ? 1 : splits;
   g.split_stride = split_stride; g.acc64 = acc64 != 0;
+  g.halve_at_term = halve_at_term;
   if (engine == 1) {
     if (!gemm_tc_supported(g)) return LORACT_ERR_UNSUPPORTED;
     return from_cuda(gemm_tc_launch(g, status_word, (cudaStream_t)stream));

@@ -103,6 +103,10 @@ struct GemmDesc {
   // Two-CTA kernel, K-major A: loads of A from this K element on ask L2 to evict them last (a later kernel
   // reads the same bytes again); negative: no hint.
   int64_t a_keep_from_k = -1;
+  // The sum of the terms before this one is multiplied by 1/2 before this term's products are added
+  // (result = (t_0 + ... + t_{h-1}) / 2 + t_h + ...); 0 or negative: plain sum.  With the pair {A^T A, A^T B} and
+  // h = 1 the result D gives D + D^T = A^T A + A^T B + B^T A: a symmetric three-term sum for two terms' work.
+  int halve_at_term = 0;
 };
 
 // tcgen05 engine: bf16 operands, fp32 accumulation in tensor memory.  Returns cudaErrorNotSupported
@@ -186,6 +190,9 @@ cudaError_t split_block_launch(const float* src, int rows, int cols, int64_t ld,
 cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_t stride,
                                    int64_t count, float* out_f32, __nv_bfloat16* out_bf16,
                                    cudaStream_t stream);
+// out (r x r) = S + S^T, S the fixed-order sum of the partials (each r x r, leading dimension r).
+cudaError_t reduce_sym_launch(const float* partials, int n_partials, int64_t stride, int r, float* out,
+                              cudaStream_t stream);
 // out = sum_s partials[s] as a bf16 triple hi + mid + lo (rows x cols, leading dimensions ld_in / ld_out).
 cudaError_t reduce_split3_launch(const float* partials, int n_partials, int64_t stride, int rows, int cols,
                                  int64_t ld_in, int64_t ld_out, __nv_bfloat16* hi, __nv_bfloat16* mid,

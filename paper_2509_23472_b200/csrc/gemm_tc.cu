@@ -64,6 +64,7 @@ struct TcParams {
   int st_units;       // streaming kernel: tiles in all (column tile major, then M)
   int st_stages;      // streaming kernel: stages of the A ring (<= kStreamStages)
   int store_bufs;     // staging boxes per epilogue warp (1 or 2)
+  int halve_at_term;  // the accumulator is multiplied by 1/2 before the first product of this term (0: never)
   int a_keep_from_kb; // two-CTA kernel: K block from which the loads of A carry an evict-last hint (kb_total: none)
 };
 
@@ -131,6 +132,15 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The same instruction with the accumulator read as D / 2 (scale-input-d = 1): D = A B + D * 2^-1.
+__device__ __forceinline__ void tc_mma_bf16_halved(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, 1, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p, 1;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
       : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t v[32]) {
@@ -568,6 +578,7 @@ gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
                              ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(p.bn >> 3) << 17) |
                              ((uint32_t)(kBM >> 4) << 24);
       bool ok = true;
+      const int halve_it = p.halve_at_term > 0 ? p.halve_at_term * kb_count : -1;
       for (int it = 0; it < n_iter && ok; ++it) {
         const int s = it % kStages;
         ok = mbar_wait_bounded(&full_bar[s], (it / kStages) & 1, &abort_flag);
@@ -582,7 +593,8 @@ gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
           // 16 elements along K: 32 bytes inside the swizzled row (K-major) or 16 rows (MN-major)
           const uint64_t a_k = a_desc + (uint64_t)((A_MN ? 2048u : 32u) >> 4) * k;
           const uint64_t b_k = b_desc + (uint64_t)((B_MN ? 2048u : 32u) >> 4) * k;
-          tc_mma_bf16(tmem_base, a_k, b_k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+          if (k == 0 && it == halve_it) tc_mma_bf16_halved(tmem_base, a_k, b_k, idesc);
+          else tc_mma_bf16(tmem_base, a_k, b_k, idesc, (it > 0 || k > 0) ? 1u : 0u);
         }
         tc_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
       }
@@ -654,6 +666,15 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair_halved(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                                        uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, 1, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p, 1;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
       : "memory");
 }
 
@@ -756,6 +777,7 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
       const uint64_t a_desc0 = make_smem_desc(smem_u32(tiles), A_MN);
       const uint64_t b_desc0 = make_smem_desc(smem_u32(tiles) + kABytes, B_MN);
       const uint32_t stage_units = stage_bytes >> 4;
+      const int halve_it = p.halve_at_term > 0 ? p.halve_at_term * kb_count : -1;
       for (int it = 0; it < n_iter && ok; ++it) {
         ok = mbar_wait_bounded(&full_bar[s], parity, &abort_flag);
         if (!ok) break;
@@ -766,7 +788,8 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
         for (int k = 0; k < kBK / 16; ++k) {
           const uint64_t a_k = a_desc + (uint64_t)((A_MN ? 2048u : 32u) >> 4) * k;
           const uint64_t b_k = b_desc + (uint64_t)((B_MN ? 2048u : 32u) >> 4) * k;
-          tc_mma_bf16_pair(tmem_base, a_k, b_k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+          if (k == 0 && it == halve_it) tc_mma_bf16_pair_halved(tmem_base, a_k, b_k, idesc);
+          else tc_mma_bf16_pair(tmem_base, a_k, b_k, idesc, (it > 0 || k > 0) ? 1u : 0u);
         }
         tc_commit_pair(&empty_bar[s]);   // frees the stage in both CTAs once these MMAs have read it
         if (++s == kPairStages) { s = 0; parity ^= 1u; }
@@ -1219,6 +1242,7 @@ bool gemm_tc_supported(const GemmDesc& g) {
   if (g.out == OUT_ACT_BWD && (!g.ep_E || g.splits > 1 || g.ep_kind < 0 || g.ep_kind > 1)) return false;
   if (g.out == OUT_RMS_BWD && (!g.ep_E || !g.ep_row_a || !g.ep_row_b || !g.ep_col || g.splits > 1)) return false;
   if (g.M < 1 || g.N < 1 || g.K < 1 || g.n_terms < 1 || g.n_terms > 3) return false;
+  if (g.halve_at_term >= g.n_terms) return false;
   if (g.lda % 8 || g.ldb % 8) return false;
   if (g.splits > 1 && g.out != OUT_F32) return false;
   if (g.alpha != 1.0f) return false;
@@ -1259,6 +1283,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   p.ep_kind = g.ep_kind;
   p.dev_status = dev_status;
   p.st_m_tiles = 0; p.st_units = 0; p.tma_store = 0; p.st_stages = kStreamStages; p.store_bufs = kStoreBufs;
+  p.halve_at_term = g.halve_at_term > 0 ? g.halve_at_term : 0;
   p.a_keep_from_kb = g.a_keep_from_k >= 0 ? (int)(g.a_keep_from_k / kBK) : p.kb_total;
 
   TmapPack maps;

@@ -27,6 +27,7 @@ struct SimtParams {
   int64_t split_stride;
   int accumulate;
   float alpha;
+  int halve_at_term;  // the sum so far is multiplied by 1/2 before this term (0: never)
 };
 
 constexpr int kTile = 64;   // output tile 64 x 64, 256 threads, 4 x 4 outputs per thread
@@ -55,6 +56,12 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(SimtParams p) {
   for (int term = 0; term < p.n_terms; ++term) {
     const TA* A = (const TA*)p.A[term];
     const TB* B = (const TB*)p.B[term];
+    if (term > 0 && term == p.halve_at_term) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] *= (TAcc)0.5;
+    }
     float ra[4], rb[4];
     auto fetch = [&](int k0) {
 #pragma unroll
@@ -137,6 +144,47 @@ __global__ void reduce_partials_kernel(const float* __restrict__ partials, int n
     for (int q = 0; q < n_partials; ++q) s += partials[(int64_t)q * stride + i];
     if (out_f32) out_f32[i] = s;
     if (out_bf16) out_bf16[i] = __float2bfloat16(s);
+  }
+}
+
+// out = S + S^T with S = sum_s partials[s] (fixed order), for r x r matrices: the tall Gram products are formed as
+// D = Yh^T Yh / 2 + Yh^T Yl (two terms), and D + D^T = Yh^T Yh + Yh^T Yl + Yl^T Yh is the three-term Gram matrix,
+// exactly symmetric.  One CTA per pair of 16 x 16 tiles (I, J), (J, I), I >= J: both tiles are summed with
+// coalesced row reads and meet through shared memory.
+constexpr int kSymTile = 16;
+// `out` may be the first partial (no __restrict__: see the caller).  1024 threads: two tiles x two halves of the
+// partials x 256 elements; a thread adds its partials eight at a time into eight running sums (eight independent
+// loads in flight); the sums are combined in a fixed order.
+__global__ void __launch_bounds__(1024) reduce_sym_kernel(const float* partials, int n_partials, int64_t stride, int r,
+                                                          float* out) {
+  __shared__ float t[2][2][kSymTile][kSymTile + 1];   // [tile][half of the partials][row][column]
+  // tile pair from the linear block index: I = largest with I (I + 1) / 2 <= b
+  const int b = blockIdx.x;
+  int I = 0;
+  while ((I + 1) * (I + 2) / 2 <= b) ++I;
+  const int J = b - I * (I + 1) / 2;
+  const int qh = threadIdx.x >> 9, tile = (threadIdx.x >> 8) & 1;
+  const int a = (threadIdx.x >> 4) & 15, c = threadIdx.x & 15;
+  // element (a, c) of tile (I, J) (tile 0) or of tile (J, I) (tile 1)
+  const int row = (tile ? J : I) * kSymTile + a, col = (tile ? I : J) * kSymTile + c;
+  pdl_wait();
+  pdl_launch_dependents();
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (row < r && col < r && !(tile == 1 && I == J)) {
+    const float* src = partials + (int64_t)row * r + col;
+    const int q_end = qh ? n_partials : n_partials / 2;
+    int q = qh ? n_partials / 2 : 0;
+    for (; q + 8 <= q_end; q += 8) {
+#pragma unroll
+      for (int u = 0; u < 8; ++u) acc[u] += src[(int64_t)(q + u) * stride];
+    }
+    for (int u = 0; q + u < q_end; ++u) acc[u] += src[(int64_t)(q + u) * stride];
+  }
+  t[tile][qh][a][c] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) + ((acc[4] + acc[5]) + (acc[6] + acc[7]));
+  __syncthreads();
+  if (qh == 0 && row < r && col < r && !(tile == 1 && I == J)) {
+    const int other = (I == J) ? 0 : 1 - tile;
+    out[(int64_t)row * r + col] = (t[tile][0][a][c] + t[tile][1][a][c]) + (t[other][0][c][a] + t[other][1][c][a]);
   }
 }
 
@@ -472,6 +520,7 @@ cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t stream) {
   p.split_stride = g.split_stride;
   p.accumulate = g.accumulate ? 1 : 0;
   p.alpha = g.alpha;
+  p.halve_at_term = g.halve_at_term > 0 ? g.halve_at_term : 0;
   if (p.splits > 1 && !(g.out == OUT_F32 || g.out == OUT_F64)) return cudaErrorInvalidValue;
   const bool a16 = g.a_type == ELEM_BF16, b16 = g.b_type == ELEM_BF16;
   if (a16 && b16) return launch_simt_typed<__nv_bfloat16, __nv_bfloat16>(p, g.acc64, stream);
@@ -488,6 +537,15 @@ cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_
   if (grid < 1) grid = 1;
   LORACT_CUDA_TRY(launch_pdl(reduce_partials_kernel, dim3(grid), dim3(256), 0, stream, partials, n_partials, stride,
                              count, out_f32, out_bf16));
+  count_launch(__func__, stream);
+  return cudaGetLastError();
+}
+
+cudaError_t reduce_sym_launch(const float* partials, int n_partials, int64_t stride, int r, float* out,
+                              cudaStream_t stream) {
+  const int nt = (r + kSymTile - 1) / kSymTile;
+  LORACT_CUDA_TRY(launch_pdl(reduce_sym_kernel, dim3(nt * (nt + 1) / 2), dim3(1024), 0, stream, partials, n_partials,
+                             stride, r, out));
   count_launch(__func__, stream);
   return cudaGetLastError();
 }

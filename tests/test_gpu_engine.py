@@ -150,3 +150,44 @@ def test_terms_that_share_operands(dev, a_mn, b_mn, M, N, K, splits, pattern):
     scale = float(ref.abs().max())
     assert float((out[True] - ref).abs().max()) <= 1e-4 * scale
     assert float((out[True] - out[False]).abs().max()) <= 1e-5 * scale
+
+
+@pytest.mark.parametrize("engine", [0, 1])
+@pytest.mark.parametrize("pair", [False, True])
+@pytest.mark.parametrize("r,n,splits,halve", [(256, 4096, 8, 1), (96, 1000, 3, 1), (256, 2048, 1, 2), (128, 520, 2, 1)])
+def test_halved_accumulator_and_the_symmetric_gram_matrix_it_is_for(dev, engine, pair, r, n, splits, halve):
+    # C = (t_0 + ... + t_{h-1}) / 2 + t_h + ...: checked against that definition in float64, for both kernels
+    # (and split over K: every split halves its own partial sum).  Then the use it is made for: with the
+    # pair {Yh^T Yh, Yh^T Yl} the partial sums D give D + D^T = Yh^T Yh + Yh^T Yl + Yl^T Yh, the three-term
+    # Gram matrix of Y = Yh + Yl, exactly symmetric.
+    if engine == 0 and pair:
+        pytest.skip("the CUDA-core kernel has one form")
+    B.debug_set_pair_mode(pair)
+    g = torch.Generator(device=dev)
+    g.manual_seed(r + n)
+    Y = torch.randn(n, r, generator=g, device=dev)
+    Yh = Y.bfloat16()
+    Yl = (Y - Yh.float()).bfloat16()
+    Z = torch.randn(n, r, generator=g, device=dev).bfloat16()
+    terms_a, terms_b = ([Yh, Yh], [Yh, Yl]) if halve == 1 else ([Yh, Z, Yh], [Yh, Yh, Yl])
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    C = B.debug_gemm(terms_a, terms_b, r, r, n, True, True, out_mode=B.OUT_F32, engine=engine, splits=splits,
+                     status=status, halve_at_term=halve)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    parts = C if splits > 1 else C[None]
+    prods = [a.double().t() @ b.double() for a, b in zip(terms_a, terms_b)]
+    ref = sum(prods[:halve]) / 2 + sum(prods[halve:])
+    scale = float(ref.abs().max())
+    assert float((parts.double().sum(0) - ref).abs().max()) <= 2e-5 * scale * max(1.0, (n / 64) ** 0.5)
+    if halve == 1:
+        W = B.debug_reduce_sym(parts.contiguous())
+        torch.cuda.synchronize()
+        assert torch.equal(W, W.t())
+        S = parts.sum(0)                     # the kernel adds the partials in index order, as torch does here
+        assert torch.equal(W, S + S.t()) or float((W - (S + S.t())).abs().max()) <= 1e-6 * scale
+        gram = Yh.double().t() @ Yh.double() + Yh.double().t() @ Yl.double() + Yl.double().t() @ Yh.double()
+        assert float((W.double() - gram).abs().max()) <= 4e-5 * scale * max(1.0, (n / 64) ** 0.5)
+        full = (Yh.double() + Yl.double()).t() @ (Yh.double() + Yl.double())
+        assert float((W.double() - full).abs().max()) <= 6e-5 * scale * max(1.0, (n / 64) ** 0.5)
+    B.debug_set_pair_mode(True)
