@@ -53,6 +53,14 @@ loract_status_t loract_debug_project(const loract_desc_t* desc, const void* U, c
  * that a test can compare the two; on = 1 (the default) restores the choice by shape.  Process-wide. */
 void loract_debug_set_pair_mode(int32_t on);
 
+/* The orthonormalisation of the bf16 path runs its second Gram round only when the first round's Gram matrix W
+ * was not conditioned well enough for one: a one-CTA kernel forms est = trace((D W D)^-1), D = diag(W)^(-1/2),
+ * from the inverse factor and compares it with a threshold (ranks up to 256; above that both rounds always run).
+ * This sets the threshold, process-wide: a negative value forces both rounds, +infinity allows one round whenever
+ * no status bit is set, 0 restores the default.  After a call the status block at the head of the workspace
+ * holds, as 32-bit words 4, 5, 6: whether the second round ran (0 / 1), est (float bits), the number of rounds. */
+void loract_debug_set_round_gate(float threshold);
+
 /* Stage trace.  Between trace_begin and trace_end every kernel the library launches on `stream` is followed by
  * a CUDA event; trace_end synchronises the stream and writes, per kernel in launch order, a label (64 bytes
  * each, zero-terminated: the step of the path and the kernel's launch function) and the time from the

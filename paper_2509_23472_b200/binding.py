@@ -347,7 +347,7 @@ OUT_F32, OUT_BF16, OUT_SPLIT, OUT_F64 = 0, 1, 2, 3
 DEBUG_EXPORTS = ("loract_debug_gemm", "loract_debug_small_block", "loract_debug_set_pair_mode",
                  "loract_debug_last_cuda_error", "loract_debug_trace_begin", "loract_debug_trace_end",
                  "loract_debug_wait_expiry", "loract_debug_project", "loract_debug_gemm_halved",
-                 "loract_debug_reduce_sym")
+                 "loract_debug_reduce_sym", "loract_debug_set_round_gate")
 
 
 def _debug_lib():
@@ -434,6 +434,21 @@ def debug_set_pair_mode(on: bool) -> None:
     l.loract_debug_set_pair_mode.restype = None
     l.loract_debug_set_pair_mode.argtypes = [ctypes.c_int32]
     l.loract_debug_set_pair_mode(1 if on else 0)
+
+
+def debug_set_round_gate(threshold: float) -> None:
+    """Test hook: threshold of the device-side decision to run the second orthonormalisation round (negative: always
+    two rounds; inf: one round unless a status bit is set; 0: the default)."""
+    l = _debug_lib()
+    l.loract_debug_set_round_gate.restype = None
+    l.loract_debug_set_round_gate.argtypes = [ctypes.c_float]
+    l.loract_debug_set_round_gate(float(threshold))
+
+
+def round_gate_words(ws: torch.Tensor):
+    """(second round ran, estimate trace((D W D)^-1), rounds) of the last orthonormalisation run on workspace `ws`."""
+    w = ws[16:28].cpu()
+    return int(w[0:4].view(torch.int32).item()), float(w[4:8].view(torch.float32).item()), int(w[8:12].view(torch.int32).item())
 
 
 def debug_trace_begin(device) -> None:

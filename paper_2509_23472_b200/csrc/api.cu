@@ -61,8 +61,19 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // relative diagonal shifts of the three Cholesky factorisations (fp32 small blocks)
 constexpr float kShiftSample = 1e-6f;  // Gram of the sampled rows
-constexpr float kShiftFirst = 3e-6f;   // first Gram of the sketch
-constexpr float kShiftSecond = 1e-7f;  // second Gram (already close to the identity)
+// first Gram of the sketch: relative to each diagonal entry itself (W_ii <- W_ii (1 + s)).  The columns of the sketch
+// differ in norm by two orders of magnitude and more; a shift relative to the mean diagonal would be of the size of
+// the small diagonal entries and leave an orthogonality defect of order one, the entry-relative shift leaves the
+// factorisation as accurate as that of the diagonally scaled matrix, whose condition number is a thousand times lower.
+constexpr float kShiftFirstDiag = 2e-7f;
+constexpr float kShiftFirstMean = 3e-6f;  // fp32 inputs (fp64 factorisation): relative to the mean diagonal
+constexpr int kGateWord = 4;               // words 4..6 of the status block: gate, estimate, rounds
+constexpr float kShiftSecond = 1e-7f;  // second Gram (already close to the identity), relative to the mean diagonal
+// Second orthonormalisation round: run only when trace((D W D)^-1) of the first round's Gram matrix exceeds this
+// (D = diag(W)^(-1/2)), or when a status bit is set.  The defect of one round is the rounding error of the fp32 Gram
+// matrix (a few 1e-9 of sqrt(W_ii W_jj) per entry) times that trace.
+constexpr float kRoundGateDefault = 3.0e4f;
+std::atomic<float> g_round_gate{kRoundGateDefault};
 
 struct Carver {
   unsigned char* base;
@@ -108,7 +119,10 @@ Plan make_plan(int64_t n, int64_t d, int l, bool bf16) {
   p.n = n; p.d = d; p.l = l; p.bf16 = bf16;
   if (bf16) {
     p.splits_gs = gemm_tc_pick_splits(l, l, (int)d, false, false);
-    p.splits_w = gemm_tc_pick_splits(l, l, (int)n, true, true);
+    // The tensor cores add every product into the fp32 accumulator with truncation, so a Gram matrix loses about
+    // half an ulp per instruction of the chain, with one sign on the diagonal; short chains (up to 64 partial sums,
+    // added with rounding afterwards) keep that bias below what one orthonormalisation round tolerates.
+    p.splits_w = gemm_tc_pick_splits(l, l, (int)n, true, true, 64);
     p.splits_v = gemm_tc_pick_splits(l, (int)d, (int)n, true, true);
   } else {
     // CUDA-core path: the generic kernel walks K sixteen elements at a time, so a long contraction with few output
@@ -190,9 +204,11 @@ constexpr int kReduceFirst = 8;    // partial count from which a separate, all-S
 // `sym`: the partials hold D = Yh^T Yh / 2 + Yh^T Yl (the two-term form of the tall Gram products); the matrix to
 // factor is D + D^T.
 cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs& w, uint32_t* status,
-                   cudaStream_t stream, bool sym = false) {
+                   cudaStream_t stream, bool sym = false, float shift_diag = 0.f, const uint32_t* gate = nullptr) {
   SmallBlockArgs a;
   a.r = l;
+  a.shift_diag_rel = shift_diag;
+  a.gate = gate;
   a.scratch = w.sb_scratch;
   a.dev_status = status;
   if (bf16) {
@@ -201,7 +217,7 @@ cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs&
     if (sym) {
       // in place, into the first partial: a CTA of that kernel reads the two tiles it owns from every partial
       // before it writes them, and no other CTA touches them (the scratch area is the factorisation's own)
-      LORACT_CUDA_TRY(reduce_sym_launch(w.gram_partials, n_partials, a.partial_stride, l, w.gram_partials, stream));
+      LORACT_CUDA_TRY(reduce_sym_launch(w.gram_partials, n_partials, a.partial_stride, l, w.gram_partials, stream, gate));
       a.n_partials = 1;
     } else if (l <= 256 && n_partials >= kReduceFirst) {
       // The factorisation runs on eight SMs; summing many partials there is a read of several MB through
@@ -269,45 +285,99 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
       LORACT_CUDA_TRY(simt_split_f32(g, simt_splits(p.d), w.part32, w.Y32, stream));
     }
   }
-  for (int round = 0; round < 2; ++round) {
-    const void* Yh = p.bf16 ? (const void*)(round ? w.Qh : w.Yh) : (const void*)(round ? w.Q32 : w.Y32);
-    const void* Yl = round ? w.Ql : w.Yl;
-    {  // W = Y^T Y
-      GemmDesc g;
-      g.M = l; g.N = l; g.K = n; g.a_mn = true; g.b_mn = true; g.lda = l; g.ldb = l;
-      g.a_type = g.b_type = el;
-      g.ldc = l;
-      if (p.bf16) {
-        // D = Yh^T Yh / 2 + Yh^T Yl: the sum of the partials, added to its transpose before the factorisation,
-        // is Yh^T Yh + Yh^T Yl + Yl^T Yh (the product of the two low parts is below fp32 rounding)
-        g.n_terms = 2;
-        g.terms[0] = {Yh, Yh}; g.terms[1] = {Yh, Yl};
-        g.halve_at_term = 1;
-        g.out = OUT_F32; g.C0 = w.gram_partials; g.splits = w.splits_gram; g.split_stride = (int64_t)l * l;
-      } else {
-        g.terms[0] = {Yh, Yh};
+  if (!p.bf16) {
+    for (int round = 0; round < 2; ++round) {
+      const void* Yc = round ? w.Q32 : w.Y32;
+      {  // W = Y^T Y
+        GemmDesc g;
+        g.M = l; g.N = l; g.K = n; g.a_mn = true; g.b_mn = true; g.lda = l; g.ldb = l;
+        g.a_type = g.b_type = el;
+        g.ldc = l;
+        g.terms[0] = {Yc, Yc};
         g.out = OUT_F64; g.C0 = w.gram64; g.acc64 = true;
         g.splits = w.splits_gram; g.split_stride = (int64_t)l * l;
+        trace_label(round ? "Gram 2" : "Gram 1");
+        LORACT_CUDA_TRY(run_gemm(g, status, stream));
       }
-      trace_label(round ? "Gram 2" : "Gram 1");
-      LORACT_CUDA_TRY(run_gemm(g, status, stream));
-    }
-    trace_label(round ? "small block 3" : "small block 2");
-    LORACT_CUDA_TRY(factor(l, p.bf16, w.splits_gram, round ? kShiftSecond : kShiftFirst, w, status, stream, p.bf16));
-    {  // Y <- Y L^{-T}:  C[m][j] = sum_k Y[m][k] Linv[j][k]
-      GemmDesc g;
-      g.M = n; g.N = l; g.K = l; g.lda = l; g.ldb = l; g.a_type = g.b_type = el;
-      g.ldc = l;
-      if (p.bf16) {
-        g.n_terms = 3;
-        g.terms[0] = {Yh, w.Lh}; g.terms[1] = {Yh, w.Ll}; g.terms[2] = {Yl, w.Lh};
-        if (round == 0) { g.out = OUT_SPLIT; g.C0 = w.Qh; g.C1 = w.Ql; } else { g.out = OUT_BF16; g.C0 = U; }
-      } else {
-        g.terms[0] = {Yh, w.Linv32};
+      trace_label(round ? "small block 3" : "small block 2");
+      LORACT_CUDA_TRY(factor(l, false, w.splits_gram, round ? kShiftSecond : kShiftFirstMean, w, status, stream, false));
+      {  // Y <- Y L^{-T}:  C[m][j] = sum_k Y[m][k] Linv[j][k]
+        GemmDesc g;
+        g.M = n; g.N = l; g.K = l; g.lda = l; g.ldb = l; g.a_type = g.b_type = el;
+        g.ldc = l;
+        g.terms[0] = {Yc, w.Linv32};
         g.out = OUT_F32; g.C0 = round == 0 ? (void*)w.Q32 : U;
+        trace_label(round ? "apply L^-T 2" : "apply L^-T 1");
+        LORACT_CUDA_TRY(run_gemm(g, status, stream));
       }
-      trace_label(round ? "apply L^-T 2" : "apply L^-T 1");
-      LORACT_CUDA_TRY(run_gemm(g, status, stream));
+    }
+    return cudaSuccess;
+  }
+  // bf16 inputs.  Round 1 always runs and writes the leading bf16 part of Q1 = Y L^-T straight into U (the rounded Q1
+  // is the result when one round is enough), the remainder into the workspace.  A one-CTA kernel then decides from the
+  // factor whether the Gram matrix was conditioned well enough for one round (gate word: 0 = done).  The kernels of
+  // round 2 are launched in any case and leave at once when the gate word is zero: no host synchronisation.
+  uint32_t* gate_words = status + kGateWord;
+  const bool can_gate = l <= 256 && l % 8 == 0;   // the block scheme above 256 columns always runs both rounds
+  const uint32_t* gate = can_gate ? gate_words : nullptr;
+  auto gram = [&](const void* Yh, const void* Yl, const uint32_t* gt) {
+    // D = (Yl^T Yl + Yh^T Yh) / 2 + Yh^T Yl: the sum of the partials, added to its transpose before the factorisation,
+    // is (Yh + Yl)^T (Yh + Yl) with every product kept.  The product of the two low parts is 2^-18 of the diagonal
+    // and always positive: left out, it biases every pivot by more than fp32 rounding does.  It goes first, while
+    // the accumulator is still small (every instruction truncates the running sum once).
+    GemmDesc g;
+    g.M = l; g.N = l; g.K = n; g.a_mn = true; g.b_mn = true; g.lda = l; g.ldb = l;
+    g.a_type = g.b_type = el;
+    g.ldc = l;
+    g.n_terms = 3;
+    g.terms[0] = {Yl, Yl}; g.terms[1] = {Yh, Yh}; g.terms[2] = {Yh, Yl};
+    g.halve_at_term = 2;
+    g.out = OUT_F32; g.C0 = w.gram_partials; g.splits = w.splits_gram; g.split_stride = (int64_t)l * l;
+    g.gate = gt;
+    return run_gemm(g, status, stream);
+  };
+  auto apply = [&](const void* Yh, const void* Yl, void* Ch, void* Cl, const uint32_t* gt) {
+    // C[m][j] = sum_k Y[m][k] Linv[j][k]
+    GemmDesc g;
+    g.M = n; g.N = l; g.K = l; g.lda = l; g.ldb = l; g.a_type = g.b_type = el;
+    g.ldc = l;
+    g.n_terms = 3;
+    g.terms[0] = {Yh, w.Lh}; g.terms[1] = {Yh, w.Ll}; g.terms[2] = {Yl, w.Lh};
+    if (Cl) { g.out = OUT_SPLIT; g.C0 = Ch; g.C1 = Cl; } else { g.out = OUT_BF16; g.C0 = Ch; }
+    g.gate = gt;
+    return run_gemm(g, status, stream);
+  };
+  trace_label("Gram 1");
+  LORACT_CUDA_TRY(gram(w.Yh, w.Yl, nullptr));
+  trace_label("small block 2");
+  // (widths above 512 take the general fp64 kernel, which knows the shift relative to the mean diagonal only)
+  LORACT_CUDA_TRY(factor(l, true, w.splits_gram, l <= 512 ? 0.f : kShiftFirstMean, w, status, stream, true,
+                         l <= 512 ? kShiftFirstDiag : 0.f));
+  trace_label("round gate");
+  LORACT_CUDA_TRY(round_gate_launch(w.gram_partials, w.Lh, l, can_gate ? g_round_gate.load() : -1.f, status, gate_words,
+                                    stream));
+  trace_label("apply L^-T 1");
+  LORACT_CUDA_TRY(apply(w.Yh, w.Yl, U, w.Ql, nullptr));
+  trace_label("Gram 2");
+  LORACT_CUDA_TRY(gram(U, w.Ql, gate));
+  trace_label("small block 3");
+  LORACT_CUDA_TRY(factor(l, true, w.splits_gram, kShiftSecond, w, status, stream, true, 0.f, gate));
+  trace_label("apply L^-T 2");
+  // In place when one CTA (pair) owns whole rows of the product: it has read its rows of U and of the remainder
+  // completely before its epilogue stores them.  With several column tiles per row block another CTA may still be
+  // reading the rows, so the result goes to the workspace and is copied.
+  GemmDesc probe;
+  probe.M = n; probe.N = l; probe.K = l; probe.lda = l; probe.ldb = l; probe.ldc = l; probe.n_terms = 3;
+  probe.terms[0] = {U, w.Lh}; probe.terms[1] = {U, w.Ll}; probe.terms[2] = {w.Ql, w.Lh};
+  probe.out = OUT_BF16; probe.C0 = U;
+  if (l <= 256 && gemm_tc_supported(probe)) {
+    LORACT_CUDA_TRY(apply(U, w.Ql, U, nullptr, gate));
+  } else {
+    LORACT_CUDA_TRY(apply(U, w.Ql, w.Qh, nullptr, gate));
+    if (gate) {
+      LORACT_CUDA_TRY(copy_bf16_gated_launch(w.Qh, (__nv_bfloat16*)U, (int64_t)n * l, gate, stream));
+    } else {
+      LORACT_CUDA_TRY(cudaMemcpyAsync(U, w.Qh, (size_t)n * l * 2, cudaMemcpyDeviceToDevice, stream));
     }
   }
   return cudaSuccess;
@@ -760,7 +830,7 @@ loract_status_t loract_joint_orthonormalise(const loract_desc_t* desc, int32_t r
   cudaStream_t st = (cudaStream_t)stream;
   const int r = desc->rank, n = (int)desc->n_tokens;
   trace_label(round ? "joint: small block 3" : "joint: small block 2");
-  cudaError_t e = factor_matrix(W_sum, r, round ? kShiftSecond : kShiftFirst, w.b, w.status, st);
+  cudaError_t e = factor_matrix(W_sum, r, round ? kShiftSecond : kShiftFirstMean, w.b, w.status, st);
   trace_label(round ? "joint: apply L^-T 2" : "joint: apply L^-T 1");
   if (round == 0) {
     if (e == cudaSuccess) e = apply_linv(w.b.Yh, w.b.Yl, n, r, w.b, w.b.Qh, w.b.Ql, w.status, st);
@@ -969,6 +1039,10 @@ int32_t loract_debug_trace_end(void* stream, char* names, float* micros, int32_t
 }
 
 void loract_debug_set_pair_mode(int32_t on) { gemm_tc_set_pair_mode(on); }
+
+void loract_debug_set_round_gate(float threshold) {
+  g_round_gate.store(threshold == 0.f ? kRoundGateDefault : threshold);
+}
 
 int32_t loract_debug_last_cuda_error(void) { return g_last_cuda_error.load(std::memory_order_relaxed); }
 

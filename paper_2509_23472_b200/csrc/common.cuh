@@ -107,13 +107,16 @@ struct GemmDesc {
   // (result = (t_0 + ... + t_{h-1}) / 2 + t_h + ...); 0 or negative: plain sum.  With the pair {A^T A, A^T B} and
   // h = 1 the result D gives D + D^T = A^T A + A^T B + B^T A: a symmetric three-term sum for two terms' work.
   int halve_at_term = 0;
+  // Tensor-core path: a device word written by an earlier kernel of the same stream; when it is zero the launch
+  // does nothing (no loads, no products, C untouched).  nullptr: unconditional.
+  const uint32_t* gate = nullptr;
 };
 
 // tcgen05 engine: bf16 operands, fp32 accumulation in tensor memory.  Returns cudaErrorNotSupported
 // for shapes it does not take (the caller then uses the SIMT kernel).
 bool gemm_tc_supported(const GemmDesc& g);
 cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t stream);
-int gemm_tc_pick_splits(int M, int N, int K, bool a_mn, bool b_mn);
+int gemm_tc_pick_splits(int M, int N, int K, bool a_mn, bool b_mn, int max_splits = 32);
 void gemm_tc_set_pair_mode(int on);   // test hook: 0 keeps every contraction on the one-CTA kernel
 // Test hooks for the give-up path of the bounded waits: a kernel that waits (with the engine's / the cluster
 // kernel's own wait) on a barrier nothing completes, for at most limit_ns, then sets LORACT_DEV_WAIT_EXPIRED.
@@ -160,6 +163,12 @@ struct SmallBlockArgs {
   bool use_f64 = false;  // compute type
   void* scratch = nullptr;
   float shift_rel = 0.f;
+  // shared-memory cluster kernel and the block scheme built on it: each diagonal entry is also multiplied by
+  // (1 + shift_diag_rel), a shift relative to the entry itself (the scale-invariant form, which leaves a
+  // matrix whose diagonal spans several orders of magnitude as well conditioned as its scaled form)
+  float shift_diag_rel = 0.f;
+  // device word written by an earlier kernel of the stream; zero: the launch does nothing.  nullptr: unconditional.
+  const uint32_t* gate = nullptr;
   void* linv_full = nullptr;  // fp32 (use_f64 == false) or fp64 (use_f64 == true), r x r
   float* linv_f32 = nullptr;  // fp32 copy, r x r
   __nv_bfloat16* linv_hi = nullptr;
@@ -191,8 +200,22 @@ cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_
                                    int64_t count, float* out_f32, __nv_bfloat16* out_bf16,
                                    cudaStream_t stream);
 // out (r x r) = S + S^T, S the fixed-order sum of the partials (each r x r, leading dimension r).
+// gate (optional): device word; zero means the launch does nothing.
 cudaError_t reduce_sym_launch(const float* partials, int n_partials, int64_t stride, int r, float* out,
-                              cudaStream_t stream);
+                              cudaStream_t stream, const uint32_t* gate = nullptr);
+// After the first orthonormalisation round: decides on the device whether the second round is needed.
+// W (r x r fp32, leading dimension r) is the Gram matrix that was factored, linv_hi the leading bf16 part of the
+// inverse factor L^-1 (leading dimension r).  With D = diag(W)^(-1/2) the kernel forms
+//   est = sum_ij (L^-1)_ij^2 W_jj = trace((D W D)^-1),
+// which lies between 1 / lambda_min and r / lambda_min of the diagonally scaled Gram matrix, the quantity that
+// multiplies the rounding error of W in the orthogonality defect of Y L^-T.  gate_words[0] = 1 if est > threshold, est is
+// not finite, or the status word is non-zero (a clamped pivot, a non-finite input), else 0; gate_words[1] = est
+// (float bits); gate_words[2] = rounds that will run (1 or 2).  One CTA, fixed summation order.
+cudaError_t round_gate_launch(const float* W, const __nv_bfloat16* linv_hi, int r, float threshold,
+                              const uint32_t* dev_status, uint32_t* gate_words, cudaStream_t stream);
+// dst = src (count bf16 elements, both 16-byte aligned, count a multiple of 8) when *gate != 0; nothing otherwise.
+cudaError_t copy_bf16_gated_launch(const __nv_bfloat16* src, __nv_bfloat16* dst, int64_t count, const uint32_t* gate,
+                                   cudaStream_t stream);
 // out = sum_s partials[s] as a bf16 triple hi + mid + lo (rows x cols, leading dimensions ld_in / ld_out).
 cudaError_t reduce_split3_launch(const float* partials, int n_partials, int64_t stride, int rows, int cols,
                                  int64_t ld_in, int64_t ld_out, __nv_bfloat16* hi, __nv_bfloat16* mid,

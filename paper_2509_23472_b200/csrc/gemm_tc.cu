@@ -66,6 +66,9 @@ struct TcParams {
   int store_bufs;     // staging boxes per epilogue warp (1 or 2)
   int halve_at_term;  // the accumulator is multiplied by 1/2 before the first product of this term (0: never)
   int a_keep_from_kb; // two-CTA kernel: K block from which the loads of A carry an evict-last hint (kb_total: none)
+  // one-tile kernels: when set and the word it points to is zero, the kernel loads, multiplies and stores nothing
+  // (a step that an earlier kernel of the same stream found unnecessary)
+  const uint32_t* gate;
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -520,7 +523,7 @@ gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   const int n0 = blockIdx.x * p.bn, m0 = blockIdx.y * kBM, split = blockIdx.z;
   const int kb_begin = split * p.kb_per_split;
   const int kb_count = max(0, min(p.kb_total, kb_begin + p.kb_per_split) - kb_begin);
-  const int n_iter = kb_count * p.n_terms;
+  int n_iter = kb_count * p.n_terms;
   const uint32_t stage_bytes = kABytes + p.b_bytes;
   // dynamic shared memory is declared 1024-aligned; round up anyway (swizzle atoms need it)
   unsigned char* tiles = (unsigned char*)(((uintptr_t)smem + 1023) & ~(uintptr_t)1023);
@@ -545,6 +548,7 @@ gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   // everything above overlaps the tail of the previous kernel; global memory only from here on
   pdl_wait();
   pdl_launch_dependents();
+  if (p.gate != nullptr && *(const volatile uint32_t*)p.gate == 0u) n_iter = -1;   // every role idles, nothing is stored
 
   if (warp == 0) {
     if (lane == 0) {
@@ -697,7 +701,7 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   const int n0 = blockIdx.y * p.bn, m0 = blockIdx.x * kBM, split = blockIdx.z;
   const int kb_begin = split * p.kb_per_split;
   const int kb_count = max(0, min(p.kb_total, kb_begin + p.kb_per_split) - kb_begin);
-  const int n_iter = kb_count * p.n_terms;
+  int n_iter = kb_count * p.n_terms;
   const uint32_t stage_bytes = kABytes + p.b_bytes;          // per CTA (b_bytes: half a B tile)
   unsigned char* tiles = (unsigned char*)(((uintptr_t)smem + 1023) & ~(uintptr_t)1023);
 
@@ -723,6 +727,7 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   const uint32_t tmem_base = tmem_slot;
   pdl_wait();
   pdl_launch_dependents();
+  if (p.gate != nullptr && *(const volatile uint32_t*)p.gate == 0u) n_iter = -1;   // every role idles, nothing is stored
 
   if (warp == 0 || warp == 2) {
     if (lane == 0) {
@@ -1252,13 +1257,13 @@ bool gemm_tc_supported(const GemmDesc& g) {
   return true;
 }
 
-int gemm_tc_pick_splits(int M, int N, int K, bool, bool) {
+int gemm_tc_pick_splits(int M, int N, int K, bool, bool, int max_splits) {
   const int tiles = ((M + kBM - 1) / kBM) * ((N + pick_bn(N) - 1) / pick_bn(N));
   const int kb = (K + kBK - 1) / kBK;
   if (tiles >= 96) return 1;
   int s = 148 / tiles;
   if (s > kb / 4) s = kb / 4;  // at least four K blocks per split
-  if (s > 32) s = 32;
+  if (s > max_splits) s = max_splits;
   return s < 1 ? 1 : s;
 }
 
@@ -1285,6 +1290,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   p.st_m_tiles = 0; p.st_units = 0; p.tma_store = 0; p.st_stages = kStreamStages; p.store_bufs = kStoreBufs;
   p.halve_at_term = g.halve_at_term > 0 ? g.halve_at_term : 0;
   p.a_keep_from_kb = g.a_keep_from_k >= 0 ? (int)(g.a_keep_from_k / kBK) : p.kb_total;
+  p.gate = g.gate;
 
   TmapPack maps;
   for (int t = 0; t < g.n_terms; ++t) {
@@ -1319,7 +1325,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   // Short contraction, large output, A K-major, B MN-major, one term (Reconstruct and the pre-norm backward):
   // the persistent kernel with B resident, when there is more than one tile per resident pair.
   if (g_pair_mode == 1 && g.M >= 2 * kBM && !g.a_mn && g.b_mn && g.n_terms == 1 && splits == 1 && p.kb_total <= 8 &&
-      g.N >= 256) {
+      g.N >= 256 && g.gate == nullptr) {
     TcParams sp = p;
     // 256 columns per tile (the tensor pipe is issue-bound on narrower instructions).  The resident B takes
     // 16 KB per K block and CTA; beyond four K blocks the A ring and the staging boxes shrink to make room

@@ -156,7 +156,7 @@ constexpr int kSymTile = 16;
 // partials x 256 elements; a thread adds its partials eight at a time into eight running sums (eight independent
 // loads in flight); the sums are combined in a fixed order.
 __global__ void __launch_bounds__(1024) reduce_sym_kernel(const float* partials, int n_partials, int64_t stride, int r,
-                                                          float* out) {
+                                                          float* out, const uint32_t* gate) {
   __shared__ float t[2][2][kSymTile][kSymTile + 1];   // [tile][half of the partials][row][column]
   // tile pair from the linear block index: I = largest with I (I + 1) / 2 <= b
   const int b = blockIdx.x;
@@ -169,6 +169,7 @@ __global__ void __launch_bounds__(1024) reduce_sym_kernel(const float* partials,
   const int row = (tile ? J : I) * kSymTile + a, col = (tile ? I : J) * kSymTile + c;
   pdl_wait();
   pdl_launch_dependents();
+  if (gate != nullptr && *(const volatile uint32_t*)gate == 0u) return;   // the whole grid: this step is not needed
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   if (row < r && col < r && !(tile == 1 && I == J)) {
     const float* src = partials + (int64_t)row * r + col;
@@ -506,6 +507,56 @@ cudaError_t launch_simt_typed(const SimtParams& p, bool acc64, cudaStream_t stre
   return cudaGetLastError();
 }
 
+// Decision after the first orthonormalisation round (see round_gate_launch in common.cuh).  One CTA of 1024
+// threads; a thread takes 8 consecutive elements of L^-1 (one 16-byte load) at a time, every sum in a fixed order.
+__global__ void __launch_bounds__(1024) round_gate_kernel(const float* __restrict__ W,
+                                                          const __nv_bfloat16* __restrict__ linv_hi, int r,
+                                                          float threshold, const uint32_t* dev_status,
+                                                          uint32_t* gate_words) {
+  __shared__ float s_diag[640];
+  __shared__ float s_red[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_wait();
+  pdl_launch_dependents();
+  for (int j = tid; j < r; j += 1024) s_diag[j] = W[(int64_t)j * r + j];
+  __syncthreads();
+  float acc = 0.f;
+  const int64_t count = (int64_t)r * r;   // r is a multiple of 8, so a group of 8 stays inside one row
+  for (int64_t e = (int64_t)tid * 8; e < count; e += 1024 * 8) {
+    const int row = (int)(e / r), col = (int)(e - (int64_t)row * r);
+    if (col > row) continue;              // strictly above the diagonal: zeros
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(linv_hi + e));
+    const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float lo = __uint_as_float(w4[q] << 16), hi = __uint_as_float(w4[q] & 0xffff0000u);
+      acc += lo * lo * s_diag[col + 2 * q] + hi * hi * s_diag[col + 2 * q + 1];
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) s_red[warp] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    float est = 0.f;
+    for (int q = 0; q < 32; ++q) est += s_red[q];
+    const uint32_t st = dev_status ? *(const volatile uint32_t*)dev_status : 0u;
+    const bool again = !(est <= threshold) || st != 0u;   // a NaN estimate compares false: second round
+    gate_words[0] = again ? 1u : 0u;
+    gate_words[1] = __float_as_uint(est);
+    gate_words[2] = again ? 2u : 1u;
+  }
+}
+
+__global__ void copy_bf16_gated_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int64_t n16,
+                                       const uint32_t* gate) {
+  pdl_wait();
+  pdl_launch_dependents();
+  if (*(const volatile uint32_t*)gate == 0u) return;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (int64_t)gridDim.x * blockDim.x)
+    dst[i] = src[i];
+}
+
 }  // namespace
 
 cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t stream) {
@@ -542,10 +593,32 @@ cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_
 }
 
 cudaError_t reduce_sym_launch(const float* partials, int n_partials, int64_t stride, int r, float* out,
-                              cudaStream_t stream) {
+                              cudaStream_t stream, const uint32_t* gate) {
   const int nt = (r + kSymTile - 1) / kSymTile;
   LORACT_CUDA_TRY(launch_pdl(reduce_sym_kernel, dim3(nt * (nt + 1) / 2), dim3(1024), 0, stream, partials, n_partials,
-                             stride, r, out));
+                             stride, r, out, gate));
+  count_launch(__func__, stream);
+  return cudaGetLastError();
+}
+
+cudaError_t round_gate_launch(const float* W, const __nv_bfloat16* linv_hi, int r, float threshold,
+                              const uint32_t* dev_status, uint32_t* gate_words, cudaStream_t stream) {
+  if (r < 8 || r > 640 || r % 8 || ((uintptr_t)linv_hi & 15)) return cudaErrorInvalidValue;
+  LORACT_CUDA_TRY(launch_pdl(round_gate_kernel, dim3(1), dim3(1024), 0, stream, W, linv_hi, r, threshold, dev_status,
+                             gate_words));
+  count_launch(__func__, stream);
+  return cudaGetLastError();
+}
+
+cudaError_t copy_bf16_gated_launch(const __nv_bfloat16* src, __nv_bfloat16* dst, int64_t count, const uint32_t* gate,
+                                   cudaStream_t stream) {
+  if (count % 8 || ((uintptr_t)src & 15) || ((uintptr_t)dst & 15) || !gate) return cudaErrorInvalidValue;
+  const int64_t n16 = count / 8;
+  int grid = (int)((n16 + 255) / 256);
+  if (grid > 148 * 8) grid = 148 * 8;
+  if (grid < 1) grid = 1;
+  LORACT_CUDA_TRY(launch_pdl(copy_bf16_gated_kernel, dim3(grid), dim3(256), 0, stream, (const uint4*)src, (uint4*)dst,
+                             n16, gate));
   count_launch(__func__, stream);
   return cudaGetLastError();
 }

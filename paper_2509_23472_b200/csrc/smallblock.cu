@@ -285,6 +285,7 @@ cudaError_t launch_typed(const SBParams& p, cudaStream_t stream) {
 // the diagonal of the whole matrix's leading block (`scale`): a Schur complement may be nothing but rounding noise.
 struct TwoLevelCtx {
   float shift_rel;
+  float shift_diag_rel;
   uint32_t* dev_status;
   int64_t ld;
   const float* scale_diag;
@@ -298,7 +299,7 @@ cudaError_t factor_blocks(const TwoLevelCtx& c, float* W, float* X, __nv_bfloat1
   if (n <= 256) {
     SmallBlockArgs s;
     s.r = n; s.partials = W; s.partial_type = ELEM_F32; s.n_partials = 1; s.partial_stride = 0;
-    s.use_f64 = false; s.shift_rel = c.shift_rel; s.in_ld = ld; s.out_ld = ld;
+    s.use_f64 = false; s.shift_rel = c.shift_rel; s.shift_diag_rel = c.shift_diag_rel; s.in_ld = ld; s.out_ld = ld;
     s.linv_f32 = X; s.linv_hi = hi; s.linv_lo = lo; s.dev_status = c.dev_status;
     if (!top) { s.scale_diag = c.scale_diag; s.scale_n = c.scale_n; s.scale_ld = ld; }
     return small_block_cluster_launch(s, c.stream);
@@ -350,7 +351,7 @@ cudaError_t small_block_two_level(const SmallBlockArgs& a, cudaStream_t stream) 
   LORACT_CUDA_TRY(cudaMemsetAsync(a.linv_hi, 0, (size_t)r * r * 2, stream));
   if (a.linv_lo) LORACT_CUDA_TRY(cudaMemsetAsync(a.linv_lo, 0, (size_t)r * r * 2, stream));
   TwoLevelCtx c;
-  c.shift_rel = a.shift_rel; c.dev_status = a.dev_status; c.ld = r; c.scale_diag = W; c.scale_n = 256;
+  c.shift_rel = a.shift_rel; c.shift_diag_rel = a.shift_diag_rel; c.dev_status = a.dev_status; c.ld = r; c.scale_diag = W; c.scale_n = 256;
   c.stream = stream;
   return factor_blocks(c, W, X, a.linv_hi, a.linv_lo, r, T, true);
 }
@@ -368,7 +369,7 @@ cudaError_t small_block_launch(const SmallBlockArgs& a, cudaStream_t stream) {
   p.n_partials = a.n_partials;
   p.partial_stride = a.partial_stride;
   p.scratch = a.scratch;
-  p.shift_rel = a.shift_rel;
+  p.shift_rel = a.shift_rel + a.shift_diag_rel;   // this kernel knows the shift relative to the mean diagonal only
   p.linv_full = a.linv_full;
   p.linv_f32 = a.linv_f32;
   p.linv_hi = a.linv_hi;

@@ -50,6 +50,8 @@ struct SCParams {
   int n_partials;
   int64_t partial_stride;
   float shift_rel;
+  float shift_diag_rel;    // each diagonal entry is also multiplied by (1 + shift_diag_rel)
+  const uint32_t* gate;    // optional device word: zero means every CTA leaves at once
   float* linv_f32;
   __nv_bfloat16* linv_hi;
   __nv_bfloat16* linv_lo;
@@ -481,6 +483,8 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
   // everything above overlaps the tail of the previous kernel; global memory only from here on
   pdl_wait();
   pdl_launch_dependents();
+  // The same word in every CTA, read before anything crosses between them: the whole cluster leaves together.
+  if (p.gate != nullptr && *(const volatile uint32_t*)p.gate == 0u) return;
 
   // ---- load.  Block t is summed over the partials by CTA t mod 8 and written into the slot of the CTA
   // that works on it first (CTA 0 for block rows 0 and 1, the owner otherwise).  All global loads of a
@@ -554,8 +558,10 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
       float4 sv = acc[u];
       if (bi == bj) {
         const int dcol = a - 4 * q4;  // position of the diagonal element inside this quad, if any
-        const float add = (bi * kB + a) < r ? shift : 1.f;  // padding rows of a ragged last block: identity
-        if (dcol == 0) sv.x += add; else if (dcol == 1) sv.y += add; else if (dcol == 2) sv.z += add; else if (dcol == 3) sv.w += add;
+        const bool in_range = (bi * kB + a) < r;            // padding rows of a ragged last block: identity
+        const float mul = in_range ? p.shift_diag_rel : 0.f, add = in_range ? shift : 1.f;
+        if (dcol == 0) sv.x += sv.x * mul + add; else if (dcol == 1) sv.y += sv.y * mul + add;
+        else if (dcol == 2) sv.z += sv.z * mul + add; else if (dcol == 3) sv.w += sv.w * mul + add;
       }
       const int dst_cta = bi <= 1 ? 0 : owner_of(bi, bj, nblk);
       const uint32_t dst = map_to_cta(smem_addr(slots + blk * kSlot), dst_cta);
@@ -846,6 +852,8 @@ cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t str
   p.n_partials = a.n_partials;
   p.partial_stride = a.partial_stride;
   p.shift_rel = a.shift_rel;
+  p.shift_diag_rel = a.shift_diag_rel;
+  p.gate = a.gate;
   p.linv_f32 = a.linv_f32;
   p.linv_hi = a.linv_hi;
   p.linv_lo = a.linv_lo;
