@@ -55,11 +55,19 @@ void loract_debug_set_pair_mode(int32_t on);
 
 /* The orthonormalisation of the bf16 path runs its second Gram round only when the first round's Gram matrix W
  * was not conditioned well enough for one: a one-CTA kernel forms est = trace((D W D)^-1), D = diag(W)^(-1/2),
- * from the inverse factor and compares it with a threshold (ranks up to 256; above that both rounds always run).
+ * from the inverse factor and compares est times the number of 64-row blocks per accumulation chain of the Gram
+ * product with a threshold (widths up to 512; above that both rounds always run).
  * This sets the threshold, process-wide: a negative value forces both rounds, +infinity allows one round whenever
  * no status bit is set, 0 restores the default.  After a call the status block at the head of the workspace
  * holds, as 32-bit words 4, 5, 6: whether the second round ran (0 / 1), est (float bits), the number of rounds. */
 void loract_debug_set_round_gate(float threshold);
+
+/* The deciding kernel alone.  W: r x r fp32 (device, leading dimension r), linv_hi: r x r bf16 lower triangular
+ * (device), r a multiple of 8 up to 640; status_word: device uint32 or NULL.  words (device, 3 x uint32) receives
+ * { est > threshold or est not finite or *status_word != 0,  est = sum_ij linv_ij^2 W_jj as float bits,
+ *   1 or 2 = the number of rounds }. */
+loract_status_t loract_debug_round_gate(const float* W, const void* linv_hi, int32_t r, float threshold,
+                                        const uint32_t* status_word, uint32_t* words, void* stream);
 
 /* Stage trace.  Between trace_begin and trace_end every kernel the library launches on `stream` is followed by
  * a CUDA event; trace_end synchronises the stream and writes, per kernel in launch order, a label (64 bytes

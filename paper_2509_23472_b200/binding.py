@@ -347,7 +347,7 @@ OUT_F32, OUT_BF16, OUT_SPLIT, OUT_F64 = 0, 1, 2, 3
 DEBUG_EXPORTS = ("loract_debug_gemm", "loract_debug_small_block", "loract_debug_set_pair_mode",
                  "loract_debug_last_cuda_error", "loract_debug_trace_begin", "loract_debug_trace_end",
                  "loract_debug_wait_expiry", "loract_debug_project", "loract_debug_gemm_halved",
-                 "loract_debug_reduce_sym", "loract_debug_set_round_gate")
+                 "loract_debug_reduce_sym", "loract_debug_set_round_gate", "loract_debug_round_gate")
 
 
 def _debug_lib():
@@ -364,6 +364,8 @@ def _debug_lib():
         l.loract_debug_reduce_sym.argtypes = [vp, i32, i64, i32, vp, vp]
         l.loract_debug_small_block.restype = ctypes.c_int
         l.loract_debug_small_block.argtypes = [i32, vp, i32, i32, i64, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp]
+        l.loract_debug_round_gate.restype = ctypes.c_int
+        l.loract_debug_round_gate.argtypes = [vp, vp, i32, ctypes.c_float, vp, vp, vp]
         l._debug_ready = True
     return l
 
@@ -443,6 +445,18 @@ def debug_set_round_gate(threshold: float) -> None:
     l.loract_debug_set_round_gate.restype = None
     l.loract_debug_set_round_gate.argtypes = [ctypes.c_float]
     l.loract_debug_set_round_gate(float(threshold))
+
+
+def debug_round_gate(W: torch.Tensor, linv_hi: torch.Tensor, threshold: float,
+                     status: Optional[torch.Tensor] = None):
+    """Test hook: the deciding kernel alone.  Returns (second round needed, est, rounds)."""
+    l = _debug_lib()
+    r = W.shape[0]
+    words = torch.zeros(3, dtype=torch.int32, device=W.device)
+    _check(l.loract_debug_round_gate(_ptr(W), _ptr(linv_hi), r, ctypes.c_float(threshold), _ptr(status), _ptr(words),
+                                     _stream(W.device)), "loract_debug_round_gate")
+    w = words.cpu()
+    return int(w[0]), float(w[1:2].view(torch.float32).item()), int(w[2])
 
 
 def round_gate_words(ws: torch.Tensor):

@@ -69,10 +69,12 @@ constexpr float kShiftFirstDiag = 2e-7f;
 constexpr float kShiftFirstMean = 3e-6f;  // fp32 inputs (fp64 factorisation): relative to the mean diagonal
 constexpr int kGateWord = 4;               // words 4..6 of the status block: gate, estimate, rounds
 constexpr float kShiftSecond = 1e-7f;  // second Gram (already close to the identity), relative to the mean diagonal
-// Second orthonormalisation round: run only when trace((D W D)^-1) of the first round's Gram matrix exceeds this
-// (D = diag(W)^(-1/2)), or when a status bit is set.  The defect of one round is the rounding error of the fp32 Gram
-// matrix (a few 1e-9 of sqrt(W_ii W_jj) per entry) times that trace.
-constexpr float kRoundGateDefault = 3.0e4f;
+// Second orthonormalisation round: run only when est = trace((D W D)^-1) of the first round's Gram matrix
+// (D = diag(W)^(-1/2)) times the number of 64-row blocks one accumulation chain of the Gram product covers exceeds
+// this, or when a status bit is set.  Measured on B200: the defect max|Q1^T Q1 - I| that one round leaves is about
+// 1e-9 * est * blocks (the tensor cores truncate the accumulator once per instruction, so the error of W grows with
+// the length of the chain); 2e5 keeps it near 2e-4, under the rounding of U to bf16.
+constexpr float kRoundGateDefault = 2.0e5f;
 std::atomic<float> g_round_gate{kRoundGateDefault};
 
 struct Carver {
@@ -318,7 +320,7 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
   // factor whether the Gram matrix was conditioned well enough for one round (gate word: 0 = done).  The kernels of
   // round 2 are launched in any case and leave at once when the gate word is zero: no host synchronisation.
   uint32_t* gate_words = status + kGateWord;
-  const bool can_gate = l <= 256 && l % 8 == 0;   // the block scheme above 256 columns always runs both rounds
+  const bool can_gate = l <= 512 && l % 8 == 0;   // widths above 512 (general fp64 kernel) always run both rounds
   const uint32_t* gate = can_gate ? gate_words : nullptr;
   auto gram = [&](const void* Yh, const void* Yl, const uint32_t* gt) {
     // D = (Yl^T Yl + Yh^T Yh) / 2 + Yh^T Yl: the sum of the partials, added to its transpose before the factorisation,
@@ -354,8 +356,10 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
   LORACT_CUDA_TRY(factor(l, true, w.splits_gram, l <= 512 ? 0.f : kShiftFirstMean, w, status, stream, true,
                          l <= 512 ? kShiftFirstDiag : 0.f));
   trace_label("round gate");
-  LORACT_CUDA_TRY(round_gate_launch(w.gram_partials, w.Lh, l, can_gate ? g_round_gate.load() : -1.f, status, gate_words,
-                                    stream));
+  const int kb_total = (n + 63) / 64, n_split = w.splits_gram < 1 ? 1 : w.splits_gram;
+  const float chain_blocks = (float)((kb_total + n_split - 1) / n_split);
+  LORACT_CUDA_TRY(round_gate_launch(w.gram_partials, w.Lh, l, can_gate ? g_round_gate.load() / chain_blocks : -1.f, status,
+                                    gate_words, stream));
   trace_label("apply L^-T 1");
   LORACT_CUDA_TRY(apply(w.Yh, w.Yl, U, w.Ql, nullptr));
   trace_label("Gram 2");
@@ -1039,6 +1043,13 @@ int32_t loract_debug_trace_end(void* stream, char* names, float* micros, int32_t
 }
 
 void loract_debug_set_pair_mode(int32_t on) { gemm_tc_set_pair_mode(on); }
+
+loract_status_t loract_debug_round_gate(const float* W, const void* linv_hi, int32_t r, float threshold,
+                                        const uint32_t* status_word, uint32_t* words, void* stream) {
+  if (!W || !linv_hi || !words) return LORACT_ERR_INVALID_ARG;
+  return from_cuda(round_gate_launch(W, (const __nv_bfloat16*)linv_hi, r, threshold, status_word, words,
+                                     (cudaStream_t)stream));
+}
 
 void loract_debug_set_round_gate(float threshold) {
   g_round_gate.store(threshold == 0.f ? kRoundGateDefault : threshold);

@@ -195,10 +195,13 @@ cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t str
 // X21 of a 2 x 2 block lower-triangular inverse as bf16 hi/lo (and optionally fp32), plus zeros in the block
 // above the diagonal: src (rows x cols fp32, leading dimension ld) -> hi/lo at the same place.
 cudaError_t split_block_launch(const float* src, int rows, int cols, int64_t ld, __nv_bfloat16* hi,
-                               __nv_bfloat16* lo, cudaStream_t stream);
+                               __nv_bfloat16* lo, cudaStream_t stream, const uint32_t* gate = nullptr);
+// Zero fill of up to three ranges (16-byte aligned, sizes multiples of 16; a null range has size 0), one launch.
+cudaError_t zero3_gated_launch(void* a, size_t a_bytes, void* b, size_t b_bytes, void* c, size_t c_bytes,
+                               const uint32_t* gate, cudaStream_t stream);
 cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_t stride,
                                    int64_t count, float* out_f32, __nv_bfloat16* out_bf16,
-                                   cudaStream_t stream);
+                                   cudaStream_t stream, const uint32_t* gate = nullptr);
 // out (r x r) = S + S^T, S the fixed-order sum of the partials (each r x r, leading dimension r).
 // gate (optional): device word; zero means the launch does nothing.
 cudaError_t reduce_sym_launch(const float* partials, int n_partials, int64_t stride, int r, float* out,

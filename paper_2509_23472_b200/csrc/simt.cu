@@ -28,6 +28,7 @@ struct SimtParams {
   int accumulate;
   float alpha;
   int halve_at_term;  // the sum so far is multiplied by 1/2 before this term (0: never)
+  const uint32_t* gate;  // 32 x 32 tile kernel: optional device word, zero means the launch does nothing
 };
 
 constexpr int kTile = 64;   // output tile 64 x 64, 256 threads, 4 x 4 outputs per thread
@@ -135,9 +136,10 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(SimtParams p) {
 
 __global__ void reduce_partials_kernel(const float* __restrict__ partials, int n_partials,
                                        int64_t stride, int64_t count, float* __restrict__ out_f32,
-                                       __nv_bfloat16* __restrict__ out_bf16) {
+                                       __nv_bfloat16* __restrict__ out_bf16, const uint32_t* gate) {
   pdl_wait();
   pdl_launch_dependents();
+  if (gate != nullptr && *(const volatile uint32_t*)gate == 0u) return;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count;
        i += (int64_t)gridDim.x * blockDim.x) {
     float s = 0.f;
@@ -228,6 +230,7 @@ __global__ void __launch_bounds__(64) gemm_f32_tile32_kernel(SimtParams p0, Simt
   const int m0 = blockIdx.y * kT32, n0 = blockIdx.x * kT32;
   pdl_wait();
   pdl_launch_dependents();
+  if (p.gate != nullptr && *(const volatile uint32_t*)p.gate == 0u) return;
   if (m0 >= p.M || n0 >= p.N) return;
   const int tm = tid >> 3, tn = tid & 7;               // outputs (4 tm + i, tn + 8 j)
   const float* A = (const float*)p.A[0];
@@ -306,7 +309,9 @@ __global__ void __launch_bounds__(64) gemm_f32_tile32_kernel(SimtParams p0, Simt
 
 // hi/lo split of a block of an fp32 matrix, in place of the same block of two bf16 matrices.
 __global__ void split_block_kernel(const float* __restrict__ src, int rows, int cols, int64_t ld,
-                                   __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+                                   __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                   const uint32_t* gate) {
+  if (gate != nullptr && *(const volatile uint32_t*)gate == 0u) return;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < (int64_t)rows * cols;
        i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t row = i / cols, col = i - row * cols;
@@ -548,6 +553,19 @@ __global__ void __launch_bounds__(1024) round_gate_kernel(const float* __restric
   }
 }
 
+// Zero fill of up to three 16-byte aligned ranges (counts in 16-byte units), skipped when *gate == 0.
+__global__ void zero3_gated_kernel(uint4* a, int64_t na, uint4* b, int64_t nb, uint4* c, int64_t nc,
+                                   const uint32_t* gate) {
+  pdl_wait();
+  pdl_launch_dependents();
+  if (gate != nullptr && *(const volatile uint32_t*)gate == 0u) return;
+  const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x, t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (int64_t i = t0; i < na; i += stride) a[i] = z;
+  for (int64_t i = t0; i < nb; i += stride) b[i] = z;
+  for (int64_t i = t0; i < nc; i += stride) c[i] = z;
+}
+
 __global__ void copy_bf16_gated_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int64_t n16,
                                        const uint32_t* gate) {
   pdl_wait();
@@ -582,12 +600,12 @@ cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t stream) {
 
 cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_t stride,
                                    int64_t count, float* out_f32, __nv_bfloat16* out_bf16,
-                                   cudaStream_t stream) {
+                                   cudaStream_t stream, const uint32_t* gate) {
   int grid = (int)((count + 255) / 256);
   if (grid > 148 * 16) grid = 148 * 16;
   if (grid < 1) grid = 1;
   LORACT_CUDA_TRY(launch_pdl(reduce_partials_kernel, dim3(grid), dim3(256), 0, stream, partials, n_partials, stride,
-                             count, out_f32, out_bf16));
+                             count, out_f32, out_bf16, gate));
   count_launch(__func__, stream);
   return cudaGetLastError();
 }
@@ -606,6 +624,15 @@ cudaError_t round_gate_launch(const float* W, const __nv_bfloat16* linv_hi, int 
   if (r < 8 || r > 640 || r % 8 || ((uintptr_t)linv_hi & 15)) return cudaErrorInvalidValue;
   LORACT_CUDA_TRY(launch_pdl(round_gate_kernel, dim3(1), dim3(1024), 0, stream, W, linv_hi, r, threshold, dev_status,
                              gate_words));
+  count_launch(__func__, stream);
+  return cudaGetLastError();
+}
+
+cudaError_t zero3_gated_launch(void* a, size_t a_bytes, void* b, size_t b_bytes, void* c, size_t c_bytes,
+                               const uint32_t* gate, cudaStream_t stream) {
+  if (((uintptr_t)a | (uintptr_t)b | (uintptr_t)c | a_bytes | b_bytes | c_bytes) & 15) return cudaErrorInvalidValue;
+  LORACT_CUDA_TRY(launch_pdl(zero3_gated_kernel, dim3(148), dim3(512), 0, stream, (uint4*)a, (int64_t)(a_bytes / 16),
+                             (uint4*)b, (int64_t)(b_bytes / 16), (uint4*)c, (int64_t)(c_bytes / 16), gate));
   count_launch(__func__, stream);
   return cudaGetLastError();
 }
@@ -637,6 +664,7 @@ cudaError_t reduce_split3_launch(const float* partials, int n_partials, int64_t 
 
 cudaError_t gemm_f32_small_launch(const GemmDesc& g, cudaStream_t stream, const GemmDesc* second) {
   auto fill = [](const GemmDesc& g, SimtParams& p) {
+    // (the gate of the first product holds for the whole launch)
     if (g.a_type != ELEM_F32 || g.b_type != ELEM_F32 || g.out != OUT_F32 || g.n_terms != 1 || g.splits > 1)
       return false;
     p = SimtParams{};
@@ -648,11 +676,13 @@ cudaError_t gemm_f32_small_launch(const GemmDesc& g, cudaStream_t stream, const 
     p.out = g.out; p.C0 = g.C0; p.ldc = g.ldc; p.splits = 1;
     p.accumulate = g.accumulate ? 1 : 0;
     p.alpha = g.alpha;
+    p.gate = nullptr;
     return true;
   };
   SimtParams p0, p1;
   if (!fill(g, p0) || (second && !fill(*second, p1))) return cudaErrorNotSupported;
   if (!second) p1 = p0;
+  p0.gate = p1.gate = g.gate;
   const int M = second ? std::max(g.M, second->M) : g.M, N = second ? std::max(g.N, second->N) : g.N;
   dim3 grid((N + kT32 - 1) / kT32, (M + kT32 - 1) / kT32, second ? 2 : 1);
   LORACT_CUDA_TRY(launch_pdl(gemm_f32_tile32_kernel, grid, dim3(64), 0, stream, p0, p1));
@@ -661,10 +691,10 @@ cudaError_t gemm_f32_small_launch(const GemmDesc& g, cudaStream_t stream, const 
 }
 
 cudaError_t split_block_launch(const float* src, int rows, int cols, int64_t ld, __nv_bfloat16* hi,
-                               __nv_bfloat16* lo, cudaStream_t stream) {
+                               __nv_bfloat16* lo, cudaStream_t stream, const uint32_t* gate) {
   int grid = (int)(((int64_t)rows * cols + 255) / 256);
   if (grid > 148 * 4) grid = 148 * 4;
-  split_block_kernel<<<grid, 256, 0, stream>>>(src, rows, cols, ld, hi, lo);
+  split_block_kernel<<<grid, 256, 0, stream>>>(src, rows, cols, ld, hi, lo, gate);
   count_launch(__func__, stream);
   return cudaGetLastError();
 }

@@ -286,6 +286,7 @@ cudaError_t launch_typed(const SBParams& p, cudaStream_t stream) {
 struct TwoLevelCtx {
   float shift_rel;
   float shift_diag_rel;
+  const uint32_t* gate;
   uint32_t* dev_status;
   int64_t ld;
   const float* scale_diag;
@@ -300,7 +301,7 @@ cudaError_t factor_blocks(const TwoLevelCtx& c, float* W, float* X, __nv_bfloat1
     SmallBlockArgs s;
     s.r = n; s.partials = W; s.partial_type = ELEM_F32; s.n_partials = 1; s.partial_stride = 0;
     s.use_f64 = false; s.shift_rel = c.shift_rel; s.shift_diag_rel = c.shift_diag_rel; s.in_ld = ld; s.out_ld = ld;
-    s.linv_f32 = X; s.linv_hi = hi; s.linv_lo = lo; s.dev_status = c.dev_status;
+    s.linv_f32 = X; s.linv_hi = hi; s.linv_lo = lo; s.dev_status = c.dev_status; s.gate = c.gate;
     if (!top) { s.scale_diag = c.scale_diag; s.scale_n = c.scale_n; s.scale_ld = ld; }
     return small_block_cluster_launch(s, c.stream);
   }
@@ -316,6 +317,7 @@ cudaError_t factor_blocks(const TwoLevelCtx& c, float* W, float* X, __nv_bfloat1
     g.a_type = g.b_type = ELEM_F32;
     g.terms[0] = {A, B};
     g.out = OUT_F32; g.C0 = C; g.ldc = ldc; g.alpha = alpha; g.accumulate = accumulate;
+    g.gate = c.gate;
     return g;
   };
   const float* W21 = W + (size_t)r1 * ld;
@@ -335,7 +337,8 @@ cudaError_t factor_blocks(const TwoLevelCtx& c, float* W, float* X, __nv_bfloat1
                                 Tnext, false));
   // X21 = -X22 T2 : X21[m][n] = -sum_k X22[m][k] T2[k][n]
   LORACT_CUDA_TRY(gemm_f32_small_launch(product(r2, r1, r2, X22, ld, T2, r1, true, X21, ld, -1.f, false), c.stream));
-  return split_block_launch(X21, r2, r1, ld, hi + (size_t)r1 * ld, lo ? lo + (size_t)r1 * ld : nullptr, c.stream);
+  return split_block_launch(X21, r2, r1, ld, hi + (size_t)r1 * ld, lo ? lo + (size_t)r1 * ld : nullptr, c.stream,
+                            c.gate);
 }
 
 // scratch: W (r x r) + X (r x r) + the temporaries of every level, fp32.
@@ -345,13 +348,12 @@ cudaError_t small_block_two_level(const SmallBlockArgs& a, cudaStream_t stream) 
   float* X = a.linv_f32 ? a.linv_f32 : W + (size_t)r * r;
   float* T = W + 2 * (size_t)r * r;
   LORACT_CUDA_TRY(reduce_partials_launch((const float*)a.partials, a.n_partials, a.partial_stride, (int64_t)r * r, W,
-                                         nullptr, stream));
+                                         nullptr, stream, a.gate));
   // blocks above the diagonal are never written below: X is read as a whole by the products of the next level up
-  LORACT_CUDA_TRY(cudaMemsetAsync(X, 0, (size_t)r * r * 4, stream));
-  LORACT_CUDA_TRY(cudaMemsetAsync(a.linv_hi, 0, (size_t)r * r * 2, stream));
-  if (a.linv_lo) LORACT_CUDA_TRY(cudaMemsetAsync(a.linv_lo, 0, (size_t)r * r * 2, stream));
+  LORACT_CUDA_TRY(zero3_gated_launch(X, (size_t)r * r * 4, a.linv_hi, (size_t)r * r * 2, a.linv_lo,
+                                     a.linv_lo ? (size_t)r * r * 2 : 0, a.gate, stream));
   TwoLevelCtx c;
-  c.shift_rel = a.shift_rel; c.shift_diag_rel = a.shift_diag_rel; c.dev_status = a.dev_status; c.ld = r; c.scale_diag = W; c.scale_n = 256;
+  c.shift_rel = a.shift_rel; c.shift_diag_rel = a.shift_diag_rel; c.gate = a.gate; c.dev_status = a.dev_status; c.ld = r; c.scale_diag = W; c.scale_n = 256;
   c.stream = stream;
   return factor_blocks(c, W, X, a.linv_hi, a.linv_lo, r, T, true);
 }
@@ -362,6 +364,7 @@ cudaError_t small_block_launch(const SmallBlockArgs& a, cudaStream_t stream) {
       a.linv_hi && a.in_ld == 0 && a.out_ld == 0 && (((uintptr_t)a.partials & 15) == 0) &&
       (a.partial_stride % 4 == 0))
     return small_block_two_level(a, stream);
+  if (a.gate) return cudaErrorNotSupported;   // the general kernel is unconditional
   SBParams p;
   p.r = a.r;
   p.partials = a.partials;
