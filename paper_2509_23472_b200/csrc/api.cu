@@ -206,11 +206,14 @@ constexpr int kReduceFirst = 8;    // partial count from which a separate, all-S
 // `sym`: the partials hold D = Yh^T Yh / 2 + Yh^T Yl (the two-term form of the tall Gram products); the matrix to
 // factor is D + D^T.
 cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs& w, uint32_t* status,
-                   cudaStream_t stream, bool sym = false, float shift_diag = 0.f, const uint32_t* gate = nullptr) {
+                   cudaStream_t stream, bool sym = false, float shift_diag = 0.f, const uint32_t* gate = nullptr,
+                   uint32_t* gate_out = nullptr, float gate_threshold = 0.f) {
   SmallBlockArgs a;
   a.r = l;
   a.shift_diag_rel = shift_diag;
   a.gate = gate;
+  a.gate_out = gate_out;
+  a.gate_threshold = gate_threshold;
   a.scratch = w.sb_scratch;
   a.dev_status = status;
   if (bf16) {
@@ -351,15 +354,19 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
   };
   trace_label("Gram 1");
   LORACT_CUDA_TRY(gram(w.Yh, w.Yl, nullptr));
+  const int kb_total = (n + 63) / 64, n_split = w.splits_gram < 1 ? 1 : w.splits_gram;
+  const float chain_blocks = (float)((kb_total + n_split - 1) / n_split);
+  const float threshold = can_gate ? g_round_gate.load() / chain_blocks : -1.f;
+  // up to 256 columns the factorisation kernel forms the estimate itself while it writes L^-1 out
+  const bool gate_in_factor = l <= 256 && l % 8 == 0;
   trace_label("small block 2");
   // (widths above 512 take the general fp64 kernel, which knows the shift relative to the mean diagonal only)
   LORACT_CUDA_TRY(factor(l, true, w.splits_gram, l <= 512 ? 0.f : kShiftFirstMean, w, status, stream, true,
-                         l <= 512 ? kShiftFirstDiag : 0.f));
-  trace_label("round gate");
-  const int kb_total = (n + 63) / 64, n_split = w.splits_gram < 1 ? 1 : w.splits_gram;
-  const float chain_blocks = (float)((kb_total + n_split - 1) / n_split);
-  LORACT_CUDA_TRY(round_gate_launch(w.gram_partials, w.Lh, l, can_gate ? g_round_gate.load() / chain_blocks : -1.f, status,
-                                    gate_words, stream));
+                         l <= 512 ? kShiftFirstDiag : 0.f, nullptr, gate_in_factor ? gate_words : nullptr, threshold));
+  if (!gate_in_factor) {
+    trace_label("round gate");
+    LORACT_CUDA_TRY(round_gate_launch(w.gram_partials, w.Lh, l, threshold, status, gate_words, stream));
+  }
   trace_label("apply L^-T 1");
   LORACT_CUDA_TRY(apply(w.Yh, w.Yl, U, w.Ql, nullptr));
   trace_label("Gram 2");

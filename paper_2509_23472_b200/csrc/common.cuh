@@ -169,6 +169,10 @@ struct SmallBlockArgs {
   float shift_diag_rel = 0.f;
   // device word written by an earlier kernel of the stream; zero: the launch does nothing.  nullptr: unconditional.
   const uint32_t* gate = nullptr;
+  // shared-memory cluster kernel only (r <= 256): three words that receive what round_gate_launch would write for
+  // this matrix and its inverse factor, computed inside the factorisation (no extra launch)
+  uint32_t* gate_out = nullptr;
+  float gate_threshold = 0.f;
   void* linv_full = nullptr;  // fp32 (use_f64 == false) or fp64 (use_f64 == true), r x r
   float* linv_f32 = nullptr;  // fp32 copy, r x r
   __nv_bfloat16* linv_hi = nullptr;

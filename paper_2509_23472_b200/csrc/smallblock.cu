@@ -360,6 +360,7 @@ cudaError_t small_block_two_level(const SmallBlockArgs& a, cudaStream_t stream) 
 
 cudaError_t small_block_launch(const SmallBlockArgs& a, cudaStream_t stream) {
   if (small_block_cluster_supported(a)) return small_block_cluster_launch(a, stream);
+  if (a.gate_out) return cudaErrorNotSupported;   // only the shared-memory kernel forms the estimate
   if (!a.use_f64 && a.partial_type == ELEM_F32 && a.r > 256 && a.r <= 512 && a.r % 8 == 0 && !a.linv_full &&
       a.linv_hi && a.in_ld == 0 && a.out_ld == 0 && (((uintptr_t)a.partials & 15) == 0) &&
       (a.partial_stride % 4 == 0))

@@ -52,6 +52,11 @@ struct SCParams {
   float shift_rel;
   float shift_diag_rel;    // each diagonal entry is also multiplied by (1 + shift_diag_rel)
   const uint32_t* gate;    // optional device word: zero means every CTA leaves at once
+  // optional: three words that receive the decision on a further orthonormalisation round
+  // { est > gate_threshold or est not finite or *dev_status != 0, est as float bits, 1 or 2 },
+  // est = sum_ij Linv_ij^2 W_jj (W_jj the diagonal as factored): trace of the inverse of the diagonally scaled matrix
+  uint32_t* gate_out;
+  float gate_threshold;
   float* linv_f32;
   __nv_bfloat16* linv_hi;
   __nv_bfloat16* linv_lo;
@@ -426,6 +431,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
   __shared__ volatile int s_urgent;                       // workers: the factorisation half is on the chain's critical path
   __shared__ volatile int s_chain_step;                   // CTA 0: what the sender warps may send
   __shared__ int s_clamped;
+  __shared__ float s_est[kCl];       // CTA 0: the workers' shares of the estimate; workers: per-warp sums
   // blocks (i, j) owned by this CTA, in column-major order
   __shared__ unsigned char s_mine_i[kMaxTri], s_mine_j[kMaxTri];
   __shared__ int s_n_mine;
@@ -726,6 +732,20 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
     // block columns of the inverse this CTA computes: j0 = cta - 1, and 7 as well on the last worker
     const int j0 = cta - 1;
     const int n_cols = (j0 < nblk ? 1 : 0) + ((cta == kWorkers && kWorkers < nblk) ? 1 : 0);
+    // for the estimate: the diagonal entries (as factored) of the one or two columns this thread writes
+    float wdiag[2] = {0.f, 0.f};
+    float est_acc = 0.f;
+    if (p.gate_out) {
+      for (int cidx = 0; cidx < n_cols; ++cidx) {
+        const int col = (j0 + cidx) * kB + (gt & 31);
+        if (col < r) {
+          float dsum = 0.f;
+          for (int q = 0; q < p.n_partials; ++q)
+            dsum += __ldg(p.partials + (int64_t)q * p.partial_stride + (int64_t)col * p.in_ld + col);
+          wdiag[cidx] = dsum + dsum * p.shift_diag_rel + s_shift;
+        }
+      }
+    }
     // zeros above the diagonal blocks
     for (int cidx = 0; cidx < n_cols; ++cidx) {
       const int j = j0 + cidx;
@@ -773,6 +793,7 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
           const int row = k * kB + a;
           if (row >= r || b >= ncol) continue;
           const float v = src[b * kLd + a];
+          est_acc = fmaf(v * v, wdiag[cidx], est_acc);
           const int64_t off = (int64_t)row * p.out_ld + j * kB + b;
           if (p.linv_f32) p.linv_f32[off] = v;
           if (p.linv_hi) {
@@ -802,11 +823,33 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
         }
       }
     }
+    if (p.gate_out) {
+      // this CTA's share of the estimate, summed in a fixed order and handed to CTA 0
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) est_acc += __shfl_xor_sync(0xffffffffu, est_acc, o);
+      if (lane == 0) s_est[warp - 8] = est_acc;
+      group_sync(2);
+      if (gt == 0) {
+        float t = 0.f;
+        for (int q = 0; q < 8; ++q) t += s_est[q];
+        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(map_to_cta(smem_addr(&s_est[cta]), 0)), "f"(t) : "memory");
+      }
+    }
   }
   __syncthreads();
   if (tid == 0 && s_gave_up && p.dev_status) atomicOr(p.dev_status, LORACT_DEV_WAIT_EXPIRED);
   // no CTA leaves while another may still write into its shared memory
   cluster_sync_all();
+  if (p.gate_out && cta == 0 && tid == 0) {
+    // after the cluster barrier: every worker's share has arrived, every status bit of this call is set
+    float est = 0.f;
+    for (int c = 1; c < kCl; ++c) est += s_est[c];
+    const uint32_t st = p.dev_status ? atomicOr(p.dev_status, 0u) : 0u;
+    const bool again = !(est <= p.gate_threshold) || st != 0u;
+    p.gate_out[0] = again ? 1u : 0u;
+    p.gate_out[1] = __float_as_uint(est);
+    p.gate_out[2] = again ? 2u : 1u;
+  }
 }
 
 // The give-up path of this file's waits, exercised on purpose: a two-CTA cluster in which CTA 1 waits, with
@@ -854,6 +897,8 @@ cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t str
   p.shift_rel = a.shift_rel;
   p.shift_diag_rel = a.shift_diag_rel;
   p.gate = a.gate;
+  p.gate_out = a.gate_out;
+  p.gate_threshold = a.gate_threshold;
   p.linv_f32 = a.linv_f32;
   p.linv_hi = a.linv_hi;
   p.linv_lo = a.linv_lo;
