@@ -207,7 +207,7 @@ constexpr int kReduceFirst = 8;    // partial count from which a separate, all-S
 // factor is D + D^T.
 cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs& w, uint32_t* status,
                    cudaStream_t stream, bool sym = false, float shift_diag = 0.f, const uint32_t* gate = nullptr,
-                   uint32_t* gate_out = nullptr, float gate_threshold = 0.f) {
+                   uint32_t* gate_out = nullptr, float gate_threshold = 0.f, bool sum_in_kernel = false) {
   SmallBlockArgs a;
   a.r = l;
   a.shift_diag_rel = shift_diag;
@@ -224,7 +224,7 @@ cudaError_t factor(int l, bool bf16, int n_partials, float shift, const BasisWs&
       // before it writes them, and no other CTA touches them (the scratch area is the factorisation's own)
       LORACT_CUDA_TRY(reduce_sym_launch(w.gram_partials, n_partials, a.partial_stride, l, w.gram_partials, stream, gate));
       a.n_partials = 1;
-    } else if (l <= 256 && n_partials >= kReduceFirst) {
+    } else if (l <= 256 && n_partials >= kReduceFirst && !sum_in_kernel) {
       // The factorisation runs on eight SMs; summing many partials there is a read of several MB through
       // eight SMs' worth of bandwidth.  All SMs sum them first (same order of additions, so the same bits).
       float* W = (float*)w.sb_scratch;
@@ -369,10 +369,29 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
   }
   trace_label("apply L^-T 1");
   LORACT_CUDA_TRY(apply(w.Yh, w.Yl, U, w.Ql, nullptr));
-  trace_label("Gram 2");
-  LORACT_CUDA_TRY(gram(U, w.Ql, gate));
-  trace_label("small block 3");
-  LORACT_CUDA_TRY(factor(l, true, w.splits_gram, kShiftSecond, w, status, stream, true, 0.f, gate));
+  if (gate_in_factor) {
+    // Round 2 is the rare path, and each of its launches costs the common path a few microseconds even when it
+    // leaves at once.  So here the Gram matrix is the plain three-term sum (no halving, no symmetrising pass) and the
+    // factorisation kernel adds the partial sums itself: three launches instead of four.  Q1 is orthonormal to a few
+    // percent, so the product of the two low parts is far below what this round corrects.
+    GemmDesc g;
+    g.M = l; g.N = l; g.K = n; g.a_mn = true; g.b_mn = true; g.lda = l; g.ldb = l;
+    g.a_type = g.b_type = el;
+    g.ldc = l;
+    g.n_terms = 3;
+    g.terms[0] = {U, U}; g.terms[1] = {U, w.Ql}; g.terms[2] = {w.Ql, U};
+    g.out = OUT_F32; g.C0 = w.gram_partials; g.splits = w.splits_gram; g.split_stride = (int64_t)l * l;
+    g.gate = gate;
+    trace_label("Gram 2");
+    LORACT_CUDA_TRY(run_gemm(g, status, stream));
+    trace_label("small block 3");
+    LORACT_CUDA_TRY(factor(l, true, w.splits_gram, kShiftSecond, w, status, stream, false, 0.f, gate, nullptr, 0.f, true));
+  } else {
+    trace_label("Gram 2");
+    LORACT_CUDA_TRY(gram(U, w.Ql, gate));
+    trace_label("small block 3");
+    LORACT_CUDA_TRY(factor(l, true, w.splits_gram, kShiftSecond, w, status, stream, true, 0.f, gate));
+  }
   trace_label("apply L^-T 2");
   // In place when one CTA (pair) owns whole rows of the product: it has read its rows of U and of the remainder
   // completely before its epilogue stores them.  With several column tiles per row block another CTA may still be
