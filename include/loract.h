@@ -88,7 +88,11 @@ loract_status_t loract_sample_indices(const loract_desc_t* desc, int32_t* idx_de
  * V = Q^T X.  (t = 0 is the setting of the paper's experiments.)
  * X: device, read only.  U (n_tokens x rank), V (rank x d): device, written.  idx_out: device, `rank`
  * int32, written if not NULL.  U has orthonormal columns; U V is the orthogonal projection of X onto
- * range(Y).  The entries of U are not unique (any orthonormal basis of range(Y) is a valid result). */
+ * range(Y).  The entries of U are not unique (any orthonormal basis of range(Y) is a valid result).
+ * The QR step is done through the Gram matrix of the sketch (Y^T Y = L L^T, Q = Y L^-T); it is repeated once on
+ * Q when a condition estimate formed on the device says that one round does not reach max|U^T U - I| <= 1e-3
+ * (or when a status bit is set): same subspace either way, no host synchronisation, and the choice is a
+ * deterministic function of the input. */
 loract_status_t loract_compress(const loract_desc_t* desc, const void* X, void* U, void* V,
                                 int32_t* idx_out, void* ws, size_t ws_bytes, void* stream);
 
