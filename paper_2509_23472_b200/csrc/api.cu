@@ -686,7 +686,10 @@ loract_status_t loract_weight_grad(const loract_desc_t* desc, const void* U, con
   t.out = OUT_F32; t.C0 = w.partials; t.ldc = g; t.splits = w.splits; t.split_stride = (int64_t)r * g;
   uint32_t* status = (uint32_t*)ws;
   trace_label("weight grad");
-  cudaError_t e = cudaMemsetAsync(status, 0, 4, st);
+  // the first kernel clears the status word itself where it can (tensor-core path); a memset node otherwise
+  cudaError_t e = cudaSuccess;
+  if (gemm_tc_supported(t)) t.clear_status = true;
+  else e = cudaMemsetAsync(status, 0, 4, st);
   if (e == cudaSuccess) e = run_gemm(t, status, st);
   if (e == cudaSuccess && el == ELEM_BF16) {
     // dW = V^T T on the tensor cores: T (fp32) is carried as a bf16 triple, so that the three products

@@ -110,6 +110,9 @@ struct GemmDesc {
   // Tensor-core path: a device word written by an earlier kernel of the same stream; when it is zero the launch
   // does nothing (no loads, no products, C untouched).  nullptr: unconditional.
   const uint32_t* gate = nullptr;
+  // Tensor-core path: the launch stores zero into the status word before any of its waits can set a bit in it (the
+  // first kernel of a call clears the word itself instead of a memset in front of it).
+  bool clear_status = false;
 };
 
 // tcgen05 engine: bf16 operands, fp32 accumulation in tensor memory.  Returns cudaErrorNotSupported
@@ -217,7 +220,7 @@ cudaError_t reduce_sym_launch(const float* partials, int n_partials, int64_t str
 // which lies between 1 / lambda_min and r / lambda_min of the diagonally scaled Gram matrix, the quantity that
 // multiplies the rounding error of W in the orthogonality defect of Y L^-T.  gate_words[0] = 1 if est > threshold, est is
 // not finite, or the status word is non-zero (a clamped pivot, a non-finite input), else 0; gate_words[1] = est
-// (float bits); gate_words[2] = rounds that will run (1 or 2).  One CTA, fixed summation order.
+// (float bits); gate_words[2] = rounds that will run (1 or 2).  One cluster of eight CTAs, fixed summation order.
 cudaError_t round_gate_launch(const float* W, const __nv_bfloat16* linv_hi, int r, float threshold,
                               const uint32_t* dev_status, uint32_t* gate_words, cudaStream_t stream);
 // dst = src (count bf16 elements, both 16-byte aligned, count a multiple of 8) when *gate != 0; nothing otherwise.

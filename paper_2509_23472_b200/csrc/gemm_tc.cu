@@ -69,6 +69,10 @@ struct TcParams {
   // one-tile kernels: when set and the word it points to is zero, the kernel loads, multiplies and stores nothing
   // (a step that an earlier kernel of the same stream found unnecessary)
   const uint32_t* gate;
+  // one-tile kernels: block (0, 0, 0) stores zero into *dev_status right after griddepcontrol.wait (for the first
+  // kernel of a call: no memset node in front of the chain).  A bounded wait of this kernel can set a bit two seconds
+  // later at the earliest, long after that store.
+  int clear_status;
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -549,6 +553,8 @@ gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   pdl_wait();
   pdl_launch_dependents();
   if (p.gate != nullptr && *(const volatile uint32_t*)p.gate == 0u) n_iter = -1;   // every role idles, nothing is stored
+  if (p.clear_status && p.dev_status && threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+    *(volatile uint32_t*)p.dev_status = 0u;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -728,6 +734,8 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   pdl_wait();
   pdl_launch_dependents();
   if (p.gate != nullptr && *(const volatile uint32_t*)p.gate == 0u) n_iter = -1;   // every role idles, nothing is stored
+  if (p.clear_status && p.dev_status && threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+    *(volatile uint32_t*)p.dev_status = 0u;
 
   if (warp == 0 || warp == 2) {
     if (lane == 0) {
@@ -1291,6 +1299,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   p.halve_at_term = g.halve_at_term > 0 ? g.halve_at_term : 0;
   p.a_keep_from_kb = g.a_keep_from_k >= 0 ? (int)(g.a_keep_from_k / kBK) : p.kb_total;
   p.gate = g.gate;
+  p.clear_status = g.clear_status ? 1 : 0;
 
   TmapPack maps;
   for (int t = 0; t < g.n_terms; ++t) {
@@ -1325,7 +1334,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   // Short contraction, large output, A K-major, B MN-major, one term (Reconstruct and the pre-norm backward):
   // the persistent kernel with B resident, when there is more than one tile per resident pair.
   if (g_pair_mode == 1 && g.M >= 2 * kBM && !g.a_mn && g.b_mn && g.n_terms == 1 && splits == 1 && p.kb_total <= 8 &&
-      g.N >= 256 && g.gate == nullptr) {
+      g.N >= 256 && g.gate == nullptr && !g.clear_status) {
     TcParams sp = p;
     // 256 columns per tile (the tensor pipe is issue-bound on narrower instructions).  The resident B takes
     // 16 KB per K block and CTA; beyond four K blocks the A ring and the staging boxes shrink to make room

@@ -512,30 +512,38 @@ cudaError_t launch_simt_typed(const SimtParams& p, bool acc64, cudaStream_t stre
   return cudaGetLastError();
 }
 
-// Decision after the first orthonormalisation round (see round_gate_launch in common.cuh).  One CTA of 1024
-// threads; a thread takes 8 consecutive elements of L^-1 (one 16-byte load) at a time, every sum in a fixed order.
+// Decision after the first orthonormalisation round (see round_gate_launch in common.cuh).  One cluster of
+// kGateCtas CTAs of 1024 threads; CTA c takes the rows c, c + kGateCtas, ...; a thread takes 8 consecutive elements of
+// L^-1 (one 16-byte load) at a time.  Every CTA stores its sum into the shared memory of CTA 0, which adds them in
+// rank order after the cluster barrier: a fixed summation order, no state in global memory.
+constexpr int kGateCtas = 8;
 __global__ void __launch_bounds__(1024) round_gate_kernel(const float* __restrict__ W,
                                                           const __nv_bfloat16* __restrict__ linv_hi, int r,
                                                           float threshold, const uint32_t* dev_status,
                                                           uint32_t* gate_words) {
   __shared__ float s_diag[640];
   __shared__ float s_red[32];
+  __shared__ float s_parts[kGateCtas];
+  uint32_t rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   pdl_wait();
   pdl_launch_dependents();
   for (int j = tid; j < r; j += 1024) s_diag[j] = W[(int64_t)j * r + j];
   __syncthreads();
   float acc = 0.f;
-  const int64_t count = (int64_t)r * r;   // r is a multiple of 8, so a group of 8 stays inside one row
-  for (int64_t e = (int64_t)tid * 8; e < count; e += 1024 * 8) {
-    const int row = (int)(e / r), col = (int)(e - (int64_t)row * r);
-    if (col > row) continue;              // strictly above the diagonal: zeros
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(linv_hi + e));
-    const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+  const int groups_per_row = r / 8;       // r is a multiple of 8, so a group of 8 stays inside one row
+  // a warp per row: 32 lanes cover 256 columns per step
+  for (int row = (int)rank + kGateCtas * warp; row < r; row += kGateCtas * 32) {
+    for (int gidx = lane; gidx < groups_per_row && gidx * 8 <= row; gidx += 32) {   // groups that start at or below the diagonal
+      const int col = gidx * 8;
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(linv_hi + (int64_t)row * r + col));
+      const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const float lo = __uint_as_float(w4[q] << 16), hi = __uint_as_float(w4[q] & 0xffff0000u);
-      acc += lo * lo * s_diag[col + 2 * q] + hi * hi * s_diag[col + 2 * q + 1];
+      for (int q = 0; q < 4; ++q) {
+        const float lo = __uint_as_float(w4[q] << 16), hi = __uint_as_float(w4[q] & 0xffff0000u);
+        acc += lo * lo * s_diag[col + 2 * q] + hi * hi * s_diag[col + 2 * q + 1];
+      }
     }
   }
 #pragma unroll
@@ -543,8 +551,17 @@ __global__ void __launch_bounds__(1024) round_gate_kernel(const float* __restric
   if (lane == 0) s_red[warp] = acc;
   __syncthreads();
   if (tid == 0) {
+    float part = 0.f;
+    for (int q = 0; q < 32; ++q) part += s_red[q];
+    uint32_t local = (uint32_t)__cvta_generic_to_shared(&s_parts[rank]), remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(0));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(part) : "memory");
+  }
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  if (rank == 0 && tid == 0) {
     float est = 0.f;
-    for (int q = 0; q < 32; ++q) est += s_red[q];
+    for (int q = 0; q < kGateCtas; ++q) est += s_parts[q];
     const uint32_t st = dev_status ? *(const volatile uint32_t*)dev_status : 0u;
     const bool again = !(est <= threshold) || st != 0u;   // a NaN estimate compares false: second round
     gate_words[0] = again ? 1u : 0u;
@@ -622,8 +639,21 @@ cudaError_t reduce_sym_launch(const float* partials, int n_partials, int64_t str
 cudaError_t round_gate_launch(const float* W, const __nv_bfloat16* linv_hi, int r, float threshold,
                               const uint32_t* dev_status, uint32_t* gate_words, cudaStream_t stream) {
   if (r < 8 || r > 640 || r % 8 || ((uintptr_t)linv_hi & 15)) return cudaErrorInvalidValue;
-  LORACT_CUDA_TRY(launch_pdl(round_gate_kernel, dim3(1), dim3(1024), 0, stream, W, linv_hi, r, threshold, dev_status,
-                             gate_words));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kGateCtas, 1, 1);
+  cfg.blockDim = dim3(1024, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kGateCtas;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  LORACT_CUDA_TRY(cudaLaunchKernelEx(&cfg, round_gate_kernel, W, linv_hi, r, threshold, dev_status, gate_words));
   count_launch(__func__, stream);
   return cudaGetLastError();
 }
