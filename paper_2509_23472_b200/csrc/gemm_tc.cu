@@ -1265,14 +1265,41 @@ bool gemm_tc_supported(const GemmDesc& g) {
   return true;
 }
 
-int gemm_tc_pick_splits(int M, int N, int K, bool, bool, int max_splits) {
-  const int tiles = ((M + kBM - 1) / kBM) * ((N + pick_bn(N) - 1) / pick_bn(N));
+int gemm_tc_pick_splits(int M, int N, int K, bool, bool b_mn, int max_splits) {
+  const int bn = pick_bn(N);
+  const int n_tiles = (N + bn - 1) / bn;
+  const int tiles = ((M + kBM - 1) / kBM) * n_tiles;
   const int kb = (K + kBK - 1) / kBK;
-  if (tiles >= 96) return 1;
-  int s = 148 / tiles;
-  if (s > kb / 4) s = kb / 4;  // at least four K blocks per split
-  if (s > max_splits) s = max_splits;
-  return s < 1 ? 1 : s;
+  int base = 1;
+  if (tiles < 96) {
+    base = 148 / tiles;
+    if (base > kb / 4) base = kb / 4;  // at least four K blocks per split
+    if (base > max_splits) base = max_splits;
+    if (base < 1) base = 1;
+  }
+  // Whole waves: with U units of work on S slots the launch takes ceil(U / S) rounds, so 86 tile pairs on 74 SM
+  // pairs cost two full rounds.  Splitting the contraction s ways makes the rounds shorter and fills the last one;
+  // it costs the partial sums (s * M * N * 4 bytes, read back by the reduction).  Time in units of one
+  // K block (about 0.35 us for a 256 x 256 pair tile); the split count of the simple rule above is kept unless
+  // another one is at least 15 % cheaper.
+  const bool pair = M >= 2 * kBM && (b_mn ? bn % 128 == 0 : bn % 32 == 0);   // by shape (not by the test hook)
+  const long long units = pair ? (long long)((M + 2 * kBM - 1) / (2 * kBM)) * n_tiles : tiles;
+  const int slots = pair ? 74 : 148;
+  auto cost = [&](int sp) {
+    const double rounds = (double)((units * sp + slots - 1) / slots);
+    // the partial sums are read back once by the reduction (about 4 TB/s) behind one more launch
+    const double reduce_us = sp > 1 ? (double)sp * (double)M * (double)N * 4.0 / 4.0e6 + 4.0 : 0.0;
+    return rounds * (double)((kb + sp - 1) / sp) + reduce_us / 0.35;
+  };
+  int best = base;
+  double best_cost = cost(base);
+  const int cap = max_splits < 8 ? max_splits : 8;
+  for (int sp = 1; sp <= cap; ++sp) {
+    if (sp > 1 && kb / sp < 4) break;
+    const double c = cost(sp);
+    if (c < best_cost && c < 0.85 * cost(base)) { best = sp; best_cost = c; }
+  }
+  return best;
 }
 
 cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t stream) {
