@@ -1299,7 +1299,11 @@ int gemm_tc_pick_splits(int M, int N, int K, bool, bool b_mn, int max_splits) {
     const double c = cost(sp);
     if (c < best_cost && c < 0.85 * cost(base)) { best = sp; best_cost = c; }
   }
-  return best;
+  // no empty split: with ceil(kb / best) K blocks each, fewer splits may already cover the contraction (197 blocks
+  // in 32 splits of 7 leave three splits with nothing to do but write zeros)
+  const int per = (kb + best - 1) / best;
+  best = (kb + per - 1) / per;
+  return best < 1 ? 1 : best;
 }
 
 cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t stream) {
