@@ -341,7 +341,8 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
     g.gate = gt;
     return run_gemm(g, status, stream);
   };
-  auto apply = [&](const void* Yh, const void* Yl, void* Ch, void* Cl, const uint32_t* gt) {
+  auto apply = [&](const void* Yh, const void* Yl, void* Ch, void* Cl, const uint32_t* gt,
+                   const uint32_t* lo_gt = nullptr) {
     // C[m][j] = sum_k Y[m][k] Linv[j][k]
     GemmDesc g;
     g.M = n; g.N = l; g.K = l; g.lda = l; g.ldb = l; g.a_type = g.b_type = el;
@@ -350,6 +351,7 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
     g.terms[0] = {Yh, w.Lh}; g.terms[1] = {Yh, w.Ll}; g.terms[2] = {Yl, w.Lh};
     if (Cl) { g.out = OUT_SPLIT; g.C0 = Ch; g.C1 = Cl; } else { g.out = OUT_BF16; g.C0 = Ch; }
     g.gate = gt;
+    g.lo_gate = lo_gt;
     return run_gemm(g, status, stream);
   };
   trace_label("Gram 1");
@@ -368,7 +370,9 @@ cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* O
     LORACT_CUDA_TRY(round_gate_launch(w.gram_partials, w.Lh, l, threshold, status, gate_words, stream));
   }
   trace_label("apply L^-T 1");
-  LORACT_CUDA_TRY(apply(w.Yh, w.Yl, U, w.Ql, nullptr));
+  // the remainder of Q1 is only read by the second round: not written when the decision (taken before this kernel
+  // starts) is that one round is enough
+  LORACT_CUDA_TRY(apply(w.Yh, w.Yl, U, w.Ql, nullptr, gate));
   if (gate_in_factor) {
     // Round 2 is the rare path, and each of its launches costs the common path a few microseconds even when it
     // leaves at once.  So here the Gram matrix is the plain three-term sum (no halving, no symmetrising pass) and the

@@ -113,6 +113,9 @@ struct GemmDesc {
   // Tensor-core path: the launch stores zero into the status word before any of its waits can set a bit in it (the
   // first kernel of a call clears the word itself instead of a memset in front of it).
   bool clear_status = false;
+  // Tensor-core path, OUT_SPLIT: a device word written by an earlier kernel; when it is zero only C0 (the leading bf16
+  // part) is written and C1 keeps its old contents.
+  const uint32_t* lo_gate = nullptr;
 };
 
 // tcgen05 engine: bf16 operands, fp32 accumulation in tensor memory.  Returns cudaErrorNotSupported

@@ -73,6 +73,8 @@ struct TcParams {
   // kernel of a call: no memset node in front of the chain).  A bounded wait of this kernel can set a bit two seconds
   // later at the earliest, long after that store.
   int clear_status;
+  // one-tile kernels, OUT_SPLIT: when set and the word is zero, the low part (C1) is not written
+  const uint32_t* lo_gate;
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -259,7 +261,7 @@ __device__ __forceinline__ void stage_drain(const StoreStage& st, int lane) {
 
 __device__ __forceinline__ void tc_store_tile_staged(const TcParams& p, const TmapPack& maps, uint32_t tmem_base,
                                                      int quad, int half_id, int lane, int m0, int n0,
-                                                     int split, StoreStage& st) {
+                                                     int split, StoreStage& st, bool lo_on = true) {
   const int row0 = m0 + quad * 32;
   const int m = row0 + lane;
   const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
@@ -278,7 +280,7 @@ __device__ __forceinline__ void tc_store_tile_staged(const TcParams& p, const Tm
     }
     return;
   }
-  const bool split_out = p.out == OUT_SPLIT;
+  const bool split_out = p.out == OUT_SPLIT && lo_on;   // lo_on false: only the leading part is wanted
   const bool rms = p.out == OUT_RMS_BWD;
   const bool act = p.out == OUT_ACT_BWD;
   const bool live = m < p.M;                                 // rows past M are clipped by the store
@@ -388,7 +390,7 @@ __device__ __forceinline__ void tc_store_tile_staged(const TcParams& p, const Tm
 // Writes one finished accumulator tile (128 rows of this CTA x bn columns, starting at tensor-memory column
 // tmem_base) in the output mode of p.  Warp w may touch the lanes 32 * (w % 4) .. + 31.
 __device__ __forceinline__ void tc_store_tile(const TcParams& p, const TmapPack& maps, uint32_t tmem_base, int warp,
-                                              int lane, int m0, int n0, int split, StoreStage& st) {
+                                              int lane, int m0, int n0, int split, StoreStage& st, bool lo_on = true) {
   const int quad = warp & 3;
   const int half_id = (warp - 2) >> 2;                       // which of the two warps of this quarter
   const int row = quad * 32 + lane;
@@ -397,7 +399,7 @@ __device__ __forceinline__ void tc_store_tile(const TcParams& p, const TmapPack&
   // staged unless the output needs read-modify-write, or (split-K partials stacked along the rows of one
   // tensor map) the warp's 32 rows are not all inside M
   if (st.base && p.tma_store && !p.accumulate && (p.split_stride == 0 || m0 + quad * 32 + 32 <= p.M)) {
-    tc_store_tile_staged(p, maps, tmem_base, quad, half_id, lane, m0, n0, split, st);
+    tc_store_tile_staged(p, maps, tmem_base, quad, half_id, lane, m0, n0, split, st, lo_on);
     return;
   }
   {
@@ -458,7 +460,7 @@ __device__ __forceinline__ void tc_store_tile(const TcParams& p, const TmapPack&
           dst[q] = __float2bfloat16(__bfloat162float(e[q]) * act_derivative(__uint_as_float(v[q]), p.ep_kind));
       } else {
         __nv_bfloat16* dst_hi = (__nv_bfloat16*)p.C0 + (int64_t)m * p.ldc + n;
-        __nv_bfloat16* dst_lo = (p.out == OUT_SPLIT) ? (__nv_bfloat16*)p.C1 + (int64_t)m * p.ldc + n : nullptr;
+        __nv_bfloat16* dst_lo = (p.out == OUT_SPLIT && lo_on) ? (__nv_bfloat16*)p.C1 + (int64_t)m * p.ldc + n : nullptr;
         if (valid == 32 && ((((uintptr_t)dst_hi) & 15) == 0)) {
           uint32_t hi[16], lo[16];
 #pragma unroll
@@ -496,6 +498,8 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const TmapPack& m
                                           uint64_t* accum_bar, volatile int* abort_flag_ptr, int warp, int lane,
                                           int m0, int n0, int split, int n_iter, unsigned char* ring) {
   const int m = m0 + (warp & 3) * 32 + lane;
+  // OUT_SPLIT with a gate on the low part: read the word while the contraction is still running
+  const bool lo_on = !(p.lo_gate != nullptr && *(const volatile uint32_t*)p.lo_gate == 0u);
   bool ok = mbar_wait_bounded(accum_bar, 0, abort_flag_ptr);
   ok = __all_sync(0xffffffffu, ok);
   tc_fence_after();
@@ -504,7 +508,7 @@ __device__ __forceinline__ void tc_epilogue(const TcParams& p, const TmapPack& m
     st.base = ring + (uint32_t)(warp - 2) * kStoreWarpBytes;
     st.cnt = 0;
     st.bufs = kStoreBufs;
-    tc_store_tile(p, maps, tmem_base, warp, lane, m0, n0, split, st);
+    tc_store_tile(p, maps, tmem_base, warp, lane, m0, n0, split, st, lo_on);
     stage_drain(st, lane);
   } else if (ok && n_iter == 0 && m < p.M && p.out == OUT_F32 && warp < 6) {
     // an empty K range still owns its partial: write zeros
@@ -1331,6 +1335,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   p.a_keep_from_kb = g.a_keep_from_k >= 0 ? (int)(g.a_keep_from_k / kBK) : p.kb_total;
   p.gate = g.gate;
   p.clear_status = g.clear_status ? 1 : 0;
+  p.lo_gate = g.lo_gate;
 
   TmapPack maps;
   for (int t = 0; t < g.n_terms; ++t) {
@@ -1365,7 +1370,7 @@ cudaError_t gemm_tc_launch(const GemmDesc& g, uint32_t* dev_status, cudaStream_t
   // Short contraction, large output, A K-major, B MN-major, one term (Reconstruct and the pre-norm backward):
   // the persistent kernel with B resident, when there is more than one tile per resident pair.
   if (g_pair_mode == 1 && g.M >= 2 * kBM && !g.a_mn && g.b_mn && g.n_terms == 1 && splits == 1 && p.kb_total <= 8 &&
-      g.N >= 256 && g.gate == nullptr && !g.clear_status) {
+      g.N >= 256 && g.gate == nullptr && !g.clear_status && g.lo_gate == nullptr) {
     TcParams sp = p;
     // 256 columns per tile (the tensor pipe is issue-bound on narrower instructions).  The resident B takes
     // 16 KB per K block and CTA; beyond four K blocks the A ring and the staging boxes shrink to make room
