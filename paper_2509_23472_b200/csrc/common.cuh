@@ -107,8 +107,9 @@ struct GemmDesc {
   // (result = (t_0 + ... + t_{h-1}) / 2 + t_h + ...); 0 or negative: plain sum.  With the pair {A^T A, A^T B} and
   // h = 1 the result D gives D + D^T = A^T A + A^T B + B^T A: a symmetric three-term sum for two terms' work.
   int halve_at_term = 0;
-  // Tensor-core path: a device word written by an earlier kernel of the same stream; when it is zero the launch
-  // does nothing (no loads, no products, C untouched).  nullptr: unconditional.
+  // Tensor-core path: a device word written by a kernel at least TWO launches earlier in the same stream (the gated
+  // kernel reads it before its griddepcontrol.wait); when it is zero the launch does nothing (no loads, no products,
+  // C untouched).  nullptr: unconditional.
   const uint32_t* gate = nullptr;
   // Tensor-core path: the launch stores zero into the status word before any of its waits can set a bit in it (the
   // first kernel of a call clears the word itself instead of a memset in front of it).

@@ -536,6 +536,12 @@ gemm_tc_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   // dynamic shared memory is declared 1024-aligned; round up anyway (swizzle atoms need it)
   unsigned char* tiles = (unsigned char*)(((uintptr_t)smem + 1023) & ~(uintptr_t)1023);
 
+  // A gated launch that is not needed leaves before any set-up.  The word may be read this early because it was
+  // written at least two kernels back in the stream: this grid only starts once its predecessor has passed its own
+  // griddepcontrol.wait, i.e. once everything before the predecessor is complete and visible.  The wait itself is
+  // still executed, so that the completion of this grid implies the completion of every earlier one.
+  if (p.gate != nullptr && *(const volatile uint32_t*)p.gate == 0u) { pdl_wait(); pdl_launch_dependents(); return; }
+
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     mbar_init(&accum_bar, 1);
@@ -714,6 +720,10 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   int n_iter = kb_count * p.n_terms;
   const uint32_t stage_bytes = kABytes + p.b_bytes;          // per CTA (b_bytes: half a B tile)
   unsigned char* tiles = (unsigned char*)(((uintptr_t)smem + 1023) & ~(uintptr_t)1023);
+
+  // a gated launch that is not needed: both CTAs of the pair read the same word and leave before any set-up (see the
+  // one-CTA kernel for why the word may be read before griddepcontrol.wait)
+  if (p.gate != nullptr && *(const volatile uint32_t*)p.gate == 0u) { pdl_wait(); pdl_launch_dependents(); return; }
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kPairStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }

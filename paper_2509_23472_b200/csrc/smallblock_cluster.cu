@@ -449,6 +449,12 @@ __global__ void __launch_bounds__(kCThreads, 1) small_block_cluster_kernel(SCPar
   const int nblk = (r + kB - 1) / kB;
   const int ntri = nblk * (nblk + 1) / 2;
 
+  // A gated launch that is not needed leaves before any set-up: the same word in every CTA of the cluster, written at
+  // least two kernels back in the stream (this grid only starts once its predecessor has passed its own
+  // griddepcontrol.wait), so it may be read this early.  The wait is still executed: the completion of this grid
+  // must imply the completion of every earlier one.
+  if (p.gate != nullptr && *(const volatile uint32_t*)p.gate == 0u) { pdl_wait(); pdl_launch_dependents(); return; }
+
   // ---- set-up, spread over threads: barriers (with the byte counts they will receive, known up front),
   // this CTA's block list, the sentinel words of the diagonal-block column buffer
   if (tid < kMaxBlk) {
