@@ -216,17 +216,21 @@ __global__ void reduce_split3_kernel(const float* __restrict__ partials, int n_p
 }
 
 // fp32 product for the r x r blocks of the two-level small-block scheme: C = alpha * A B (+ C), all of a few
-// hundred rows and columns.  32 x 32 output tiles on 64 threads (4 x 4 outputs each, operands read from
-// shared memory along the contraction index with 16-byte loads), so that a 256 x 256 product spreads over
-// 64 SMs; the K loop is double-buffered through registers.  One launch carries up to two independent products
+// hundred rows and columns.  32 x 32 output tiles, four groups of 64 threads per tile, each group on a quarter of
+// the contraction (4 x 4 outputs per thread, operands read from shared memory along the contraction index with
+// 16-byte loads; the four partial tiles are added in group order), so that a 256 x 256 product spreads over
+// 64 SMs and no thread walks more than a quarter of K; the K loop is double-buffered through registers.  One launch carries up to two independent products
 // (grid.z picks one): the two-level scheme has a pair of them at one point of its chain.
 constexpr int kT32 = 32, kT32Ld = 36;
 
-__global__ void __launch_bounds__(64) gemm_f32_tile32_kernel(SimtParams p0, SimtParams p1) {
-  __shared__ __align__(16) float As[kT32 * kT32Ld];   // [m][k]
-  __shared__ __align__(16) float Bs[kT32 * kT32Ld];   // [n][k]
+constexpr int kT32Groups = 4;   // thread groups of 64 that share one output tile, each on a quarter of the contraction
+__global__ void __launch_bounds__(64 * kT32Groups) gemm_f32_tile32_kernel(SimtParams p0, SimtParams p1) {
+  // per group: As [m][k] and Bs [n][k]; after the K loop the same memory carries the partial tiles of groups 1..3
+  __shared__ __align__(16) float tiles[kT32Groups][2][kT32 * kT32Ld];
   const SimtParams& p = blockIdx.z ? p1 : p0;
-  const int tid = threadIdx.x;
+  const int grp = threadIdx.x >> 6, tid = threadIdx.x & 63;
+  float* As = tiles[grp][0];
+  float* Bs = tiles[grp][1];
   const int m0 = blockIdx.y * kT32, n0 = blockIdx.x * kT32;
   pdl_wait();
   pdl_launch_dependents();
@@ -235,6 +239,10 @@ __global__ void __launch_bounds__(64) gemm_f32_tile32_kernel(SimtParams p0, Simt
   const int tm = tid >> 3, tn = tid & 7;               // outputs (4 tm + i, tn + 8 j)
   const float* A = (const float*)p.A[0];
   const float* B = (const float*)p.B[0];
+  // this group's share of the contraction: whole chunks of 32, the same number of chunks in every group
+  const int chunks = ((p.K + kT32 - 1) / kT32 + kT32Groups - 1) / kT32Groups;
+  const int k_begin = grp * chunks * kT32;
+  const int k_end = min(p.K, k_begin + chunks * kT32);
   float acc[4][4];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
@@ -249,11 +257,11 @@ __global__ void __launch_bounds__(64) gemm_f32_tile32_kernel(SimtParams p0, Simt
       int mm, kk;
       if (p.sak == 1) { kk = e & 31; mm = e >> 5; } else { mm = e & 31; kk = e >> 5; }
       const int m = m0 + mm, k = k0 + kk;
-      ra[u] = (m < p.M && k < p.K) ? A[m * p.sam + k * p.sak] : 0.f;
+      ra[u] = (m < p.M && k < k_end) ? A[m * p.sam + k * p.sak] : 0.f;
       int nn, kb;
       if (p.sbk == 1) { kb = e & 31; nn = e >> 5; } else { nn = e & 31; kb = e >> 5; }
       const int n = n0 + nn, k2 = k0 + kb;
-      rb[u] = (n < p.N && k2 < p.K) ? B[k2 * p.sbk + n * p.sbn] : 0.f;
+      rb[u] = (n < p.N && k2 < k_end) ? B[k2 * p.sbk + n * p.sbn] : 0.f;
     }
   };
   auto stash = [&]() {
@@ -268,12 +276,14 @@ __global__ void __launch_bounds__(64) gemm_f32_tile32_kernel(SimtParams p0, Simt
       Bs[nn * kT32Ld + kb] = rb[u];
     }
   };
-  fetch(0);
-  for (int k0 = 0; k0 < p.K; k0 += kT32) {
-    __syncthreads();
+  auto group_barrier = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(grp + 1) : "memory"); };
+  fetch(k_begin);
+  for (int c = 0; c < chunks; ++c) {
+    const int k0 = k_begin + c * kT32;
+    group_barrier();
     stash();
-    __syncthreads();
-    if (k0 + kT32 < p.K) fetch(k0 + kT32);
+    group_barrier();
+    if (c + 1 < chunks) fetch(k0 + kT32);
 #pragma unroll
     for (int q4 = 0; q4 < kT32 / 4; ++q4) {
       float4 a[4], b[4];
@@ -292,6 +302,16 @@ __global__ void __launch_bounds__(64) gemm_f32_tile32_kernel(SimtParams p0, Simt
         }
     }
   }
+  // the quarters of the contraction meet in shared memory and are added in group order
+  group_barrier();   // this group has finished reading its tiles
+  if (grp > 0) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) As[(4 * tm + i) * kT32Ld + tn + 8 * j] = acc[i][j];
+  }
+  __syncthreads();
+  if (grp > 0) return;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int m = m0 + 4 * tm + i;
@@ -300,8 +320,11 @@ __global__ void __launch_bounds__(64) gemm_f32_tile32_kernel(SimtParams p0, Simt
     for (int j = 0; j < 4; ++j) {
       const int n = n0 + tn + 8 * j;
       if (n >= p.N) continue;
+      float sum = acc[i][j];
+#pragma unroll
+      for (int g2 = 1; g2 < kT32Groups; ++g2) sum += tiles[g2][0][(4 * tm + i) * kT32Ld + tn + 8 * j];
       float* c = (float*)p.C0 + (int64_t)m * p.ldc + n;
-      const float v = acc[i][j] * p.alpha;
+      const float v = sum * p.alpha;
       *c = p.accumulate ? (*c + v) : v;
     }
   }
@@ -715,7 +738,7 @@ cudaError_t gemm_f32_small_launch(const GemmDesc& g, cudaStream_t stream, const 
   p0.gate = p1.gate = g.gate;
   const int M = second ? std::max(g.M, second->M) : g.M, N = second ? std::max(g.N, second->N) : g.N;
   dim3 grid((N + kT32 - 1) / kT32, (M + kT32 - 1) / kT32, second ? 2 : 1);
-  LORACT_CUDA_TRY(launch_pdl(gemm_f32_tile32_kernel, grid, dim3(64), 0, stream, p0, p1));
+  LORACT_CUDA_TRY(launch_pdl(gemm_f32_tile32_kernel, grid, dim3(64 * kT32Groups), 0, stream, p0, p1));
   count_launch(__func__, stream);
   return cudaGetLastError();
 }
