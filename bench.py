@@ -350,6 +350,8 @@ def main():
     # clears the word at its start, so it is read between the two calls here)
     B.compress(Xs[0], r, ws=ws, out=(U, V, idx), desc=desc)
     status_compress = B.read_device_status(ws)
+    # what the device decided about the second orthonormalisation round, and the estimate it decided on
+    second_round, orth_estimate, orth_rounds = B.round_gate_words(ws) if w.dtype == "bf16" else (1, float("nan"), 2)
     B.weight_grad(U, V, Gs[0], dW=dW, ws=ws)
     status_wgrad = B.read_device_status(ws)
 
@@ -500,6 +502,7 @@ def main():
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": X.numel() * es + G.numel() * es,
                 "d2h_bytes_per_step": dW.numel() * 4, "ms_per_step": e2e_ms / e2e_steps},
         "gpu_launches": int(launches), "gpu_launches_per_step": int(launches) // n_timed, "device_status": status_compress, "device_status_weight_grad": status_wgrad,
+        "orthonormalisation": {"rounds": orth_rounds, "estimate_trace_inv_scaled_gram": orth_estimate},
         "clocks": clocks,
         "roofline": rooflines[0] if rooflines else None, "rooflines": rooflines, "cpu_baseline": cpu,
     }

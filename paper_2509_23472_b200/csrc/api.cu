@@ -264,7 +264,8 @@ cudaError_t precondition_rows(const void* T, int l, int64_t d, bool bf16, void* 
 }
 
 // The sketch and the orthonormalisation of Algorithm 1 for a test matrix Omega (l x d, rows are the test vectors):
-// Y = X Omega^T, then two rounds of { W = Y^T Y = L L^T ; Y <- Y L^{-T} }.  U (n x l) receives Q.
+// Y = X Omega^T, then { W = Y^T Y = L L^T ; Y <- Y L^{-T} }, once or (decided on the device, bf16 inputs) twice.
+// U (n x l) receives Q.
 cudaError_t range_basis(const void* X, int64_t ldx, const Plan& p, const void* Omega, void* U,
                         const BasisWs& w, uint32_t* status, cudaStream_t stream) {
   const int l = p.l;

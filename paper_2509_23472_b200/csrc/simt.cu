@@ -149,6 +149,37 @@ __global__ void reduce_partials_kernel(const float* __restrict__ partials, int n
   }
 }
 
+// The same sums four elements at a time (16-byte loads, all partials of a quad in flight together): `count4` quads,
+// everything 16-byte aligned, stride a multiple of four.  Same order of additions per element as the scalar kernel.
+__global__ void __launch_bounds__(256) reduce_partials_vec4_kernel(const float4* __restrict__ partials, int n_partials,
+                                                                   int64_t stride4, int64_t count4,
+                                                                   float4* __restrict__ out_f32,
+                                                                   uint2* __restrict__ out_bf16, const uint32_t* gate) {
+  pdl_wait();
+  pdl_launch_dependents();
+  if (gate != nullptr && *(const volatile uint32_t*)gate == 0u) return;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < count4;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    int q = 0;
+    for (; q + 4 <= n_partials; q += 4) {
+      const float4 a = partials[(int64_t)q * stride4 + i], b = partials[(int64_t)(q + 1) * stride4 + i];
+      const float4 c = partials[(int64_t)(q + 2) * stride4 + i], d = partials[(int64_t)(q + 3) * stride4 + i];
+      s.x = (((s.x + a.x) + b.x) + c.x) + d.x; s.y = (((s.y + a.y) + b.y) + c.y) + d.y;
+      s.z = (((s.z + a.z) + b.z) + c.z) + d.z; s.w = (((s.w + a.w) + b.w) + c.w) + d.w;
+    }
+    for (; q < n_partials; ++q) {
+      const float4 a = partials[(int64_t)q * stride4 + i];
+      s.x += a.x; s.y += a.y; s.z += a.z; s.w += a.w;
+    }
+    if (out_f32) out_f32[i] = s;
+    if (out_bf16) {
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(s.x, s.y), hi = __floats2bfloat162_rn(s.z, s.w);
+      out_bf16[i] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+    }
+  }
+}
+
 // out = S + S^T with S = sum_s partials[s] (fixed order), for r x r matrices: the tall Gram products are formed as
 // D = Yh^T Yh / 2 + Yh^T Yl (two terms), and D + D^T = Yh^T Yh + Yh^T Yl + Yl^T Yh is the three-term Gram matrix,
 // exactly symmetric.  One CTA per pair of 16 x 16 tiles (I, J), (J, I), I >= J: both tiles are summed with
@@ -641,6 +672,18 @@ cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t stream) {
 cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_t stride,
                                    int64_t count, float* out_f32, __nv_bfloat16* out_bf16,
                                    cudaStream_t stream, const uint32_t* gate) {
+  const bool vec = count % 4 == 0 && stride % 4 == 0 && (((uintptr_t)partials | (uintptr_t)out_f32) & 15) == 0 &&
+                   ((uintptr_t)out_bf16 & 7) == 0;
+  if (vec) {
+    const int64_t count4 = count / 4;
+    int grid = (int)((count4 + 255) / 256);
+    if (grid > 148 * 8) grid = 148 * 8;
+    if (grid < 1) grid = 1;
+    LORACT_CUDA_TRY(launch_pdl(reduce_partials_vec4_kernel, dim3(grid), dim3(256), 0, stream, (const float4*)partials,
+                               n_partials, stride / 4, count4, (float4*)out_f32, (uint2*)out_bf16, gate));
+    count_launch(__func__, stream);
+    return cudaGetLastError();
+  }
   int grid = (int)((count + 255) / 256);
   if (grid > 148 * 16) grid = 148 * 16;
   if (grid < 1) grid = 1;

@@ -101,6 +101,8 @@ def measure(w: synth.Workload, reps: int, dev, flush) -> dict:
         row["compress_us"], row["compress_min_us"] = _median_us(run, reps, flush)
         target, _, _, U, V, _ = holder["out"]
     row["status"] = B.read_device_status(ws)
+    # rounds of the Gram-based orthonormalisation the device chose (fp32 inputs always take two)
+    row["rounds"] = B.round_gate_words(ws)[2] if w.dtype == "bf16" else 2
     row["rel_err"] = _rel_error(target, U, V)
 
     dW = torch.empty(d, g, dtype=torch.float32, device=dev)
@@ -167,7 +169,7 @@ COLUMNS = [("workload", "workload", "{}"), ("N", "N", "{}"), ("d", "d", "{}"), (
            ("wgrad_per_consumer_us", "wgrad per consumer us", "{:.0f}"), ("reconstruct_us", "reconstruct us", "{:.0f}"),
            ("gbs_of_x", "GB/s of X", "{:.0f}"), ("tokens_per_s", "tokens/s", "{:.3g}"),
            ("floor_us", "floor us", "{:.0f}"), ("frac_of_floor", "floor / time", "{:.3f}"),
-           ("rel_err", "rel. error", "{:.4f}"), ("rsvd_l", "RSVD l", "{}"), ("rsvd_us", "RSVD us", "{:.0f}"),
+           ("rel_err", "rel. error", "{:.4f}"), ("rounds", "rounds", "{}"), ("rsvd_l", "RSVD l", "{}"), ("rsvd_us", "RSVD us", "{:.0f}"),
            ("rsvd_truncate_us", "RSVD cut to r us", "{:.0f}"), ("rsvd_rel_err", "RSVD rel. error at rank r", "{:.4f}"), ("rsvd_status", "RSVD status", "{}"), ("status", "status", "{}")]
 
 
