@@ -29,7 +29,7 @@ loract_status_t loract_debug_gemm(int32_t M, int32_t N, int32_t K, int32_t a_mn,
 
 /* The same contraction with the sum of the terms before `halve_at_term` multiplied by 1/2 before that term's
  * products are added: C = (A_0 B_0 + ... ) / 2 + A_h B_h + ...  (0: the plain sum; must be < n_terms).  The tall Gram
- * products of the orthonormalisation use it with the pair {Yh^T Yh, Yh^T Yl}. */
+ * products of the orthonormalisation use it with {Yl^T Yl, Yh^T Yh, Yh^T Yl} and h = 2. */
 loract_status_t loract_debug_gemm_halved(int32_t M, int32_t N, int32_t K, int32_t a_mn, int32_t b_mn,
                                          const void* const* A, int64_t lda, const void* const* B, int64_t ldb,
                                          int32_t a_type, int32_t b_type, int32_t n_terms, int32_t halve_at_term,
@@ -38,7 +38,7 @@ loract_status_t loract_debug_gemm_halved(int32_t M, int32_t N, int32_t K, int32_
                                          void* stream);
 
 /* out (r x r, fp32, device) = S + S^T, S the sum in index order of `n_partials` r x r fp32 matrices `stride` elements
- * apart: the step that turns the partial sums of the two-term Gram product into the symmetric Gram matrix. */
+ * apart: the step that turns the partial sums of the halved-accumulator Gram product into the symmetric Gram matrix. */
 loract_status_t loract_debug_reduce_sym(const float* partials, int32_t n_partials, int64_t stride, int32_t r,
                                         float* out, void* stream);
 

@@ -191,3 +191,34 @@ def test_halved_accumulator_and_the_symmetric_gram_matrix_it_is_for(dev, engine,
         full = (Yh.double() + Yl.double()).t() @ (Yh.double() + Yl.double())
         assert float((W.double() - full).abs().max()) <= 6e-5 * scale * max(1.0, (n / 64) ** 0.5)
     B.debug_set_pair_mode(True)
+
+
+@pytest.mark.parametrize("r,n,splits", [(256, 8192, 128), (96, 1000, 16), (384, 3072, 48), (256, 8192, 32)])
+def test_three_term_gram_matrix_of_a_split_sketch(dev, r, n, splits):
+    # The form the orthonormalisation uses: D = (Yl^T Yl + Yh^T Yh) / 2 + Yh^T Yl per split, W = sum D + (sum D)^T,
+    # which is (Yh + Yl)^T (Yh + Yl) with all four products.  Against float64; the diagonal in particular, where
+    # leaving Yl^T Yl out would show as a relative deficit of about 2^-18 / 3 = 1.3e-6.
+    g = torch.Generator(device=dev)
+    g.manual_seed(3 * r + n)
+    Y = torch.randn(n, r, generator=g, device=dev) * torch.logspace(0, -2, r, device=dev)
+    Yh = Y.bfloat16()
+    Yl = (Y - Yh.float()).bfloat16()
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    P = B.debug_gemm([Yl, Yh, Yh], [Yl, Yh, Yl], r, r, n, True, True, out_mode=B.OUT_F32, engine=1, splits=splits,
+                     status=status, halve_at_term=2)
+    W = B.debug_reduce_sym(P.contiguous())
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(W, W.t())
+    Yd = Yh.double() + Yl.double()
+    full = Yd.t() @ Yd
+    sc = full.diagonal().sqrt()
+    rel = (W.double() - full) / (sc[:, None] * sc[None, :])
+    chain = -(-n // 64 // splits) * 12          # tensor-core instructions that add into one accumulator
+    # the tensor cores truncate: up to an ulp (2^-23 relative) per instruction of the chain, one-signed on the diagonal
+    # (about a quarter of that on average)
+    assert float(rel.abs().max()) <= 2.0 ** -23 * chain + 2e-7
+    without_ll = float((Yl.double() ** 2).sum(0).div(full.diagonal()).mean())
+    assert without_ll > 1e-6                                            # the term is not negligible ...
+    if chain == 12:                                                     # ... and with short chains one can see that it is in W
+        assert float(rel.diagonal().mean()) > -(2.0 ** -24) * chain - 1e-7

@@ -74,3 +74,20 @@ def test_non_finite_input_is_flagged_and_the_next_call_is_clean(dev, dtype):
     assert bool(torch.isfinite(U.float()).all()) and bool(torch.isfinite(V.float()).all())
     G = U.double().t() @ U.double()
     assert float((G - torch.eye(64, dtype=torch.float64, device=dev)).abs().max()) <= 4e-3
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_weight_grad_starts_from_a_clean_status_word(dev, dtype):
+    # The first kernel of loract_weight_grad clears the status word itself (tensor-core path) or a memset does
+    # (CUDA-core path): whatever an earlier call left there must not be reported for this one.
+    w = synth.scaled(synth.WORKLOADS["llama7b_block"], n_tokens=2048, d=512, rank=64, signal_rank=128)
+    inp = synth.make_inputs(w, device=dev)
+    X, G = inp["X"].to(dtype), inp["G"].to(dtype)
+    ws = B.alloc_workspace(B.make_desc(X, 64, w.seed), dev)
+    U, V, _ = B.compress(X, 64, seed=w.seed, ws=ws)
+    ws[0:4] = torch.tensor([0xEF, 0xBE, 0x00, 0x00], dtype=torch.uint8, device=dev)   # stale bits of some earlier call
+    torch.cuda.synchronize()
+    dW = B.weight_grad(U, V, G, ws=ws)
+    assert B.read_device_status(ws) == 0
+    ref = (U.double() @ V.double()).t() @ G.double()
+    assert float(torch.linalg.norm(dW.double() - ref) / torch.linalg.norm(ref)) <= 1e-3
