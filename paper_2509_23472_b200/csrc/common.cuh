@@ -113,6 +113,9 @@ struct GemmDesc {
   const uint32_t* gate = nullptr;
   // Tensor-core path: the launch stores zero into the status word before any of its waits can set a bit in it (the
   // first kernel of a call clears the word itself instead of a memset in front of it).
+  // fp32 32 x 32 tile kernel (gemm_f32_small_launch): optional bf16 hi / lo copies of the result (leading dimension ldc)
+  void* split_hi = nullptr;
+  void* split_lo = nullptr;
   bool clear_status = false;
   // Tensor-core path, OUT_SPLIT: a device word written by an earlier kernel; when it is zero only C0 (the leading bf16
   // part) is written and C1 keeps its old contents.
@@ -208,8 +211,10 @@ cudaError_t small_block_cluster_launch(const SmallBlockArgs& a, cudaStream_t str
 cudaError_t split_block_launch(const float* src, int rows, int cols, int64_t ld, __nv_bfloat16* hi,
                                __nv_bfloat16* lo, cudaStream_t stream, const uint32_t* gate = nullptr);
 // Zero fill of up to three ranges (16-byte aligned, sizes multiples of 16; a null range has size 0), one launch.
+// Optionally the same launch also forms sum_dst[i] = sum over n_src partials of sum_src[q * src_stride + i], i < count.
 cudaError_t zero3_gated_launch(void* a, size_t a_bytes, void* b, size_t b_bytes, void* c, size_t c_bytes,
-                               const uint32_t* gate, cudaStream_t stream);
+                               const uint32_t* gate, cudaStream_t stream, const float* sum_src = nullptr,
+                               int n_src = 0, int64_t src_stride = 0, int64_t count = 0, float* sum_dst = nullptr);
 cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_t stride,
                                    int64_t count, float* out_f32, __nv_bfloat16* out_bf16,
                                    cudaStream_t stream, const uint32_t* gate = nullptr);

@@ -29,6 +29,9 @@ struct SimtParams {
   float alpha;
   int halve_at_term;  // the sum so far is multiplied by 1/2 before this term (0: never)
   const uint32_t* gate;  // 32 x 32 tile kernel: optional device word, zero means the launch does nothing
+  // 32 x 32 tile kernel: optional bf16 hi / lo copies of the result, same leading dimension as C0
+  __nv_bfloat16* split_hi;
+  __nv_bfloat16* split_lo;
 };
 
 constexpr int kTile = 64;   // output tile 64 x 64, 256 threads, 4 x 4 outputs per thread
@@ -355,8 +358,14 @@ __global__ void __launch_bounds__(64 * kT32Groups) gemm_f32_tile32_kernel(SimtPa
 #pragma unroll
       for (int g2 = 1; g2 < kT32Groups; ++g2) sum += tiles[g2][0][(4 * tm + i) * kT32Ld + tn + 8 * j];
       float* c = (float*)p.C0 + (int64_t)m * p.ldc + n;
-      const float v = sum * p.alpha;
-      *c = p.accumulate ? (*c + v) : v;
+      const float v0 = sum * p.alpha;
+      const float v = p.accumulate ? (*c + v0) : v0;
+      *c = v;
+      if (p.split_hi) {
+        const __nv_bfloat16 h = __float2bfloat16(v);
+        p.split_hi[(int64_t)m * p.ldc + n] = h;
+        if (p.split_lo) p.split_lo[(int64_t)m * p.ldc + n] = __float2bfloat16(v - __bfloat162float(h));
+      }
     }
   }
 }
@@ -624,14 +633,22 @@ __global__ void __launch_bounds__(1024) round_gate_kernel(const float* __restric
   }
 }
 
-// Zero fill of up to three 16-byte aligned ranges (counts in 16-byte units), skipped when *gate == 0.
+// Zero fill of up to three 16-byte aligned ranges (counts in 16-byte units) and, in the same launch, an optional
+// fixed-order sum of partial matrices (dst[i] = sum_q src[q * stride + i], i < count; count 0: none).  Skipped when
+// *gate == 0.
 __global__ void zero3_gated_kernel(uint4* a, int64_t na, uint4* b, int64_t nb, uint4* c, int64_t nc,
-                                   const uint32_t* gate) {
+                                   const float* __restrict__ src, int n_src, int64_t src_stride, int64_t count,
+                                   float* __restrict__ dst, const uint32_t* gate) {
   pdl_wait();
   pdl_launch_dependents();
   if (gate != nullptr && *(const volatile uint32_t*)gate == 0u) return;
   const uint4 z = make_uint4(0u, 0u, 0u, 0u);
   const int64_t stride = (int64_t)gridDim.x * blockDim.x, t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (int64_t i = t0; i < count; i += stride) {
+    float sum = 0.f;
+    for (int q = 0; q < n_src; ++q) sum += src[(int64_t)q * src_stride + i];
+    dst[i] = sum;
+  }
   for (int64_t i = t0; i < na; i += stride) a[i] = z;
   for (int64_t i = t0; i < nb; i += stride) b[i] = z;
   for (int64_t i = t0; i < nc; i += stride) c[i] = z;
@@ -725,10 +742,12 @@ cudaError_t round_gate_launch(const float* W, const __nv_bfloat16* linv_hi, int 
 }
 
 cudaError_t zero3_gated_launch(void* a, size_t a_bytes, void* b, size_t b_bytes, void* c, size_t c_bytes,
-                               const uint32_t* gate, cudaStream_t stream) {
+                               const uint32_t* gate, cudaStream_t stream, const float* sum_src, int n_src,
+                               int64_t src_stride, int64_t count, float* sum_dst) {
   if (((uintptr_t)a | (uintptr_t)b | (uintptr_t)c | a_bytes | b_bytes | c_bytes) & 15) return cudaErrorInvalidValue;
   LORACT_CUDA_TRY(launch_pdl(zero3_gated_kernel, dim3(148), dim3(512), 0, stream, (uint4*)a, (int64_t)(a_bytes / 16),
-                             (uint4*)b, (int64_t)(b_bytes / 16), (uint4*)c, (int64_t)(c_bytes / 16), gate));
+                             (uint4*)b, (int64_t)(b_bytes / 16), (uint4*)c, (int64_t)(c_bytes / 16), sum_src, n_src,
+                             src_stride, sum_src ? count : (int64_t)0, sum_dst, gate));
   count_launch(__func__, stream);
   return cudaGetLastError();
 }
@@ -773,6 +792,8 @@ cudaError_t gemm_f32_small_launch(const GemmDesc& g, cudaStream_t stream, const 
     p.accumulate = g.accumulate ? 1 : 0;
     p.alpha = g.alpha;
     p.gate = nullptr;
+    p.split_hi = (__nv_bfloat16*)g.split_hi;
+    p.split_lo = (__nv_bfloat16*)g.split_lo;
     return true;
   };
   SimtParams p0, p1;

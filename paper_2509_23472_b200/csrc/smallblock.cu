@@ -335,10 +335,11 @@ cudaError_t factor_blocks(const TwoLevelCtx& c, float* W, float* X, __nv_bfloat1
   }
   LORACT_CUDA_TRY(factor_blocks(c, W22, X22, hi + (size_t)r1 * ld + r1, lo ? lo + (size_t)r1 * ld + r1 : nullptr, r2,
                                 Tnext, false));
-  // X21 = -X22 T2 : X21[m][n] = -sum_k X22[m][k] T2[k][n]
-  LORACT_CUDA_TRY(gemm_f32_small_launch(product(r2, r1, r2, X22, ld, T2, r1, true, X21, ld, -1.f, false), c.stream));
-  return split_block_launch(X21, r2, r1, ld, hi + (size_t)r1 * ld, lo ? lo + (size_t)r1 * ld : nullptr, c.stream,
-                            c.gate);
+  // X21 = -X22 T2 : X21[m][n] = -sum_k X22[m][k] T2[k][n], written as fp32 and as the bf16 pair in the same launch
+  GemmDesc last = product(r2, r1, r2, X22, ld, T2, r1, true, X21, ld, -1.f, false);
+  last.split_hi = hi + (size_t)r1 * ld;
+  last.split_lo = lo ? lo + (size_t)r1 * ld : nullptr;
+  return gemm_f32_small_launch(last, c.stream);
 }
 
 // scratch: W (r x r) + X (r x r) + the temporaries of every level, fp32.
@@ -347,11 +348,11 @@ cudaError_t small_block_two_level(const SmallBlockArgs& a, cudaStream_t stream) 
   float* W = (float*)a.scratch;
   float* X = a.linv_f32 ? a.linv_f32 : W + (size_t)r * r;
   float* T = W + 2 * (size_t)r * r;
-  LORACT_CUDA_TRY(reduce_partials_launch((const float*)a.partials, a.n_partials, a.partial_stride, (int64_t)r * r, W,
-                                         nullptr, stream, a.gate));
-  // blocks above the diagonal are never written below: X is read as a whole by the products of the next level up
+  // one launch: W = sum of the partials, and zeros where the blocks above the diagonal are never written below (X is
+  // read as a whole by the products of the next level up)
   LORACT_CUDA_TRY(zero3_gated_launch(X, (size_t)r * r * 4, a.linv_hi, (size_t)r * r * 2, a.linv_lo,
-                                     a.linv_lo ? (size_t)r * r * 2 : 0, a.gate, stream));
+                                     a.linv_lo ? (size_t)r * r * 2 : 0, a.gate, stream, (const float*)a.partials,
+                                     a.n_partials, a.partial_stride, (int64_t)r * r, W));
   TwoLevelCtx c;
   c.shift_rel = a.shift_rel; c.shift_diag_rel = a.shift_diag_rel; c.gate = a.gate; c.dev_status = a.dev_status; c.ld = r; c.scale_diag = W; c.scale_n = 256;
   c.stream = stream;
