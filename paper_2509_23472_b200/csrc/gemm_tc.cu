@@ -713,8 +713,13 @@ gemm_tc_pair_kernel(const __grid_constant__ TmapPack maps, const TcParams p) {
   const bool leader = cta_rank == 0;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int half_n = p.bn / 2;                               // B rows (or columns) this CTA loads
-  // grid: x = 128-row tiles (the two CTAs of a pair are neighbours in x), y = column tiles, z = K splits
-  const int n0 = blockIdx.y * p.bn, m0 = blockIdx.x * kBM, split = blockIdx.z;
+  // grid: x = 128-row tiles (the two CTAs of a pair are neighbours in x), y = column tiles, z = K splits.  CTAs start
+  // in the order x, then y; the tile a pair works on is taken from that order with the column tile running fastest,
+  // so that the pairs that share a row tile of A (pass 1 at r = 512: the same 256 rows of X, two column tiles) run
+  // side by side and the second one finds those rows in L2 instead of streaming X from HBM a second time.
+  const int pair_lin = (int)(blockIdx.x >> 1) + (int)(gridDim.x >> 1) * (int)blockIdx.y;
+  const int tile_m = pair_lin / (int)gridDim.y, tile_n = pair_lin - tile_m * (int)gridDim.y;
+  const int n0 = tile_n * p.bn, m0 = (2 * tile_m + (int)cta_rank) * kBM, split = blockIdx.z;
   const int kb_begin = split * p.kb_per_split;
   const int kb_count = max(0, min(p.kb_total, kb_begin + p.kb_per_split) - kb_begin);
   int n_iter = kb_count * p.n_terms;
