@@ -689,8 +689,10 @@ cudaError_t gemm_simt_launch(const GemmDesc& g, cudaStream_t stream) {
 cudaError_t reduce_partials_launch(const float* partials, int n_partials, int64_t stride,
                                    int64_t count, float* out_f32, __nv_bfloat16* out_bf16,
                                    cudaStream_t stream, const uint32_t* gate) {
-  const bool vec = count % 4 == 0 && stride % 4 == 0 && (((uintptr_t)partials | (uintptr_t)out_f32) & 15) == 0 &&
-                   ((uintptr_t)out_bf16 & 7) == 0;
+  // four elements per thread only where that still leaves a few CTAs per SM (a small matrix is summed faster by
+  // more threads with one element each)
+  const bool vec = count >= (1 << 18) && count % 4 == 0 && stride % 4 == 0 &&
+                   (((uintptr_t)partials | (uintptr_t)out_f32) & 15) == 0 && ((uintptr_t)out_bf16 & 7) == 0;
   if (vec) {
     const int64_t count4 = count / 4;
     int grid = (int)((count4 + 255) / 256);
